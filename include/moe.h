@@ -1,0 +1,181 @@
+/*
+ * moe.h -- C ABI of the B200 (sm_100a) MoE forward library, EP=1 on one GPU.
+ *
+ * The calls restate the expert-parallel problem the paper analyses (Sec. 2.2: token hidden vectors are
+ * sent to their experts, expert outputs are returned to the rank that owns the token; Sec. 4.3: the fused
+ * kernel is Dispatch, Linear-1, Linear-2 and a Combine buffer written by the Linear-2 epilogue), run with
+ * a single rank.  The per-expert receive buffer (x_perm) and the combine buffer (y_perm) that the paper's
+ * kernels reach with remote stores are ordinary allocations in this GPU's HBM, separate from x and out.
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers unless the parameter name ends in _host.  The caller owns
+ *     every buffer; the library keeps no reference after the call's work has finished on the stream.
+ *   - bf16 tensors are passed as void* (2 bytes per element, row-major, innermost dimension contiguous).
+ *   - Pointers must be 16-byte aligned.  H and F must be multiples of 64; 1 <= k <= min(E, 32); E <= 1024.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls are asynchronous:
+ *     they enqueue work and return.  Argument and shape errors are returned synchronously, before any
+ *     launch.  Errors detected on the device (a bounded wait that expired) are written to a status word
+ *     read by moe_last_device_status; kernels never trap.
+ *   - The context's device must be the calling thread's current device.
+ *   - Notation: T tokens, H hidden, F per-expert ffn width, E experts, k experts per token, R = T*k rows.
+ */
+#ifndef MOE_B200_H_
+#define MOE_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = 1,         /* null pointer, misaligned pointer, wrong device, bad tuning value */
+  MOE_ERR_UNSUPPORTED_SHAPE = 2,   /* H or F not a multiple of 64, k or E out of range, T < 0 */
+  MOE_ERR_WORKSPACE_TOO_SMALL = 3,
+  MOE_ERR_BAD_ROUTING = 4,         /* reserved: routing input violates the contract */
+  MOE_ERR_CUDA = 5,                /* a CUDA runtime or driver call failed */
+  MOE_ERR_TIMEOUT = 6,             /* device status only: a bounded on-device wait expired */
+  MOE_ERR_UNSUPPORTED = 7          /* ep_size != 1, unknown schedule */
+} moe_status;
+
+typedef struct {
+  int32_t T, H, F, E, k;
+  int32_t ep_size, ep_rank;        /* must be 1 and 0: nothing is sharded across GPUs */
+} moe_shape;
+
+/*
+ * Store pacing of the grouped-GEMM epilogue: the one part of the paper's burst/gap idea (Sec. 3.1: a
+ * producer emits a burst, then an interval with no stores; Eq. 1) that has a meaning on local HBM.
+ * A "store tile" is 128 rows x 32 output columns of bf16 (8 KiB), the unit one pass of the four epilogue
+ * warps drains from tensor memory.  A burst is `store_burst_tiles` store tiles issued back to back by a
+ * CTA.  interleave_mode 0 ("after-mainloop"): bursts follow one another with no enforced gap.
+ * interleave_mode 1 ("every-k-iterations"): after each burst the epilogue holds further stores until the
+ * MMA warp has issued `interleave_k` more 64-deep K-blocks of the next tile's mainloop (or has nothing
+ * left to issue).  Pacing never changes values: outputs are bitwise identical for every setting.
+ */
+typedef struct {
+  int32_t store_burst_tiles;       /* 1, 2, 4, 8 or 16 (values above the tiles in one output tile act as that count) */
+  int32_t interleave_mode;         /* 0 or 1 */
+  int32_t interleave_k;            /* 1, 2 or 4; used when interleave_mode == 1 */
+  int32_t schedule;                /* 0 = expert-wave order (Sec. 4.3): all Linear-1 tiles, then Linear-2 */
+  int32_t dep_lead_D;              /* reserved for the interleaved schedule (Algorithm 1); must be 0 */
+  int32_t debug_flags;             /* must be 0 */
+} moe_tuning;
+
+/* Byte offsets of the slices of the workspace used by moe_fused_forward (each 256-byte aligned). */
+typedef struct {
+  size_t topk_ids;   /* int32 [T,k]  */
+  size_t topk_w;     /* fp32  [T,k]  */
+  size_t counts;     /* int32 [E]    */
+  size_t offsets;    /* int32 [E+1]  */
+  size_t perm;       /* int32 [R]    */
+  size_t inv_perm;   /* int32 [R]    */
+  size_t x_perm;     /* bf16  [R,H]  expert-contiguous receive buffer (Dispatch) */
+  size_t h;          /* bf16  [R,F]  Linear-1 output after SiLU*mul */
+  size_t y_perm;     /* bf16  [R,H]  combine buffer written by the Linear-2 epilogue */
+  size_t x_stage;    /* bf16  [T,H]  device staging for moe_fused_forward_host */
+  size_t logits_stage; /* fp32 [T,E] device staging for moe_fused_forward_host */
+  size_t out_stage;  /* bf16  [T,H]  device staging for moe_fused_forward_host */
+  size_t total;      /* = moe_workspace_bytes */
+} moe_workspace_layout;
+
+typedef struct moe_ctx moe_ctx;    /* opaque: shape, device, SM count, small device scratch */
+
+/* Human-readable name of a status code.  Never NULL. */
+const char* moe_status_string(moe_status s);
+
+/*
+ * Create a context for one layer shape on `device` (must be the current device).  Allocates the small
+ * device scratch the routing kernels need (per-chunk histograms, a status word); no later call allocates.
+ * Errors: INVALID_ARG, UNSUPPORTED_SHAPE, UNSUPPORTED (ep_size != 1), CUDA.
+ */
+moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device);
+void moe_destroy(moe_ctx* ctx);
+
+/* Size and slicing of the caller-provided workspace of moe_fused_forward.  Returns 0 / fills zeros for a
+ * shape moe_create would reject. */
+size_t moe_workspace_bytes(const moe_shape* shape);
+moe_status moe_get_workspace_layout(const moe_shape* shape, moe_workspace_layout* out_layout);
+
+/*
+ * Routing plan (the Dispatch bookkeeping of Sec. 4.3; the paper leaves routing unchanged, Sec. 7).
+ * For each token: the k largest logits (ties to the lower expert index), slots in descending-logit
+ * order, weights = softmax over the k selected logits (fp32).  Then per-expert counts, exclusive
+ * offsets, and the stable permutation: flat slot s = t*k+j is placed at row offsets[e] + (number of
+ * slots s' < s with the same expert).  perm[row] = s, inv_perm[s] = row.
+ *   logits [T,E] fp32 (finite)  ->  topk_ids [T,k] int32, topk_w [T,k] fp32, counts [E] int32,
+ *   offsets [E+1] int32, perm [R] int32, inv_perm [R] int32.
+ * T == 0 writes zero counts/offsets and launches nothing else.
+ */
+moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids, float* topk_w,
+                            int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
+                            void* stream);
+
+/*
+ * Dispatch (Sec. 2.2 / Sec. 4.3 "Dispatch input"): x_perm[inv_perm[t*k+j], :] = x[t, :] for every slot,
+ * i.e. x_perm[row, :] = x[perm[row] div k, :].  Each token row is read once and written k times with
+ * 16-byte accesses.   x [T,H] bf16, inv_perm [R] int32 -> x_perm [R,H] bf16 (bit-exact copies).
+ */
+moe_status moe_dispatch(moe_ctx* ctx, const void* x, const int32_t* inv_perm, void* x_perm, void* stream);
+
+/*
+ * Expert feed-forward over the expert-contiguous buffer (Sec. 4.3 "Linear-1", "Linear-2"; Linear-1 is
+ * twice the intermediate width, App. A.2, i.e. a gate half and an up half).  For expert e and its rows
+ * offsets[e] <= r < offsets[e+1]:
+ *     h[r,f] = silu(sum_c x_perm[r,c] w_gate[e,f,c]) * (sum_c x_perm[r,c] w_up[e,f,c])      (bf16 out)
+ *     y_perm[r,c] = sum_f h[r,f] w_down[e,c,f]                                               (bf16 out)
+ * bf16 operands, fp32 accumulation in tensor memory, outputs rounded to nearest even.
+ *   x_perm [R,H] bf16, offsets [E+1] int32, w_gate/w_up [E,F,H] bf16, w_down [E,H,F] bf16
+ *   -> h_ws [R,F] bf16 (also the Linear-2 input), y_perm [R,H] bf16.
+ *   h_fp32_debug: NULL, or fp32 [R,F] that receives h before its rounding to bf16.
+ *   tuning: NULL for defaults {1,0,1,0,0,0}.
+ * Rows of empty experts do not exist; rows outside every expert are never written.
+ */
+moe_status moe_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* offsets, const void* w_gate,
+                          const void* w_up, const void* w_down, void* h_ws, void* y_perm,
+                          float* h_fp32_debug, const moe_tuning* tuning, void* stream);
+
+/*
+ * Combine (Sec. 2.2: expert outputs return to the token's owner; Sec. 4.3 "Combine buffer"):
+ *     out[t,:] = bf16( sum_{j=0..k-1} topk_w[t,j] * float(y_perm[inv_perm[t*k+j], :]) )
+ * summed in ascending j with fp32 accumulation: deterministic, no atomics.
+ *   y_perm [R,H] bf16, inv_perm [R] int32, topk_w [T,k] fp32 -> out [T,H] bf16.
+ */
+moe_status moe_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_perm, const float* topk_w,
+                       void* out, void* stream);
+
+/*
+ * The whole layer on one stream: plan_routing, dispatch, expert_ffn, combine (Sec. 4.3, the fused
+ * Dispatch + Linear-1 + Linear-2 + Combine path).  Intermediates live in `workspace` at the offsets
+ * moe_get_workspace_layout reports.  Errors: as the four calls, plus WORKSPACE_TOO_SMALL.
+ */
+moe_status moe_fused_forward(moe_ctx* ctx, const void* x, const float* logits, const void* w_gate,
+                             const void* w_up, const void* w_down, void* out, void* workspace,
+                             size_t workspace_bytes, const moe_tuning* tuning, void* stream);
+
+/*
+ * Same, with the per-step tensors in HOST memory (pinned memory makes the copies asynchronous):
+ * x_host [T,H] bf16 and logits_host [T,E] fp32 are copied to the workspace's staging slices, the layer
+ * runs, and out [T,H] bf16 is copied back to out_host, all on `stream`.  Expert weights stay on the
+ * device.  The caller synchronises the stream before reading out_host.
+ */
+moe_status moe_fused_forward_host(moe_ctx* ctx, const void* x_host, const float* logits_host,
+                                  const void* w_gate, const void* w_up, const void* w_down,
+                                  void* out_host, void* workspace, size_t workspace_bytes,
+                                  const moe_tuning* tuning, void* stream);
+
+/*
+ * Synchronise `stream`, then read and clear the device status word.  *code is MOE_OK or MOE_ERR_TIMEOUT;
+ * *detail identifies the wait that gave up (kernel id * 65536 + role).  Blocking.
+ */
+moe_status moe_last_device_status(moe_ctx* ctx, int32_t* code, int32_t* detail, void* stream);
+
+/* Number of kernels the last call on this context launched (host-side count, for benchmarking). */
+int32_t moe_last_launch_count(const moe_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H_ */

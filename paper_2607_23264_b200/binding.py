@@ -1,0 +1,214 @@
+"""ctypes binding of libmoe_b200.so: the same names as include/moe.h, argument marshalling only.
+
+Tensors are torch CUDA tensors (torch is used for device memory and streams); bf16 buffers are
+``torch.bfloat16`` (or int16/uint16 views of the same bytes).  Every step of the path runs inside the
+library's kernels.  Loading fails loudly when the library has not been built: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmoe_b200.so")
+
+MOE_OK = 0
+STATUS_NAMES = {
+    0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED_SHAPE", 3: "MOE_ERR_WORKSPACE_TOO_SMALL",
+    4: "MOE_ERR_BAD_ROUTING", 5: "MOE_ERR_CUDA", 6: "MOE_ERR_TIMEOUT", 7: "MOE_ERR_UNSUPPORTED",
+}
+
+EXPORTS = (
+    "moe_status_string", "moe_create", "moe_destroy", "moe_workspace_bytes", "moe_get_workspace_layout",
+    "moe_plan_routing", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_fused_forward",
+    "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count",
+)
+
+
+class MoeError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)}")
+
+
+class moe_shape(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("T", "H", "F", "E", "k", "ep_size", "ep_rank")]
+
+
+class moe_tuning(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("store_burst_tiles", "interleave_mode", "interleave_k", "schedule",
+                                         "dep_lead_D", "debug_flags")]
+
+
+class moe_workspace_layout(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("topk_ids", "topk_w", "counts", "offsets", "perm", "inv_perm", "x_perm",
+                                          "h", "y_perm", "x_stage", "logits_stage", "out_stage", "total")]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """dlopen the library (once) and declare the prototypes.  Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2607_23264_b200.build` "
+            "(the MoE path has no CPU or PyTorch fallback)")
+    lib = C.CDLL(_LIB_PATH)
+    vp, i32p, f32p = C.c_void_p, C.c_void_p, C.c_void_p
+    lib.moe_status_string.restype = C.c_char_p
+    lib.moe_status_string.argtypes = [C.c_int]
+    lib.moe_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(moe_shape), C.c_int]
+    lib.moe_destroy.argtypes = [C.c_void_p]
+    lib.moe_destroy.restype = None
+    lib.moe_workspace_bytes.argtypes = [C.POINTER(moe_shape)]
+    lib.moe_workspace_bytes.restype = C.c_size_t
+    lib.moe_get_workspace_layout.argtypes = [C.POINTER(moe_shape), C.POINTER(moe_workspace_layout)]
+    lib.moe_plan_routing.argtypes = [vp, f32p, i32p, f32p, i32p, i32p, i32p, i32p, vp]
+    lib.moe_dispatch.argtypes = [vp, vp, i32p, vp, vp]
+    lib.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp, f32p, C.POINTER(moe_tuning), vp]
+    lib.moe_combine.argtypes = [vp, vp, i32p, f32p, vp, vp]
+    lib.moe_fused_forward.argtypes = [vp, vp, f32p, vp, vp, vp, vp, vp, C.c_size_t, C.POINTER(moe_tuning), vp]
+    lib.moe_fused_forward_host.argtypes = [vp, vp, f32p, vp, vp, vp, vp, vp, C.c_size_t, C.POINTER(moe_tuning), vp]
+    lib.moe_last_device_status.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
+    lib.moe_last_launch_count.argtypes = [vp]
+    lib.moe_last_launch_count.restype = C.c_int32
+    for name in EXPORTS:
+        if name not in ("moe_status_string", "moe_destroy", "moe_workspace_bytes", "moe_last_launch_count"):
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    """Device (or host) address of a tensor, None -> NULL."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return C.c_void_p(t)
+    if not t.is_contiguous():
+        raise ValueError("tensors passed to the MoE library must be contiguous")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _check(code: int, where: str):
+    if code != MOE_OK:
+        raise MoeError(code, where)
+
+
+def make_tuning(store_burst_tiles=1, interleave_mode=0, interleave_k=1, schedule=0, dep_lead_D=0, debug_flags=0):
+    return moe_tuning(store_burst_tiles, interleave_mode, interleave_k, schedule, dep_lead_D, debug_flags)
+
+
+def _tuning_ref(tuning):
+    return None if tuning is None else C.byref(tuning)
+
+
+def moe_status_string(code: int) -> str:
+    return load_library().moe_status_string(code).decode()
+
+
+def moe_workspace_bytes(T, H, F, E, k) -> int:
+    return load_library().moe_workspace_bytes(C.byref(moe_shape(T, H, F, E, k, 1, 0)))
+
+
+def moe_get_workspace_layout(T, H, F, E, k) -> dict:
+    L = moe_workspace_layout()
+    _check(load_library().moe_get_workspace_layout(C.byref(moe_shape(T, H, F, E, k, 1, 0)), C.byref(L)),
+           "moe_get_workspace_layout")
+    return {n: getattr(L, n) for n, _ in moe_workspace_layout._fields_}
+
+
+@dataclass
+class Context:
+    """Owner of a moe_ctx*; methods carry the C function names."""
+    T: int
+    H: int
+    F: int
+    E: int
+    k: int
+    device: int = 0
+    ep_size: int = 1
+    ep_rank: int = 0
+
+    def __post_init__(self):
+        import torch
+        self._lib = load_library()
+        self._handle = C.c_void_p()
+        torch.cuda.set_device(self.device)
+        torch.cuda.init()
+        torch.zeros(1, device=f"cuda:{self.device}")  # make sure the primary context exists and is current
+        shape = moe_shape(self.T, self.H, self.F, self.E, self.k, self.ep_size, self.ep_rank)
+        _check(self._lib.moe_create(C.byref(self._handle), C.byref(shape), self.device), "moe_create")
+
+    @property
+    def R(self):
+        return self.T * self.k
+
+    def close(self):
+        if getattr(self, "_handle", None) and self._handle.value:
+            self._lib.moe_destroy(self._handle)
+            self._handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def workspace_bytes(self) -> int:
+        return moe_workspace_bytes(self.T, self.H, self.F, self.E, self.k)
+
+    def workspace_layout(self) -> dict:
+        return moe_get_workspace_layout(self.T, self.H, self.F, self.E, self.k)
+
+    def moe_plan_routing(self, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, stream=None):
+        _check(self._lib.moe_plan_routing(self._handle, _ptr(logits), _ptr(topk_ids), _ptr(topk_w), _ptr(counts),
+                                          _ptr(offsets), _ptr(perm), _ptr(inv_perm), _stream(stream)),
+               "moe_plan_routing")
+
+    def moe_dispatch(self, x, inv_perm, x_perm, stream=None):
+        _check(self._lib.moe_dispatch(self._handle, _ptr(x), _ptr(inv_perm), _ptr(x_perm), _stream(stream)),
+               "moe_dispatch")
+
+    def moe_expert_ffn(self, x_perm, offsets, w_gate, w_up, w_down, h_ws, y_perm, h_fp32_debug=None, tuning=None,
+                       stream=None):
+        _check(self._lib.moe_expert_ffn(self._handle, _ptr(x_perm), _ptr(offsets), _ptr(w_gate), _ptr(w_up),
+                                        _ptr(w_down), _ptr(h_ws), _ptr(y_perm), _ptr(h_fp32_debug),
+                                        _tuning_ref(tuning), _stream(stream)), "moe_expert_ffn")
+
+    def moe_combine(self, y_perm, inv_perm, topk_w, out, stream=None):
+        _check(self._lib.moe_combine(self._handle, _ptr(y_perm), _ptr(inv_perm), _ptr(topk_w), _ptr(out),
+                                     _stream(stream)), "moe_combine")
+
+    def moe_fused_forward(self, x, logits, w_gate, w_up, w_down, out, workspace, tuning=None, stream=None):
+        _check(self._lib.moe_fused_forward(self._handle, _ptr(x), _ptr(logits), _ptr(w_gate), _ptr(w_up),
+                                           _ptr(w_down), _ptr(out), _ptr(workspace),
+                                           workspace.numel() * workspace.element_size(), _tuning_ref(tuning),
+                                           _stream(stream)), "moe_fused_forward")
+
+    def moe_fused_forward_host(self, x_host, logits_host, w_gate, w_up, w_down, out_host, workspace, tuning=None,
+                               stream=None):
+        _check(self._lib.moe_fused_forward_host(self._handle, _ptr(x_host), _ptr(logits_host), _ptr(w_gate),
+                                                _ptr(w_up), _ptr(w_down), _ptr(out_host), _ptr(workspace),
+                                                workspace.numel() * workspace.element_size(), _tuning_ref(tuning),
+                                                _stream(stream)), "moe_fused_forward_host")
+
+    def moe_last_device_status(self, stream=None):
+        code, detail = C.c_int32(0), C.c_int32(0)
+        _check(self._lib.moe_last_device_status(self._handle, C.byref(code), C.byref(detail), _stream(stream)),
+               "moe_last_device_status")
+        return code.value, detail.value
+
+    def moe_last_launch_count(self) -> int:
+        return self._lib.moe_last_launch_count(self._handle)

@@ -1,0 +1,295 @@
+// Host side of the C ABI (include/moe.h): argument validation, context, workspace carving, call order.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "moe_internal.h"
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+moe_status check_shape(const moe_shape* s) {
+  if (!s) return MOE_ERR_INVALID_ARG;
+  if (s->ep_size != 1 || s->ep_rank != 0) return MOE_ERR_UNSUPPORTED;
+  if (s->T < 0 || s->H <= 0 || s->F <= 0 || s->E <= 0 || s->k <= 0) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (s->H % 64 != 0 || s->F % 64 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (s->E > 1024 || s->k > 32 || s->k > s->E) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (static_cast<long long>(s->T) * s->k > 0x7FFFFFFFLL / 2) return MOE_ERR_UNSUPPORTED_SHAPE;
+  return MOE_OK;
+}
+
+moe_status check_tuning(const moe_tuning* t) {
+  if (!t) return MOE_OK;
+  const int b = t->store_burst_tiles;
+  if (!(b == 1 || b == 2 || b == 4 || b == 8 || b == 16)) return MOE_ERR_INVALID_ARG;
+  if (t->interleave_mode != 0 && t->interleave_mode != 1) return MOE_ERR_INVALID_ARG;
+  if (!(t->interleave_k == 1 || t->interleave_k == 2 || t->interleave_k == 4)) return MOE_ERR_INVALID_ARG;
+  if (t->schedule != 0) return MOE_ERR_UNSUPPORTED;
+  if (t->dep_lead_D != 0 || t->debug_flags != 0) return MOE_ERR_INVALID_ARG;
+  return MOE_OK;
+}
+
+moe_status check_ctx(const moe_ctx* ctx) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+  return dev == ctx->device ? MOE_OK : MOE_ERR_INVALID_ARG;
+}
+
+inline size_t up256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+
+void fill_layout(const moe_shape& s, moe_workspace_layout* L) {
+  const size_t T = s.T, H = s.H, F = s.F, E = s.E, k = s.k, R = T * k;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t at = off; off += up256(bytes); return at; };
+  L->topk_ids = take(R * 4);
+  L->topk_w = take(R * 4);
+  L->counts = take(E * 4);
+  L->offsets = take((E + 1) * 4);
+  L->perm = take(R * 4);
+  L->inv_perm = take(R * 4);
+  L->x_perm = take(R * H * 2);
+  L->h = take(R * F * 2);
+  L->y_perm = take(R * H * 2);
+  L->x_stage = take(T * H * 2);
+  L->logits_stage = take(T * E * 4);
+  L->out_stage = take(T * H * 2);
+  L->total = off;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* moe_status_string(moe_status s) {
+  switch (s) {
+    case MOE_OK: return "MOE_OK";
+    case MOE_ERR_INVALID_ARG: return "MOE_ERR_INVALID_ARG";
+    case MOE_ERR_UNSUPPORTED_SHAPE: return "MOE_ERR_UNSUPPORTED_SHAPE";
+    case MOE_ERR_WORKSPACE_TOO_SMALL: return "MOE_ERR_WORKSPACE_TOO_SMALL";
+    case MOE_ERR_BAD_ROUTING: return "MOE_ERR_BAD_ROUTING";
+    case MOE_ERR_CUDA: return "MOE_ERR_CUDA";
+    case MOE_ERR_TIMEOUT: return "MOE_ERR_TIMEOUT";
+    case MOE_ERR_UNSUPPORTED: return "MOE_ERR_UNSUPPORTED";
+  }
+  return "MOE_ERR_UNKNOWN";
+}
+
+size_t moe_workspace_bytes(const moe_shape* shape) {
+  if (check_shape(shape) != MOE_OK) return 0;
+  moe_workspace_layout L;
+  fill_layout(*shape, &L);
+  return L.total;
+}
+
+moe_status moe_get_workspace_layout(const moe_shape* shape, moe_workspace_layout* out_layout) {
+  if (!out_layout) return MOE_ERR_INVALID_ARG;
+  std::memset(out_layout, 0, sizeof(*out_layout));
+  const moe_status st = check_shape(shape);
+  if (st != MOE_OK) return st;
+  fill_layout(*shape, out_layout);
+  return MOE_OK;
+}
+
+moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
+  if (!out_ctx) return MOE_ERR_INVALID_ARG;
+  *out_ctx = nullptr;
+  const moe_status st = check_shape(shape);
+  if (st != MOE_OK) return st;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+  if (dev != device) return MOE_ERR_INVALID_ARG;
+
+  moe_ctx* ctx = new (std::nothrow) moe_ctx();
+  if (!ctx) return MOE_ERR_CUDA;
+  ctx->shape = *shape;
+  ctx->device = device;
+  ctx->last_launches = 0;
+  if (cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+    delete ctx;
+    return MOE_ERR_CUDA;
+  }
+  ctx->tokens_per_chunk = kRouteThreads / shape->k;   // k <= 32, so at least 8 tokens
+  ctx->num_chunks = shape->T ? (shape->T + ctx->tokens_per_chunk - 1) / ctx->tokens_per_chunk : 0;
+  const size_t hist_elems = static_cast<size_t>(ctx->num_chunks ? ctx->num_chunks : 1) * shape->E;
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) {
+    delete ctx;
+    return MOE_ERR_CUDA;
+  }
+  ctx->encode_tiled = reinterpret_cast<moe_encode_tiled_fn>(fn);
+
+  bool ok = cudaMalloc(&ctx->d_chunk_hist, hist_elems * 4) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_chunk_base, hist_elems * 4) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_status, 2 * 4) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->d_status, 0, 2 * 4) == cudaSuccess;
+  ok = ok && moe::prepare_expert_ffn(ctx) == cudaSuccess;
+  if (!ok) {
+    moe_destroy(ctx);
+    return MOE_ERR_CUDA;
+  }
+  *out_ctx = ctx;
+  return MOE_OK;
+}
+
+void moe_destroy(moe_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->d_chunk_hist) cudaFree(ctx->d_chunk_hist);
+  if (ctx->d_chunk_base) cudaFree(ctx->d_chunk_base);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  delete ctx;
+}
+
+moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids, float* topk_w,
+                            int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
+                            void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  ctx->last_launches = 0;
+  const moe_shape& s = ctx->shape;
+  if (!counts || !offsets) return MOE_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (s.T == 0) {
+    if (cudaMemsetAsync(counts, 0, static_cast<size_t>(s.E) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaMemsetAsync(offsets, 0, static_cast<size_t>(s.E + 1) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+  }
+  if (!logits || !topk_ids || !topk_w || !perm || !inv_perm) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(logits) || !aligned16(topk_ids) || !aligned16(topk_w) || !aligned16(counts) ||
+      !aligned16(offsets) || !aligned16(perm) || !aligned16(inv_perm))
+    return MOE_ERR_INVALID_ARG;
+  return moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_dispatch(moe_ctx* ctx, const void* x, const int32_t* inv_perm, void* x_perm, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  ctx->last_launches = 0;
+  if (ctx->shape.T == 0) return MOE_OK;
+  if (!x || !inv_perm || !x_perm) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(inv_perm) || !aligned16(x_perm)) return MOE_ERR_INVALID_ARG;
+  return moe::launch_dispatch(ctx, x, inv_perm, x_perm, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* offsets, const void* w_gate,
+                          const void* w_up, const void* w_down, void* h_ws, void* y_perm,
+                          float* h_fp32_debug, const moe_tuning* tuning, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  ctx->last_launches = 0;
+  st = check_tuning(tuning);
+  if (st != MOE_OK) return st;
+  if (ctx->shape.T == 0) return MOE_OK;
+  if (!x_perm || !offsets || !w_gate || !w_up || !w_down || !h_ws || !y_perm) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x_perm) || !aligned16(offsets) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) ||
+      !aligned16(h_ws) || !aligned16(y_perm) || !aligned16(h_fp32_debug))
+    return MOE_ERR_INVALID_ARG;
+  return moe::launch_expert_ffn(ctx, x_perm, offsets, w_gate, w_up, w_down, h_ws, y_perm, h_fp32_debug, tuning,
+                                static_cast<cudaStream_t>(stream));
+}
+
+moe_status moe_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_perm, const float* topk_w,
+                       void* out, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  ctx->last_launches = 0;
+  if (ctx->shape.T == 0) return MOE_OK;
+  if (!y_perm || !inv_perm || !topk_w || !out) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(y_perm) || !aligned16(inv_perm) || !aligned16(topk_w) || !aligned16(out)) return MOE_ERR_INVALID_ARG;
+  return moe::launch_combine(ctx, y_perm, inv_perm, topk_w, out, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_fused_forward(moe_ctx* ctx, const void* x, const float* logits, const void* w_gate,
+                             const void* w_up, const void* w_down, void* out, void* workspace,
+                             size_t workspace_bytes, const moe_tuning* tuning, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  ctx->last_launches = 0;
+  st = check_tuning(tuning);
+  if (st != MOE_OK) return st;
+  const moe_shape& s = ctx->shape;
+  if (s.T == 0) return MOE_OK;
+  if (!x || !logits || !w_gate || !w_up || !w_down || !out || !workspace) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(logits) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) ||
+      !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+    return MOE_ERR_INVALID_ARG;
+  moe_workspace_layout L;
+  fill_layout(s, &L);
+  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE_TOO_SMALL;
+
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  int32_t* topk_ids = reinterpret_cast<int32_t*>(ws + L.topk_ids);
+  float* topk_w = reinterpret_cast<float*>(ws + L.topk_w);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+  int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
+  int32_t* perm = reinterpret_cast<int32_t*>(ws + L.perm);
+  int32_t* inv_perm = reinterpret_cast<int32_t*>(ws + L.inv_perm);
+  void* x_perm = ws + L.x_perm;
+  void* h = ws + L.h;
+  void* y_perm = ws + L.y_perm;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+  if (moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (moe::launch_dispatch(ctx, x, inv_perm, x_perm, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  st = moe::launch_expert_ffn(ctx, x_perm, offsets, w_gate, w_up, w_down, h, y_perm, nullptr, tuning, cs);
+  if (st != MOE_OK) return st;
+  if (moe::launch_combine(ctx, y_perm, inv_perm, topk_w, out, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+moe_status moe_fused_forward_host(moe_ctx* ctx, const void* x_host, const float* logits_host,
+                                  const void* w_gate, const void* w_up, const void* w_down,
+                                  void* out_host, void* workspace, size_t workspace_bytes,
+                                  const moe_tuning* tuning, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  const moe_shape& s = ctx->shape;
+  if (s.T == 0) { ctx->last_launches = 0; return MOE_OK; }
+  if (!x_host || !logits_host || !out_host || !workspace) return MOE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MOE_ERR_INVALID_ARG;
+  moe_workspace_layout L;
+  fill_layout(s, &L);
+  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE_TOO_SMALL;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const size_t act_bytes = static_cast<size_t>(s.T) * s.H * 2;
+  const size_t logit_bytes = static_cast<size_t>(s.T) * s.E * 4;
+  if (cudaMemcpyAsync(ws + L.x_stage, x_host, act_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  if (cudaMemcpyAsync(ws + L.logits_stage, logits_host, logit_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  st = moe_fused_forward(ctx, ws + L.x_stage, reinterpret_cast<const float*>(ws + L.logits_stage), w_gate, w_up,
+                         w_down, ws + L.out_stage, workspace, workspace_bytes, tuning, stream);
+  if (st != MOE_OK) return st;
+  if (cudaMemcpyAsync(out_host, ws + L.out_stage, act_bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+moe_status moe_last_device_status(moe_ctx* ctx, int32_t* code, int32_t* detail, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  if (!code || !detail) return MOE_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  int32_t host[2] = {0, 0};
+  if (cudaMemcpyAsync(host, ctx->d_status, sizeof(host), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->d_status, 0, sizeof(host), cs) != cudaSuccess) return MOE_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return MOE_ERR_CUDA;
+  *code = host[0];
+  *detail = host[1];
+  return MOE_OK;
+}
+
+int32_t moe_last_launch_count(const moe_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,50 @@
+// Internal declarations shared by the translation units of the library (not part of the C ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/moe.h"
+
+// Rows per M tile of the grouped GEMM and slots per routing chunk.
+constexpr int kRouteThreads = 256;
+
+typedef CUresult (*moe_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                        const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                        CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                        CUtensorMapFloatOOBfill);
+
+struct moe_ctx {
+  moe_shape shape;
+  int device;
+  int num_sms;
+  int tokens_per_chunk;  // routing: tokens handled by one CTA, so that a chunk has at most 256 slots
+  int num_chunks;
+  int32_t* d_chunk_hist;  // [num_chunks, E] slots of each chunk per expert
+  int32_t* d_chunk_base;  // [num_chunks, E] exclusive prefix of d_chunk_hist over chunks
+  int32_t* d_status;      // [2] device status word: code, detail
+  moe_encode_tiled_fn encode_tiled;
+  int32_t last_launches;
+};
+
+// Launchers (each returns the cudaError_t of its launches).  `stream` is the caller's stream.
+namespace moe {
+
+cudaError_t launch_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids, float* topk_w,
+                                int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
+                                cudaStream_t stream);
+
+cudaError_t launch_dispatch(moe_ctx* ctx, const void* x, const int32_t* inv_perm, void* x_perm,
+                            cudaStream_t stream);
+
+cudaError_t launch_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_perm, const float* topk_w,
+                           void* out, cudaStream_t stream);
+
+// Returns MOE_OK, MOE_ERR_CUDA (driver/runtime failure) or MOE_ERR_INVALID_ARG.
+moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* offsets, const void* w_gate,
+                             const void* w_up, const void* w_down, void* h_ws, void* y_perm,
+                             float* h_fp32_debug, const moe_tuning* tuning, cudaStream_t stream);
+
+cudaError_t prepare_expert_ffn(moe_ctx* ctx);  // one-time kernel attributes (dynamic shared memory size)
+
+}  // namespace moe

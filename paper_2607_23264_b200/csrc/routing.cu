@@ -1,0 +1,172 @@
+// Routing plan: top-k + softmax weights, per-expert histogram, exclusive scan, stable permutation.
+//
+// The token range is cut into chunks of `tokens_per_chunk` tokens (at most 256 slots).  Three launches:
+//   1. route_topk_hist : one CTA per chunk; a warp per token selects the k largest logits by k rounds of
+//                        warp arg-max (shuffle reduction, ties to the lower index) and computes the
+//                        softmax weights; the CTA then histograms its slots per expert.
+//   2. route_scan      : one CTA; exclusive prefix of the chunk histograms over chunks (per expert) and
+//                        the exclusive scan of the totals over experts (offsets).
+//   3. route_scatter   : one CTA per chunk, one thread per slot; the stable rank of a slot among the
+//                        slots of its expert is (slots of earlier chunks) + (slots of earlier warps in
+//                        the chunk) + (earlier lanes in the warp, from a match-any ballot).
+// Everything is integer work on identical fp32 inputs, so ids, counts, offsets and both permutations are
+// reproducible bit for bit.
+#include "moe_internal.h"
+
+namespace {
+
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+__global__ void __launch_bounds__(kRouteThreads)
+route_topk_hist(const float* __restrict__ logits, int T, int E, int k, int tokens_per_chunk,
+                int32_t* __restrict__ topk_ids, float* __restrict__ topk_w, int32_t* __restrict__ chunk_hist) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int warps = kRouteThreads / 32;
+  float* s_logit = reinterpret_cast<float*>(smem_raw);                    // [warps][E]
+  int32_t* s_hist = reinterpret_cast<int32_t*>(s_logit + warps * E);      // [E]
+  int32_t* s_ids = s_hist + E;                                            // [256]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int chunk = blockIdx.x;
+  const int t_begin = chunk * tokens_per_chunk;
+  const int t_end = min(T, t_begin + tokens_per_chunk);
+
+  for (int e = tid; e < E; e += kRouteThreads) s_hist[e] = 0;
+
+  float* my = s_logit + warp * E;
+  for (int t = t_begin + warp; t < t_end; t += warps) {
+    const float* row = logits + static_cast<size_t>(t) * E;
+    for (int e = lane; e < E; e += 32) my[e] = row[e];
+    __syncwarp();
+    float sel_logit = 0.f;   // lane j keeps the logit picked in round j
+    int sel_id = 0;
+    for (int j = 0; j < k; ++j) {
+      float best = -INFINITY;
+      int best_e = 0x7FFFFFFF;
+      for (int e = lane; e < E; e += 32) {      // ascending e with strict '>' keeps the lowest index
+        const float v = my[e];
+        if (v > best) { best = v; best_e = e; }
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(kFull, best, off);
+        const int oe = __shfl_xor_sync(kFull, best_e, off);
+        if (ov > best || (ov == best && oe < best_e)) { best = ov; best_e = oe; }
+      }
+      if (lane == j) { sel_logit = best; sel_id = best_e; }
+      if (lane == 0) my[best_e] = -INFINITY;    // taken
+      __syncwarp();
+    }
+    // softmax over the k selected logits; round 0 picked the maximum
+    const float m = __shfl_sync(kFull, sel_logit, 0);
+    float p = (lane < k) ? expf(sel_logit - m) : 0.f;
+    float sum = p;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
+    if (lane < k) {
+      const size_t s = static_cast<size_t>(t) * k + lane;
+      topk_ids[s] = sel_id;
+      topk_w[s] = p / sum;
+      s_ids[(t - t_begin) * k + lane] = sel_id;
+    }
+    __syncwarp();
+  }
+  __syncthreads();
+  const int n_slots = (t_end - t_begin) * k;
+  if (tid < n_slots) atomicAdd(&s_hist[s_ids[tid]], 1);   // integer counts: order does not matter
+  __syncthreads();
+  for (int e = tid; e < E; e += kRouteThreads) chunk_hist[static_cast<size_t>(chunk) * E + e] = s_hist[e];
+}
+
+// One CTA of 1024 threads, E <= 1024: thread e walks the chunks of expert e, then a block scan over e.
+__global__ void __launch_bounds__(1024)
+route_scan(const int32_t* __restrict__ chunk_hist, int32_t* __restrict__ chunk_base, int num_chunks, int E,
+           int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+  __shared__ int32_t s_warp[32];
+  const int e = threadIdx.x, lane = e & 31, warp = e >> 5;
+  int32_t total = 0;
+  if (e < E) {
+    for (int c = 0; c < num_chunks; ++c) {
+      const size_t i = static_cast<size_t>(c) * E + e;
+      const int32_t v = chunk_hist[i];
+      chunk_base[i] = total;
+      total += v;
+    }
+    counts[e] = total;
+  }
+  int32_t incl = total;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int32_t o = __shfl_up_sync(kFull, incl, off);
+    if (lane >= off) incl += o;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int32_t w = s_warp[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int32_t o = __shfl_up_sync(kFull, w, off);
+      if (lane >= off) w += o;
+    }
+    s_warp[lane] = w;   // inclusive over warps
+  }
+  __syncthreads();
+  const int32_t before = (warp ? s_warp[warp - 1] : 0) + incl - total;   // exclusive prefix of counts
+  if (e < E) offsets[e] = before;
+  if (e == E - 1) offsets[E] = before + total;
+}
+
+__global__ void __launch_bounds__(kRouteThreads)
+route_scatter(const int32_t* __restrict__ topk_ids, const int32_t* __restrict__ offsets,
+              const int32_t* __restrict__ chunk_base, int T, int E, int k, int tokens_per_chunk,
+              int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int warps = kRouteThreads / 32;
+  int32_t* s_warp_cnt = reinterpret_cast<int32_t*>(smem_raw);   // [warps][E]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int chunk = blockIdx.x;
+  const int t_begin = chunk * tokens_per_chunk;
+  const int t_end = min(T, t_begin + tokens_per_chunk);
+  const int n_slots = (t_end - t_begin) * k;
+  const int s = t_begin * k + tid;
+
+  for (int i = tid; i < warps * E; i += kRouteThreads) s_warp_cnt[i] = 0;
+  __syncthreads();
+
+  const bool active = tid < n_slots;
+  const int e = active ? topk_ids[s] : (E + lane);   // idle lanes get distinct keys outside [0,E)
+  const unsigned same = __match_any_sync(kFull, e);
+  const int rank_in_warp = __popc(same & ((1u << lane) - 1u));
+  if (active && rank_in_warp == 0) s_warp_cnt[warp * E + e] = __popc(same);
+  __syncthreads();
+  if (active) {
+    int before = 0;
+    for (int w = 0; w < warp; ++w) before += s_warp_cnt[w * E + e];
+    const int row = offsets[e] + chunk_base[static_cast<size_t>(chunk) * E + e] + before + rank_in_warp;
+    perm[row] = s;
+    inv_perm[s] = row;
+  }
+}
+
+}  // namespace
+
+namespace moe {
+
+cudaError_t launch_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids, float* topk_w,
+                                int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
+                                cudaStream_t stream) {
+  const moe_shape& s = ctx->shape;
+  const int warps = kRouteThreads / 32;
+  const size_t smem1 = (static_cast<size_t>(warps) * s.E + s.E + 256) * 4;
+  const size_t smem3 = static_cast<size_t>(warps) * s.E * 4;
+  route_topk_hist<<<ctx->num_chunks, kRouteThreads, smem1, stream>>>(logits, s.T, s.E, s.k, ctx->tokens_per_chunk,
+                                                                     topk_ids, topk_w, ctx->d_chunk_hist);
+  route_scan<<<1, 1024, 0, stream>>>(ctx->d_chunk_hist, ctx->d_chunk_base, ctx->num_chunks, s.E, counts, offsets);
+  route_scatter<<<ctx->num_chunks, kRouteThreads, smem3, stream>>>(topk_ids, offsets, ctx->d_chunk_base, s.T, s.E,
+                                                                   s.k, ctx->tokens_per_chunk, perm, inv_perm);
+  ctx->last_launches += 3;
+  return cudaGetLastError();
+}
+
+}  // namespace moe

@@ -176,3 +176,37 @@ def random_small_config(rng: np.random.Generator, **fixed) -> MoEConfig:
         seed=int(fixed.get("seed", rng.integers(0, 2**31))),
         router=str(fixed.get("router", "xWr")),
     )
+
+
+class WeightStream:
+    """``weights(e)`` callable that regenerates experts on demand instead of holding them.
+
+    ``order`` is the ascending list of experts the consumer will ask for; the next few are generated
+    ahead of time on a thread pool.  Asking for an expert outside ``order`` generates it on the spot.
+    """
+
+    def __init__(self, cfg: MoEConfig, order, threads: int | None = None):
+        self.cfg = cfg
+        self.order = [int(e) for e in order]
+        self.pos = {e: i for i, e in enumerate(self.order)}
+        self.pool = ThreadPoolExecutor(max_workers=threads or default_threads())
+        self.ahead = 2 * (threads or default_threads())
+        self.pending = {}
+        self.next_submit = 0
+
+    def _fill(self, upto: int):
+        while self.next_submit < min(len(self.order), upto):
+            e = self.order[self.next_submit]
+            self.pending[e] = self.pool.submit(expert_weights, self.cfg, e)
+            self.next_submit += 1
+
+    def __call__(self, e: int):
+        e = int(e)
+        if e not in self.pos:
+            return expert_weights(self.cfg, e)
+        self._fill(self.pos[e] + 1 + self.ahead)
+        fut = self.pending.pop(e, None)
+        return fut.result() if fut is not None else expert_weights(self.cfg, e)
+
+    def close(self):
+        self.pool.shutdown(wait=False, cancel_futures=True)

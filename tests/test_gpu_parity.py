@@ -1,0 +1,219 @@
+"""GPU parity: every C-ABI call against the CPU oracle on the same seeded inputs (small sizes, full
+element-by-element comparison).  Indices bit-exact; values within the stated tolerances."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as orc
+from paper_2607_23264_b200 import binding, inputs as gen
+from moe_testlib import (DEV, TOL_FRO, Layer, assert_out_close, assert_plan_matches, bits_to_dev, dev_bf16_to_f64,
+                         dev_to_bits, rel_fro)
+
+pytestmark = pytest.mark.gpu
+
+# Small layers spanning several 128-row tiles, ragged tails, empty experts and N tails (F=192, H=320).
+SMALL = [
+    gen.CONFIGS["C1"],
+    gen.MoEConfig("ragged", T=333, H=320, F=192, E=5, k=2, seed=11, router="xWr"),
+    gen.MoEConfig("k1", T=200, H=128, F=128, E=3, k=1, seed=12, router="xWr"),
+    gen.MoEConfig("one_expert", T=300, H=64, F=64, E=1, k=1, seed=13, router="xWr"),
+    gen.MoEConfig("k_eq_E", T=50, H=128, F=256, E=4, k=4, seed=14, router="xWr"),
+    gen.MoEConfig("skewed", T=700, H=256, F=128, E=40, k=4, seed=15, router="xWr_zipf"),
+    gen.MoEConfig("tiny_T", T=3, H=64, F=64, E=16, k=2, seed=16, router="iid"),
+    gen.MoEConfig("deep_k", T=130, H=1024, F=1088, E=6, k=3, seed=17, router="xWr"),
+]
+IDS = [c.name for c in SMALL]
+
+
+def oracle_for(layer: Layer) -> dict:
+    return orc.forward(layer.x_bits, layer.logits, layer.cfg.k, layer.weights)
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+def test_plan_routing_bit_exact(cfg):
+    L = Layer(cfg, upload_weights=False)
+    L.plan()
+    ids, w = orc.topk_route(L.logits, cfg.k)
+    counts, offsets, perm, inv = orc.plan_permutation(ids, cfg.E)
+    assert_plan_matches(L, dict(topk_ids=ids, topk_w=w, counts=counts, offsets=offsets, perm=perm, inv_perm=inv))
+
+
+def test_plan_routing_ties_and_wide_experts():
+    """Logits with many exact ties (tie-break to the lower index) and E beyond one warp's width."""
+    rng = np.random.default_rng(5)
+    for (T, E, k) in [(97, 8, 3), (260, 256, 8), (64, 1000, 32), (33, 31, 31)]:
+        cfg = gen.MoEConfig("ties", T=T, H=64, F=64, E=E, k=k, seed=0, router="iid")
+        logits = (rng.integers(-3, 4, size=(T, E)) * 0.25).astype(np.float32)
+        L = Layer(cfg, upload_weights=False, logits=logits)
+        L.plan()
+        ids, w = orc.topk_route(logits, k)
+        counts, offsets, perm, inv = orc.plan_permutation(ids, E)
+        assert_plan_matches(L, dict(topk_ids=ids, topk_w=w, counts=counts, offsets=offsets, perm=perm, inv_perm=inv))
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+def test_dispatch_bit_exact(cfg):
+    L = Layer(cfg, upload_weights=False)
+    ids, _ = orc.topk_route(L.logits, cfg.k)
+    _, _, perm, inv = orc.plan_permutation(ids, cfg.E)
+    x_perm = L.nan_bf16(cfg.R + 1, cfg.H)          # one canary row after the buffer
+    L.ctx.moe_dispatch(L.x, torch.from_numpy(inv).to(DEV), x_perm)
+    torch.cuda.synchronize()
+    got = dev_to_bits(x_perm)
+    assert np.array_equal(got[:cfg.R], orc.dispatch(L.x_bits, perm, cfg.k))
+    assert np.all(got[cfg.R] == got[cfg.R, 0]) and np.isnan(gen.bf16_bits_to_f32(got[cfg.R, :1]))[0], "canary row"
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+def test_expert_ffn_parity(cfg):
+    L = Layer(cfg)
+    ref = oracle_for(L)
+    x_perm = bits_to_dev(ref["x_perm"])
+    offsets = torch.from_numpy(ref["offsets"]).to(DEV)
+    h = L.nan_bf16(cfg.R + 1, cfg.F)
+    y = L.nan_bf16(cfg.R + 1, cfg.H)
+    h32 = torch.full((cfg.R, cfg.F), float("nan"), dtype=torch.float32, device=DEV)
+    L.ctx.moe_expert_ffn(x_perm, offsets, L.w_gate, L.w_up, L.w_down, h, y, h_fp32_debug=h32)
+    torch.cuda.synchronize()
+    L.check_device_status()
+    assert L.ctx.moe_last_launch_count() == 2
+    h32_np = h32.cpu().numpy().astype(np.float64)
+    assert np.isfinite(h32_np).all(), "every row of h belongs to an expert and must be written"
+    assert rel_fro(h32_np, ref["h"]) <= TOL_FRO
+    h_np, y_np = dev_bf16_to_f64(h), dev_bf16_to_f64(y)
+    assert np.isnan(h_np[cfg.R]).all() and np.isnan(y_np[cfg.R]).all(), "canary rows must stay untouched"
+    assert rel_fro(h_np[:cfg.R], ref["h"]) <= TOL_FRO
+    assert rel_fro(y_np[:cfg.R], ref["y_perm"]) <= TOL_FRO
+    # per expert too, so that a small expert cannot hide behind a large one
+    for e in range(cfg.E):
+        lo, hi = ref["offsets"][e], ref["offsets"][e + 1]
+        if hi > lo:
+            assert rel_fro(y_np[lo:hi], ref["y_perm"][lo:hi]) <= 2 * TOL_FRO, f"expert {e}"
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+def test_combine_parity(cfg):
+    L = Layer(cfg, upload_weights=False)
+    rng = np.random.default_rng(cfg.seed)
+    y_bits = gen.f32_to_bf16_bits(rng.standard_normal((cfg.R, cfg.H)).astype(np.float32))
+    ids, w = orc.topk_route(L.logits, cfg.k)
+    _, _, _, inv = orc.plan_permutation(ids, cfg.E)
+    w32 = w.astype(np.float32)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_combine(bits_to_dev(y_bits), torch.from_numpy(inv).to(DEV), torch.from_numpy(w32).to(DEV), out)
+    torch.cuda.synchronize()
+    ref = orc.combine(orc.bf16_to_f64(y_bits), inv, w32.astype(np.float64))
+    got = dev_bf16_to_f64(out)
+    # fp32 accumulation of k terms then one bf16 rounding: relative error about 2^-9
+    np.testing.assert_allclose(got, ref, rtol=2.0 ** -8, atol=1e-6)
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+def test_fused_forward_parity(cfg):
+    L = Layer(cfg)
+    ref = oracle_for(L)
+    lay = L.ctx.workspace_layout()
+    ws = torch.empty(lay["total"], dtype=torch.uint8, device=DEV)
+    ws.fill_(0xFF)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
+    torch.cuda.synchronize()
+    L.check_device_status()
+    assert L.ctx.moe_last_launch_count() == 7
+
+    def sl(name, count, dtype):
+        nbytes = count * torch.empty((), dtype=dtype).element_size()
+        return ws[lay[name]:lay[name] + nbytes].view(dtype)
+
+    R = cfg.R
+    for name, count in (("topk_ids", R), ("counts", cfg.E), ("offsets", cfg.E + 1), ("perm", R), ("inv_perm", R)):
+        got = sl(name, count, torch.int32).cpu().numpy()
+        assert np.array_equal(got, np.asarray(ref[name]).reshape(-1)), name
+    assert np.abs(sl("topk_w", R, torch.float32).cpu().numpy() - ref["topk_w"].reshape(-1)).max() <= 1e-6
+    assert np.array_equal(dev_to_bits(sl("x_perm", R * cfg.H, torch.bfloat16)).reshape(R, cfg.H), ref["x_perm"])
+    assert rel_fro(dev_bf16_to_f64(sl("h", R * cfg.F, torch.bfloat16)).reshape(R, cfg.F), ref["h"]) <= TOL_FRO
+    assert rel_fro(dev_bf16_to_f64(sl("y_perm", R * cfg.H, torch.bfloat16)).reshape(R, cfg.H), ref["y_perm"]) <= TOL_FRO
+    assert_out_close(dev_bf16_to_f64(out), ref["out"], f"out[{cfg.name}]")
+
+    # determinism: a second run is bitwise identical
+    out2 = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+
+
+def test_fused_forward_host_matches_device_path():
+    cfg = SMALL[1]
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
+    x_host = torch.from_numpy(L.x_bits.view(np.int16)).pin_memory()
+    logits_host = torch.from_numpy(L.logits).pin_memory()
+    out_host = torch.zeros((cfg.T, cfg.H), dtype=torch.int16).pin_memory()
+    L.ctx.moe_fused_forward_host(x_host, logits_host, L.w_gate, L.w_up, L.w_down, out_host, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_host.numpy().view(np.uint16), dev_to_bits(out))
+
+
+def test_pacing_points_are_bitwise_identical():
+    """Store pacing reorders stores in time only: all 20 sweep points give the same bits."""
+    cfg = gen.MoEConfig("pace", T=900, H=512, F=768, E=4, k=2, seed=31, router="xWr")
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    base = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, base, ws)
+    torch.cuda.synchronize()
+    ref = orc.forward(L.x_bits, L.logits, cfg.k, L.weights)
+    assert_out_close(dev_bf16_to_f64(base), ref["out"], "pacing baseline")
+    points = [(b, 0, 1) for b in (1, 2, 4, 8, 16)] + [(b, 1, ik) for b in (1, 2, 4, 8, 16) for ik in (1, 2, 4)]
+    assert len(points) == 20
+    for b, mode, ik in points:
+        out = L.nan_bf16(cfg.T, cfg.H)
+        L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws,
+                                tuning=binding.make_tuning(b, mode, ik))
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), base.view(torch.int16)), (b, mode, ik)
+    L.check_device_status()
+
+
+def test_zero_tokens_is_a_no_op():
+    ctx = binding.Context(0, 128, 128, 4, 2)
+    counts = torch.full((4,), -1, dtype=torch.int32, device=DEV)
+    offsets = torch.full((5,), -1, dtype=torch.int32, device=DEV)
+    ctx.moe_plan_routing(None, None, None, counts, offsets, None, None)
+    ctx.moe_dispatch(None, None, None)
+    ctx.moe_combine(None, None, None, None)
+    ctx.moe_expert_ffn(None, None, None, None, None, None, None)
+    torch.cuda.synchronize()
+    assert counts.eq(0).all() and offsets.eq(0).all()
+
+
+def test_host_side_errors_are_synchronous():
+    cfg = SMALL[0]
+    L = Layer(cfg, upload_weights=False)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    w = torch.zeros(8, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(binding.MoeError) as ei:       # workspace too small
+        L.ctx.moe_fused_forward(L.x, L.d_logits, w, w, w, out, ws[:4096])
+    assert ei.value.code == 3
+    with pytest.raises(binding.MoeError) as ei:       # misaligned pointer
+        L.ctx.moe_dispatch(L.x.view(-1)[1:], L.inv_perm, out)
+    assert ei.value.code == 1
+    with pytest.raises(binding.MoeError) as ei:       # null pointer
+        L.ctx.moe_combine(None, L.inv_perm, L.topk_w, out)
+    assert ei.value.code == 1
+    for bad in (binding.make_tuning(3, 0, 1), binding.make_tuning(1, 2, 1), binding.make_tuning(1, 1, 3),
+                binding.make_tuning(1, 0, 1, dep_lead_D=1)):
+        with pytest.raises(binding.MoeError) as ei:
+            L.ctx.moe_fused_forward(L.x, L.d_logits, w, w, w, out, ws, tuning=bad)
+        assert ei.value.code == 1
+    with pytest.raises(binding.MoeError) as ei:       # interleaved schedule not built
+        L.ctx.moe_fused_forward(L.x, L.d_logits, w, w, w, out, ws, tuning=binding.make_tuning(1, 0, 1, schedule=1))
+    assert ei.value.code == 7
+    with pytest.raises(binding.MoeError) as ei:
+        binding.Context(8, 100, 128, 4, 2)
+    assert ei.value.code == 2
+    torch.cuda.synchronize()
+    L.check_device_status()
