@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the fused MoE forward (EP=1) on the Mixtral-like layer (T=8192, H=4096, F=14336, E=8, top-2).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--impl reference] [--sweep]
+
+A step is one pass of the whole hot path (routing plan, dispatch, Linear-1 + SiLU*mul, Linear-2,
+combine) over one batch of seeded synthetic tokens.  With N > 1 (torchrun) every rank runs the same
+layer on its own batch (experts replicated, tokens data-parallel, no collective on the data path):
+weak scaling; the reported value is all ranks' tokens over the slowest rank's device time.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2607_23264_b200 import inputs as gen  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one expert_gemm_kernel<true> (Linear-1) launch on the
+# bench workload, from the ncu capture summarised in profiles/; None until a capture exists.
+LINEAR1_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.tmp.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        busy = [v for v in sm if v > 0]
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample_rate(cfg, x_bits, logits, weights, n_tokens, seed=1234):
+    """Time the CPU oracle on a seeded sample of tokens of this workload.  Returns (tokens/s, seconds)."""
+    from oracle import moe_oracle as orc
+    rng = np.random.default_rng(seed)
+    toks = np.sort(rng.choice(cfg.T, size=min(n_tokens, cfg.T), replace=False))
+    t0 = time.perf_counter()
+    orc.forward_tokens(toks, x_bits, logits, cfg.k, weights)
+    dt = time.perf_counter() - t0
+    return len(toks) / dt, dt
+
+
+def run_reference(args, cfg, rank, world):
+    """--impl reference: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    x_bits = gen.make_x(cfg)
+    logits = gen.make_logits(cfg, x_bits)
+    W = gen.stacked_weights(cfg)
+    weights = lambda e: (W[0][e], W[1][e], W[2][e])
+    n_tok = args.ref_tokens
+    for _ in range(args.warmup):
+        oracle_sample_rate(cfg, x_bits, logits, weights, n_tok)
+    times = []
+    for s in range(args.steps):
+        _, dt = oracle_sample_rate(cfg, x_bits, logits, weights, n_tok, seed=1000 + s)
+        times.append(dt)
+    total = sum(times)
+    value = n_tok * args.steps / total
+    cores = oracle_threads()
+    sample = f"{n_tok} seeded-random tokens of {cfg.name} per step (row-sampled oracle, exact per row)"
+    line = {
+        "impl": "reference", "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, args.gpus),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, n_gpus):
+    return {"workload": f"{cfg.name}: T={cfg.T} tokens per GPU, hidden={cfg.H}, ffn={cfg.F}, E={cfg.E}, top-{cfg.k}, "
+                        f"SwiGLU, bf16, router={cfg.router}, seed={cfg.seed}",
+            "tokens_per_gpu": cfg.T, "global_tokens": cfg.T * n_gpus, "parallelism": f"ep1 x {n_gpus} replicas",
+            "l2_policy": "inputs larger than L2 (weights 2.8 GB + activations 1.1 GB per step vs 126 MB L2)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="C2", choices=sorted(gen.CONFIGS))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--ref-tokens", type=int, default=128, help="tokens per step of the reference (oracle) arm")
+    ap.add_argument("--cpu-baseline-tokens", type=int, default=384)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--burst", type=int, default=1)
+    ap.add_argument("--mode", type=int, default=0)
+    ap.add_argument("--ik", type=int, default=1)
+    ap.add_argument("--sweep", action="store_true", help="store-pacing sweep (20 points) instead of the bench line")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = gen.CONFIGS[args.config]
+    if args.warmup < 3 and args.impl == "b200" and not args.sweep:
+        args.warmup = 3   # timing rule: at least three warm-up steps
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2607_23264_b200 import binding
+
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    # every rank gets its own batch (the seeded batch, rows rotated by rank); expert weights are replicated
+    x_bits = gen.make_x(cfg)
+    if rank != 0:
+        x_bits = np.roll(x_bits, rank * 17, axis=0)
+    logits = gen.make_logits(cfg, x_bits)
+
+    to_dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+    w_gate = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
+    w_up = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
+    w_down = torch.empty((cfg.E, cfg.H, cfg.F), dtype=torch.bfloat16, device=dev)
+    keep_host = rank == 0 and not args.no_cpu_baseline and not args.sweep and cfg.E <= 16
+    host_w = {}
+
+    def sink(e, g, u, d):
+        w_gate[e].copy_(to_dev(g))
+        w_up[e].copy_(to_dev(u))
+        w_down[e].copy_(to_dev(d))
+        if keep_host:
+            host_w[e] = (g, u, d)
+
+    gen.for_each_expert(cfg, sink)
+    x = to_dev(x_bits)
+    d_logits = torch.from_numpy(logits).to(dev)
+    ctx = binding.Context(cfg.T, cfg.H, cfg.F, cfg.E, cfg.k, device=local_rank)
+    ws = torch.empty(ctx.workspace_bytes(), dtype=torch.uint8, device=dev)
+    out = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    if args.sweep:
+        run_sweep(args, cfg, ctx, binding, (x, d_logits, w_gate, w_up, w_down, out, ws), timed, rank)
+        return
+
+    tuning = binding.make_tuning(args.burst, args.mode, args.ik)
+    step = lambda: ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tuning)
+
+    # ---- device-resident throughput, with per-kernel events, clocks sampled during the timed region
+    ctx.moe_set_kernel_timing(True)
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    per_step_kernel = []
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    total_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = ctx.moe_last_launch_count() * args.steps
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # per-kernel average launch duration: the same steps again, reading the event pairs after each step
+    for _ in range(args.steps):
+        step()
+        per_step_kernel.append(ctx.moe_get_kernel_times())
+    ctx.moe_set_kernel_timing(False)
+    kernel_ms = [float(np.mean([s[i] for s in per_step_kernel])) for i in range(len(binding.KERNEL_NAMES))]
+
+    code, detail = ctx.moe_last_device_status()
+    if code != 0:
+        raise RuntimeError(f"device status {binding.STATUS_NAMES.get(code, code)} detail {detail:#x}")
+
+    # ---- end to end through the host-buffer entry point: H2D of x and logits, D2H of out, every step
+    x_host = torch.from_numpy(x_bits.view(np.int16)).pin_memory()
+    logits_host = torch.from_numpy(logits).pin_memory()
+    out_host = torch.empty((cfg.T, cfg.H), dtype=torch.int16).pin_memory()
+    e2e_step = lambda: ctx.moe_fused_forward_host(x_host, logits_host, w_gate, w_up, w_down, out_host, ws,
+                                                  tuning=tuning)
+    e2e_ms = timed(e2e_step, args.steps, args.warmup)
+    h2d = x_host.numel() * 2 + logits_host.numel() * 4
+    d2h = out_host.numel() * 2
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    ms_per_step = total_ms / args.steps
+    tokens = cfg.T * world
+    value = tokens / (ms_per_step * 1e-3)
+    tflops = cfg.flops * world / (ms_per_step * 1e-3) / 1e12
+    R = cfg.R
+    l1_flops = 4 * R * cfg.H * cfg.F
+    l2_flops = 2 * R * cfg.H * cfg.F
+    l1_tf = l1_flops / (kernel_ms[4] * 1e-3) / 1e12
+    l2_tf = l2_flops / (kernel_ms[5] * 1e-3) / 1e12
+    move_bytes = 2 * cfg.H * (cfg.T + R)
+    disp_gbs = move_bytes / (kernel_ms[3] * 1e-3) / 1e9
+    comb_gbs = (move_bytes + 8 * R) / (kernel_ms[6] * 1e-3) / 1e9
+    peak_tf = float(peaks["bf16_tflops"])
+    roofline = {
+        "kernel": "expert_gemm_kernel<gated> (Linear-1 + SiLU*mul)", "bound": "tensor", "achieved": l1_tf,
+        "peak": peak_tf, "unit": "TFLOP/s", "frac": l1_tf / peak_tf, "traffic": LINEAR1_DRAM_TRAFFIC_BYTES,
+        "peak_source": f"{peak_kind} bf16_tflops (burst)",
+        "frac_of_sustained": l1_tf / float(peaks.get("bf16_tflops_sustained", peak_tf)),
+        "flops_per_launch": l1_flops, "ms_per_launch": kernel_ms[4],
+    }
+    line = {
+        "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(cfg, world),
+        "tflops": tflops, "frac_bf16_peak": tflops / world / peak_tf,
+        "kernels_ms": dict(zip(binding.KERNEL_NAMES, kernel_ms)),
+        "linear2_tflops": l2_tf, "dispatch_gbs": disp_gbs, "combine_gbs": comb_gbs,
+        "dispatch_frac_hbm": disp_gbs / float(peaks["hbm_gbs"]), "combine_frac_hbm": comb_gbs / float(peaks["hbm_gbs"]),
+        "roofline": roofline,
+        "e2e": {"value": tokens / (e2e_ms / args.steps * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": launches, "clocks": clocks, "tuning": [args.burst, args.mode, args.ik],
+    }
+    if keep_host:
+        rate, dt = oracle_sample_rate(cfg, x_bits, logits, lambda e: host_w[e], args.cpu_baseline_tokens)
+        line["cpu_baseline"] = {
+            "value": rate, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"{args.cpu_baseline_tokens} seeded-random tokens of {cfg.name} (row-sampled fp64 oracle, "
+                      f"{dt:.1f} s)"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_sweep(args, cfg, ctx, binding, bufs, timed, rank):
+    """Store-pacing sweep: burst in {1,2,4,8,16} x {after-mainloop, every-k-iterations k in {1,2,4}}."""
+    import torch
+    x, d_logits, w_gate, w_up, w_down, out, ws = bufs
+    points = [(b, 0, 1) for b in (1, 2, 4, 8, 16)] + [(b, 1, ik) for b in (1, 2, 4, 8, 16) for ik in (1, 2, 4)]
+    base = None
+    rows = []
+    ctx.moe_set_kernel_timing(True)
+    for b, mode, ik in points:
+        tn = binding.make_tuning(b, mode, ik)
+        fn = lambda: ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tn)
+        ms = timed(fn, args.steps, max(1, args.warmup)) / args.steps
+        km = ctx.moe_get_kernel_times()
+        bits = out.view(torch.int16).clone()
+        if base is None:
+            base = bits
+        rows.append({"burst": b, "mode": mode, "k": ik, "ms_per_step": ms, "linear1_ms": km[4], "linear2_ms": km[5],
+                     "tflops": cfg.flops / (ms * 1e-3) / 1e12, "identical_bits": bool(torch.equal(bits, base))})
+    if rank == 0:
+        print(json.dumps({"sweep": rows, "config": workload_config(cfg, 1)}), flush=True)
+
+
+if __name__ == "__main__":
+    main()

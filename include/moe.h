@@ -175,6 +175,16 @@ moe_status moe_last_device_status(moe_ctx* ctx, int32_t* code, int32_t* detail, 
 /* Number of kernels the last call on this context launched (host-side count, for benchmarking). */
 int32_t moe_last_launch_count(const moe_ctx* ctx);
 
+/*
+ * Per-kernel timing (measurement aid; the paper times its kernel with CUDA events, Sec. 5.1).  When
+ * enabled, each call records a CUDA event on the stream before its first kernel and after every kernel.
+ * moe_get_kernel_times waits for the last call's events and writes the seven device durations in
+ * milliseconds, in launch order {top-k + histogram, scan, scatter, dispatch, Linear-1, Linear-2, combine},
+ * to the HOST array ms_host[n], n == 7; kernels the last call did not launch read -1.
+ */
+moe_status moe_set_kernel_timing(moe_ctx* ctx, int32_t enable);
+moe_status moe_get_kernel_times(moe_ctx* ctx, float* ms_host, int32_t n);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,8 +21,12 @@ STATUS_NAMES = {
 EXPORTS = (
     "moe_status_string", "moe_create", "moe_destroy", "moe_workspace_bytes", "moe_get_workspace_layout",
     "moe_plan_routing", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_fused_forward",
-    "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count",
+    "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count", "moe_set_kernel_timing",
+    "moe_get_kernel_times",
 )
+
+KERNEL_NAMES = ("route_topk_hist", "route_scan", "route_scatter", "dispatch_rows", "expert_gemm_linear1",
+                "expert_gemm_linear2", "combine_rows")
 
 
 class MoeError(RuntimeError):
@@ -76,6 +80,8 @@ def load_library() -> C.CDLL:
     lib.moe_last_device_status.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_last_launch_count.argtypes = [vp]
     lib.moe_last_launch_count.restype = C.c_int32
+    lib.moe_set_kernel_timing.argtypes = [vp, C.c_int32]
+    lib.moe_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32]
     for name in EXPORTS:
         if name not in ("moe_status_string", "moe_destroy", "moe_workspace_bytes", "moe_last_launch_count"):
             getattr(lib, name).restype = C.c_int
@@ -212,3 +218,11 @@ class Context:
 
     def moe_last_launch_count(self) -> int:
         return self._lib.moe_last_launch_count(self._handle)
+
+    def moe_set_kernel_timing(self, enable: bool):
+        _check(self._lib.moe_set_kernel_timing(self._handle, 1 if enable else 0), "moe_set_kernel_timing")
+
+    def moe_get_kernel_times(self) -> list:
+        ms = (C.c_float * len(KERNEL_NAMES))()
+        _check(self._lib.moe_get_kernel_times(self._handle, ms, len(KERNEL_NAMES)), "moe_get_kernel_times")
+        return list(ms)

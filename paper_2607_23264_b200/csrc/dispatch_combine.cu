@@ -119,6 +119,7 @@ cudaError_t launch_dispatch(moe_ctx* ctx, const void* x, const int32_t* inv_perm
   if (blocks > cap) blocks = cap;
   dispatch_rows<<<blocks, kThreads, 0, stream>>>(static_cast<const uint4*>(x), inv_perm,
                                                  static_cast<uint4*>(x_perm), s.T, s.k, vec_per_row);
+  moe_mark(ctx, 4, stream);
   ctx->last_launches += 1;
   return cudaGetLastError();
 }
@@ -136,6 +137,7 @@ cudaError_t launch_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_
   combine_rows<<<static_cast<int>(blocks), kThreads, 0, stream>>>(
       static_cast<const uint4*>(y_perm), inv_perm, topk_w, static_cast<uint4*>(out), s.T, s.k, vec_per_row,
       blocks_per_row);
+  moe_mark(ctx, 7, stream);
   ctx->last_launches += 1;
   return cudaGetLastError();
 }

@@ -404,7 +404,9 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
 
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
   expert_gemm_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, p1);
+  moe_mark(ctx, 5, stream);
   expert_gemm_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(tm_h, tm_wd, tm_wd, p2);
+  moe_mark(ctx, 6, stream);
   ctx->last_launches += 2;
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -37,6 +37,14 @@ moe_status check_ctx(const moe_ctx* ctx) {
   return dev == ctx->device ? MOE_OK : MOE_ERR_INVALID_ARG;
 }
 
+// Start of a public call: reset the launch counter and the timing marks, record the mark that
+// precedes the call's first kernel.
+inline void begin_call(moe_ctx* ctx, int first_mark, void* stream) {
+  ctx->last_launches = 0;
+  ctx->ev_recorded = 0;
+  moe_mark(ctx, first_mark, static_cast<cudaStream_t>(stream));
+}
+
 inline size_t up256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
 void fill_layout(const moe_shape& s, moe_workspace_layout* L) {
@@ -128,6 +136,7 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   ok = ok && cudaMalloc(&ctx->d_status, 2 * 4) == cudaSuccess;
   ok = ok && cudaMemset(ctx->d_status, 0, 2 * 4) == cudaSuccess;
   ok = ok && moe::prepare_expert_ffn(ctx) == cudaSuccess;
+  for (int i = 0; ok && i <= kMoeKernels; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
   if (!ok) {
     moe_destroy(ctx);
     return MOE_ERR_CUDA;
@@ -141,6 +150,8 @@ void moe_destroy(moe_ctx* ctx) {
   if (ctx->d_chunk_hist) cudaFree(ctx->d_chunk_hist);
   if (ctx->d_chunk_base) cudaFree(ctx->d_chunk_base);
   if (ctx->d_status) cudaFree(ctx->d_status);
+  for (int i = 0; i <= kMoeKernels; ++i)
+    if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
   delete ctx;
 }
 
@@ -149,7 +160,7 @@ moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids
                             void* stream) {
   moe_status st = check_ctx(ctx);
   if (st != MOE_OK) return st;
-  ctx->last_launches = 0;
+  begin_call(ctx, 0, stream);
   const moe_shape& s = ctx->shape;
   if (!counts || !offsets) return MOE_ERR_INVALID_ARG;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
@@ -170,7 +181,7 @@ moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids
 moe_status moe_dispatch(moe_ctx* ctx, const void* x, const int32_t* inv_perm, void* x_perm, void* stream) {
   moe_status st = check_ctx(ctx);
   if (st != MOE_OK) return st;
-  ctx->last_launches = 0;
+  begin_call(ctx, 3, stream);
   if (ctx->shape.T == 0) return MOE_OK;
   if (!x || !inv_perm || !x_perm) return MOE_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(inv_perm) || !aligned16(x_perm)) return MOE_ERR_INVALID_ARG;
@@ -184,7 +195,7 @@ moe_status moe_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* offse
                           float* h_fp32_debug, const moe_tuning* tuning, void* stream) {
   moe_status st = check_ctx(ctx);
   if (st != MOE_OK) return st;
-  ctx->last_launches = 0;
+  begin_call(ctx, 4, stream);
   st = check_tuning(tuning);
   if (st != MOE_OK) return st;
   if (ctx->shape.T == 0) return MOE_OK;
@@ -200,7 +211,7 @@ moe_status moe_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_perm
                        void* out, void* stream) {
   moe_status st = check_ctx(ctx);
   if (st != MOE_OK) return st;
-  ctx->last_launches = 0;
+  begin_call(ctx, 6, stream);
   if (ctx->shape.T == 0) return MOE_OK;
   if (!y_perm || !inv_perm || !topk_w || !out) return MOE_ERR_INVALID_ARG;
   if (!aligned16(y_perm) || !aligned16(inv_perm) || !aligned16(topk_w) || !aligned16(out)) return MOE_ERR_INVALID_ARG;
@@ -214,11 +225,10 @@ moe_status moe_fused_forward(moe_ctx* ctx, const void* x, const float* logits, c
                              size_t workspace_bytes, const moe_tuning* tuning, void* stream) {
   moe_status st = check_ctx(ctx);
   if (st != MOE_OK) return st;
-  ctx->last_launches = 0;
   st = check_tuning(tuning);
   if (st != MOE_OK) return st;
   const moe_shape& s = ctx->shape;
-  if (s.T == 0) return MOE_OK;
+  if (s.T == 0) { ctx->last_launches = 0; return MOE_OK; }
   if (!x || !logits || !w_gate || !w_up || !w_down || !out || !workspace) return MOE_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(logits) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) ||
       !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
@@ -239,6 +249,7 @@ moe_status moe_fused_forward(moe_ctx* ctx, const void* x, const float* logits, c
   void* y_perm = ws + L.y_perm;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
+  begin_call(ctx, 0, stream);
   if (moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
     return MOE_ERR_CUDA;
   if (moe::launch_dispatch(ctx, x, inv_perm, x_perm, cs) != cudaSuccess) return MOE_ERR_CUDA;
@@ -291,5 +302,26 @@ moe_status moe_last_device_status(moe_ctx* ctx, int32_t* code, int32_t* detail, 
 }
 
 int32_t moe_last_launch_count(const moe_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+
+moe_status moe_set_kernel_timing(moe_ctx* ctx, int32_t enable) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->timing = enable ? 1 : 0;
+  ctx->ev_recorded = 0;
+  return MOE_OK;
+}
+
+moe_status moe_get_kernel_times(moe_ctx* ctx, float* ms_host, int32_t n) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  if (!ms_host || n != kMoeKernels) return MOE_ERR_INVALID_ARG;
+  for (int i = 0; i < kMoeKernels; ++i) {
+    ms_host[i] = -1.f;
+    const uint32_t need = (1u << i) | (1u << (i + 1));
+    if ((ctx->ev_recorded & need) != need) continue;
+    if (cudaEventSynchronize(ctx->ev[i + 1]) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms_host[i], ctx->ev[i], ctx->ev[i + 1]) != cudaSuccess) return MOE_ERR_CUDA;
+  }
+  return MOE_OK;
+}
 
 }  // extern "C"

@@ -8,6 +8,8 @@
 
 // Rows per M tile of the grouped GEMM and slots per routing chunk.
 constexpr int kRouteThreads = 256;
+// Kernels of one forward, in launch order: top-k+histogram, scan, scatter, dispatch, Linear-1, Linear-2, combine.
+constexpr int kMoeKernels = 7;
 
 typedef CUresult (*moe_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -25,7 +27,16 @@ struct moe_ctx {
   int32_t* d_status;      // [2] device status word: code, detail
   moe_encode_tiled_fn encode_tiled;
   int32_t last_launches;
+  // Optional per-kernel timing: event i is recorded after kernel i (event 0 before the first kernel).
+  int timing;
+  uint32_t ev_recorded;          // bit i set when ev[i] was recorded by the last call
+  cudaEvent_t ev[kMoeKernels + 1];
 };
+
+// Record timing mark i on the stream when per-kernel timing is enabled.
+inline void moe_mark(moe_ctx* ctx, int i, cudaStream_t stream) {
+  if (ctx->timing && cudaEventRecord(ctx->ev[i], stream) == cudaSuccess) ctx->ev_recorded |= 1u << i;
+}
 
 // Launchers (each returns the cudaError_t of its launches).  `stream` is the caller's stream.
 namespace moe {

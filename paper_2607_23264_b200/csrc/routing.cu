@@ -162,9 +162,12 @@ cudaError_t launch_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk
   const size_t smem3 = static_cast<size_t>(warps) * s.E * 4;
   route_topk_hist<<<ctx->num_chunks, kRouteThreads, smem1, stream>>>(logits, s.T, s.E, s.k, ctx->tokens_per_chunk,
                                                                      topk_ids, topk_w, ctx->d_chunk_hist);
+  moe_mark(ctx, 1, stream);
   route_scan<<<1, 1024, 0, stream>>>(ctx->d_chunk_hist, ctx->d_chunk_base, ctx->num_chunks, s.E, counts, offsets);
+  moe_mark(ctx, 2, stream);
   route_scatter<<<ctx->num_chunks, kRouteThreads, smem3, stream>>>(topk_ids, offsets, ctx->d_chunk_base, s.T, s.E,
                                                                    s.k, ctx->tokens_per_chunk, perm, inv_perm);
+  moe_mark(ctx, 3, stream);
   ctx->last_launches += 3;
   return cudaGetLastError();
 }
