@@ -148,7 +148,8 @@ def workload_config(cfg, n_gpus):
     return {"workload": f"{cfg.name}: T={cfg.T} tokens per GPU, hidden={cfg.H}, ffn={cfg.F}, E={cfg.E}, top-{cfg.k}, "
                         f"SwiGLU, bf16, router={cfg.router}, seed={cfg.seed}",
             "tokens_per_gpu": cfg.T, "global_tokens": cfg.T * n_gpus, "parallelism": f"ep1 x {n_gpus} replicas",
-            "l2_policy": "inputs larger than L2 (weights 2.8 GB + activations 1.1 GB per step vs 126 MB L2)"}
+            "l2_policy": "inputs larger than L2 (%.1f GB of weights + %.2f GB of activations per step vs 126 MB L2)"
+                         % (6 * cfg.E * cfg.H * cfg.F / 1e9, (2 * cfg.T * cfg.H + 4 * cfg.R * cfg.H + 2 * cfg.R * cfg.F) * 2 / 1e9)}
 
 
 def main():
@@ -165,6 +166,8 @@ def main():
     ap.add_argument("--mode", type=int, default=0)
     ap.add_argument("--ik", type=int, default=1)
     ap.add_argument("--sweep", action="store_true", help="store-pacing sweep (20 points) instead of the bench line")
+    ap.add_argument("--profile", action="store_true",
+                    help="profiler run: warm-up and timed steps only (no per-kernel pass, end-to-end or CPU legs)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -197,7 +200,7 @@ def main():
     w_gate = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
     w_up = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
     w_down = torch.empty((cfg.E, cfg.H, cfg.F), dtype=torch.bfloat16, device=dev)
-    keep_host = rank == 0 and not args.no_cpu_baseline and not args.sweep and cfg.E <= 16
+    keep_host = rank == 0 and not (args.no_cpu_baseline or args.sweep or args.profile) and cfg.E <= 16
     host_w = {}
 
     def sink(e, g, u, d):
@@ -268,6 +271,14 @@ def main():
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
+
+    if args.profile:
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "ms_per_step": total_ms / args.steps,
+                              "config": workload_config(cfg, world), "clocks": clocks}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # per-kernel average launch duration: the same steps again, reading the event pairs after each step
     for _ in range(args.steps):

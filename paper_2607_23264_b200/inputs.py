@@ -63,6 +63,11 @@ CONFIGS = {
     "C3": MoEConfig("C3", T=4096, H=7168, F=2048, E=256, k=8, seed=2, router="xWr_zipf"),
     # decode-like small batch, uniform-random routing
     "C4": MoEConfig("C4", T=64, H=7168, F=2048, E=256, k=8, seed=3, router="iid"),
+    # profiler-sized cases (small device footprint, still larger than L2):
+    # P1 = two Mixtral-like experts at C2's rows per expert (a quarter of C2's grouped-GEMM work)
+    "P1": MoEConfig("P1", T=2048, H=4096, F=14336, E=2, k=2, seed=4, router="xWr"),
+    # P2 = C2's row movers (dispatch/combine traffic of a 16384-token batch) with token-sized experts
+    "P2": MoEConfig("P2", T=16384, H=4096, F=64, E=8, k=2, seed=5, router="xWr"),
 }
 
 
