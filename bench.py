@@ -31,8 +31,10 @@ from paper_2607_23264_b200 import inputs as gen  # noqa: E402
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one expert_gemm_kernel<true> (Linear-1) launch on the
-# bench workload, from the ncu capture summarised in profiles/; None until a capture exists.
-LINEAR1_DRAM_TRAFFIC_BYTES = None
+# C2 workload: the ncu capture of the two-expert case P1 (503.5 MB read + 106.9 MB written, see
+# profiles/expert_gemm_P1_ncu_full.md) scaled by 4, since DRAM traffic is per expert and C2 has four times
+# P1's experts at the same rows per expert.
+LINEAR1_DRAM_TRAFFIC_BYTES = {"C2": 4 * (503_479_040 + 106_861_824)}
 
 
 def load_peaks():
@@ -322,7 +324,7 @@ def main():
     peak_tf = float(peaks["bf16_tflops"])
     roofline = {
         "kernel": "expert_gemm_kernel<gated> (Linear-1 + SiLU*mul)", "bound": "tensor", "achieved": l1_tf,
-        "peak": peak_tf, "unit": "TFLOP/s", "frac": l1_tf / peak_tf, "traffic": LINEAR1_DRAM_TRAFFIC_BYTES,
+        "peak": peak_tf, "unit": "TFLOP/s", "frac": l1_tf / peak_tf, "traffic": LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name),
         "peak_source": f"{peak_kind} bf16_tflops (burst)",
         "frac_of_sustained": l1_tf / float(peaks.get("bf16_tflops_sustained", peak_tf)),
         "flops_per_launch": l1_flops, "ms_per_launch": kernel_ms[4],
