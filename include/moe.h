@@ -37,7 +37,8 @@ typedef enum {
   MOE_ERR_BAD_ROUTING = 4,         /* reserved: routing input violates the contract */
   MOE_ERR_CUDA = 5,                /* a CUDA runtime or driver call failed */
   MOE_ERR_TIMEOUT = 6,             /* device status only: a bounded on-device wait expired */
-  MOE_ERR_UNSUPPORTED = 7          /* ep_size != 1, unknown schedule */
+  MOE_ERR_UNSUPPORTED = 7,         /* ep_size != 1, unknown schedule */
+  MOE_ERR_STATIC_SCRATCH_TOO_SMALL = 8  /* moe_plan_routing_static: the shape exceeds the built-in scratch */
 } moe_status;
 
 typedef struct {
@@ -112,6 +113,32 @@ moe_status moe_get_workspace_layout(const moe_shape* shape, moe_workspace_layout
 moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids, float* topk_w,
                             int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
                             void* stream);
+
+/*
+ * The routing plan for callers that must not allocate.  (The paper has no counterpart: this entry point
+ * exists for the library's users, not for the method.)
+ *
+ * moe_create obtains its scratch with cudaMalloc.  Some callers cannot do that: code that runs after a
+ * framework has handed the whole device to its own memory pool, plugins whose execute hook is forbidden
+ * to allocate, or a serving loop that cannot afford the device-wide synchronisation an allocation may
+ * imply.  This call needs no context and calls no cudaMalloc, cudaFree or allocating library routine.
+ * Its scratch (the per-chunk histograms and their prefix) is a fixed array of 512 KiB that is part of
+ * the library image: every GPU on which the library is loaded holds it until the process exits.
+ *
+ * Same inputs, outputs and results as moe_plan_routing (shape->T, E, k are used; H and F are ignored).
+ *   - Limit: ceil(T / floor(256/k)) * E <= 65536, e.g. T <= 8192 at E = 256, k = 8.  Beyond it the call
+ *     returns MOE_ERR_STATIC_SCRATCH_TOO_SMALL and launches nothing.
+ *   - The first call on each device looks up the array's device address (with that device current).
+ *     Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (each call
+ *     rewrites every entry it later reads), so calls may follow one another on a stream freely; two
+ *     calls that overlap on the GPU (different streams, no ordering) race on it and give wrong plans.
+ *   - Works on the calling thread's current device.  Errors: INVALID_ARG (null or misaligned pointer),
+ *     UNSUPPORTED_SHAPE, UNSUPPORTED (ep_size != 1), STATIC_SCRATCH_TOO_SMALL, CUDA.
+ */
+moe_status moe_plan_routing_static(const moe_shape* shape, const float* logits, int32_t* topk_ids,
+                                   float* topk_w, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                   int32_t* inv_perm, void* stream);
 
 /*
  * Dispatch (Sec. 2.2 / Sec. 4.3 "Dispatch input"): x_perm[inv_perm[t*k+j], :] = x[t, :] for every slot,

@@ -16,13 +16,14 @@ MOE_OK = 0
 STATUS_NAMES = {
     0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED_SHAPE", 3: "MOE_ERR_WORKSPACE_TOO_SMALL",
     4: "MOE_ERR_BAD_ROUTING", 5: "MOE_ERR_CUDA", 6: "MOE_ERR_TIMEOUT", 7: "MOE_ERR_UNSUPPORTED",
+    8: "MOE_ERR_STATIC_SCRATCH_TOO_SMALL",
 }
 
 EXPORTS = (
     "moe_status_string", "moe_create", "moe_destroy", "moe_workspace_bytes", "moe_get_workspace_layout",
     "moe_plan_routing", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_fused_forward",
     "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count", "moe_set_kernel_timing",
-    "moe_get_kernel_times",
+    "moe_get_kernel_times", "moe_plan_routing_static",
 )
 
 KERNEL_NAMES = ("route_topk_hist", "route_scan", "route_scatter", "dispatch_rows", "expert_gemm_linear1",
@@ -72,6 +73,7 @@ def load_library() -> C.CDLL:
     lib.moe_workspace_bytes.restype = C.c_size_t
     lib.moe_get_workspace_layout.argtypes = [C.POINTER(moe_shape), C.POINTER(moe_workspace_layout)]
     lib.moe_plan_routing.argtypes = [vp, f32p, i32p, f32p, i32p, i32p, i32p, i32p, vp]
+    lib.moe_plan_routing_static.argtypes = [C.POINTER(moe_shape), f32p, i32p, f32p, i32p, i32p, i32p, i32p, vp]
     lib.moe_dispatch.argtypes = [vp, vp, i32p, vp, vp]
     lib.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp, f32p, C.POINTER(moe_tuning), vp]
     lib.moe_combine.argtypes = [vp, vp, i32p, f32p, vp, vp]
@@ -133,6 +135,15 @@ def moe_get_workspace_layout(T, H, F, E, k) -> dict:
     _check(load_library().moe_get_workspace_layout(C.byref(moe_shape(T, H, F, E, k, 1, 0)), C.byref(L)),
            "moe_get_workspace_layout")
     return {n: getattr(L, n) for n, _ in moe_workspace_layout._fields_}
+
+
+def moe_plan_routing_static(T, E, k, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, stream=None):
+    """Routing plan through the entry point that allocates nothing and needs no context: its scratch is a
+    fixed array inside the library (see include/moe.h for the size limit and the sharing rules)."""
+    shape = moe_shape(T, 0, 0, E, k, 1, 0)
+    _check(load_library().moe_plan_routing_static(C.byref(shape), _ptr(logits), _ptr(topk_ids), _ptr(topk_w),
+                                                  _ptr(counts), _ptr(offsets), _ptr(perm), _ptr(inv_perm),
+                                                  _stream(stream)), "moe_plan_routing_static")
 
 
 @dataclass

@@ -80,6 +80,7 @@ const char* moe_status_string(moe_status s) {
     case MOE_ERR_CUDA: return "MOE_ERR_CUDA";
     case MOE_ERR_TIMEOUT: return "MOE_ERR_TIMEOUT";
     case MOE_ERR_UNSUPPORTED: return "MOE_ERR_UNSUPPORTED";
+    case MOE_ERR_STATIC_SCRATCH_TOO_SMALL: return "MOE_ERR_STATIC_SCRATCH_TOO_SMALL";
   }
   return "MOE_ERR_UNKNOWN";
 }

@@ -173,3 +173,68 @@ cudaError_t launch_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk
 }
 
 }  // namespace moe
+
+
+// ------------------------------------------------------------------------------------------------
+// Routing plan without any allocation: same three kernels, scratch in a file-scope device array.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+// Largest num_chunks * E the static scratch holds (two arrays of this many int32: 512 KiB in total,
+// resident on every GPU that loads the library until the process exits).
+constexpr int kStaticScratchInts = 65536;
+static __device__ __align__(256) int32_t g_route_static_scratch[2 * kStaticScratchInts];
+
+constexpr int kMaxDevices = 64;
+int32_t* g_route_static_addr[kMaxDevices] = {};   // device address of the array, per device, once resolved
+
+}  // namespace
+
+extern "C" moe_status moe_plan_routing_static(const moe_shape* shape, const float* logits, int32_t* topk_ids,
+                                              float* topk_w, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                              int32_t* inv_perm, void* stream) {
+  if (!shape) return MOE_ERR_INVALID_ARG;
+  if (shape->ep_size != 1 || shape->ep_rank != 0) return MOE_ERR_UNSUPPORTED;
+  if (shape->T < 0 || shape->E <= 0 || shape->k <= 0 || shape->E > 1024 || shape->k > 32 || shape->k > shape->E)
+    return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (!counts || !offsets) return MOE_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const int T = shape->T, E = shape->E, k = shape->k;
+  if (T == 0) {
+    if (cudaMemsetAsync(counts, 0, static_cast<size_t>(E) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaMemsetAsync(offsets, 0, static_cast<size_t>(E + 1) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+  }
+  if (!logits || !topk_ids || !topk_w || !perm || !inv_perm) return MOE_ERR_INVALID_ARG;
+  const void* ptrs[] = {logits, topk_ids, topk_w, counts, offsets, perm, inv_perm};
+  for (const void* q : ptrs)
+    if (reinterpret_cast<uintptr_t>(q) & 15u) return MOE_ERR_INVALID_ARG;
+
+  const int tokens_per_chunk = kRouteThreads / k;
+  const long long num_chunks = (static_cast<long long>(T) + tokens_per_chunk - 1) / tokens_per_chunk;
+  if (num_chunks * E > kStaticScratchInts) return MOE_ERR_STATIC_SCRATCH_TOO_SMALL;
+
+  // Set-up, once per device, with that device current: in host code the array's name is only a
+  // stand-in, the address a kernel may use comes from cudaGetSymbolAddress.
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MOE_ERR_CUDA;
+  int32_t* scratch = g_route_static_addr[dev];
+  if (!scratch) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_route_static_scratch) != cudaSuccess || !addr) return MOE_ERR_CUDA;
+    scratch = static_cast<int32_t*>(addr);
+    g_route_static_addr[dev] = scratch;
+  }
+  int32_t* chunk_hist = scratch;                        // [num_chunks, E], every entry rewritten by kernel 1
+  int32_t* chunk_base = scratch + kStaticScratchInts;   // [num_chunks, E], every entry rewritten by kernel 2
+
+  const int warps = kRouteThreads / 32;
+  const size_t smem1 = (static_cast<size_t>(warps) * E + E + 256) * 4;
+  const size_t smem3 = static_cast<size_t>(warps) * E * 4;
+  const int nc = static_cast<int>(num_chunks);
+  route_topk_hist<<<nc, kRouteThreads, smem1, cs>>>(logits, T, E, k, tokens_per_chunk, topk_ids, topk_w, chunk_hist);
+  route_scan<<<1, 1024, 0, cs>>>(chunk_hist, chunk_base, nc, E, counts, offsets);
+  route_scatter<<<nc, kRouteThreads, smem3, cs>>>(topk_ids, offsets, chunk_base, T, E, k, tokens_per_chunk, perm,
+                                                  inv_perm);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
