@@ -168,6 +168,8 @@ def main():
     ap.add_argument("--mode", type=int, default=0)
     ap.add_argument("--ik", type=int, default=1)
     ap.add_argument("--sweep", action="store_true", help="store-pacing sweep (20 points) instead of the bench line")
+    ap.add_argument("--trace", action="store_true",
+                    help="add the grouped GEMMs' per-CTA wait counters (one extra traced step) to the JSON line")
     ap.add_argument("--profile", action="store_true",
                     help="profiler run: warm-up and timed steps only (no per-kernel pass, end-to-end or CPU legs)")
     args = ap.parse_args()
@@ -289,6 +291,20 @@ def main():
     ctx.moe_set_kernel_timing(False)
     kernel_ms = [float(np.mean([s[i] for s in per_step_kernel])) for i in range(len(binding.KERNEL_NAMES))]
 
+    ffn_trace = None
+    if args.trace:
+        ttn = binding.make_tuning(args.burst, args.mode, args.ik, debug_flags=1)
+        ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=ttn)
+        tr = ctx.moe_get_ffn_trace().astype(np.float64)          # [2, CTAs, 8]
+        ffn_trace = {}
+        for i, name in enumerate(("linear1", "linear2")):
+            mean = tr[i].mean(axis=0)
+            tiles = max(mean[6], 1.0)
+            ffn_trace[name] = {f: float(v) for f, v in zip(binding.TRACE_FIELDS, mean)}
+            ffn_trace[name]["per_tile_clocks"] = {f: float(v / tiles) for f, v in zip(binding.TRACE_FIELDS, mean)
+                                                  if f != "tiles"}
+            ffn_trace[name]["tiles_min_max"] = [float(tr[i][:, 6].min()), float(tr[i][:, 6].max())]
+
     code, detail = ctx.moe_last_device_status()
     if code != 0:
         raise RuntimeError(f"device status {binding.STATUS_NAMES.get(code, code)} detail {detail:#x}")
@@ -322,13 +338,35 @@ def main():
     disp_gbs = move_bytes / (kernel_ms[3] * 1e-3) / 1e9
     comb_gbs = (move_bytes + 8 * R) / (kernel_ms[6] * 1e-3) / 1e9
     peak_tf = float(peaks["bf16_tflops"])
-    roofline = {
-        "kernel": "expert_gemm_kernel<gated> (Linear-1 + SiLU*mul)", "bound": "tensor", "achieved": l1_tf,
-        "peak": peak_tf, "unit": "TFLOP/s", "frac": l1_tf / peak_tf, "traffic": LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name),
-        "peak_source": f"{peak_kind} bf16_tflops (burst)",
-        "frac_of_sustained": l1_tf / float(peaks.get("bf16_tflops_sustained", peak_tf)),
-        "flops_per_launch": l1_flops, "ms_per_launch": kernel_ms[4],
-    }
+    peak_hbm = float(peaks["hbm_gbs"])
+    lay = ctx.workspace_layout()
+    counts = ws[lay["counts"]:lay["counts"] + 4 * cfg.E].view(torch.int32).cpu().numpy()
+    nonempty = int((counts > 0).sum())
+    # algorithmic bytes of one Linear-1 launch: gate+up weights of the non-empty experts, x_perm read, h written
+    l1_bytes = nonempty * 2 * cfg.F * cfg.H * 2 + R * cfg.H * 2 + R * cfg.F * 2
+    l2_bytes = nonempty * cfg.F * cfg.H * 2 + R * cfg.F * 2 + R * cfg.H * 2
+    l1_gbs = l1_bytes / (kernel_ms[4] * 1e-3) / 1e9
+    l2_gbs = l2_bytes / (kernel_ms[5] * 1e-3) / 1e9
+    # the roofline that binds Linear-1: tensor time at the measured GEMM peak vs HBM time at the measured copy rate
+    t_tensor = l1_flops / (peak_tf * 1e12)
+    t_hbm = l1_bytes / (peak_hbm * 1e9)
+    if t_tensor >= t_hbm:
+        roofline = {
+            "kernel": "expert_gemm_kernel<gated> (Linear-1 + SiLU*mul)", "bound": "tensor", "achieved": l1_tf,
+            "peak": peak_tf, "unit": "TFLOP/s", "frac": l1_tf / peak_tf,
+            "traffic": LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name),
+            "peak_source": f"{peak_kind} bf16_tflops (burst)",
+            "frac_of_sustained": l1_tf / float(peaks.get("bf16_tflops_sustained", peak_tf)),
+            "flops_per_launch": l1_flops, "ms_per_launch": kernel_ms[4],
+        }
+    else:
+        roofline = {
+            "kernel": "expert_gemm_kernel<gated> (Linear-1 + SiLU*mul)", "bound": "hbm", "achieved": l1_gbs,
+            "peak": peak_hbm, "unit": "GB/s", "frac": l1_gbs / peak_hbm,
+            "traffic": LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name), "peak_source": f"{peak_kind} hbm_gbs (copy)",
+            "bytes_per_launch": l1_bytes, "ms_per_launch": kernel_ms[4], "nonempty_experts": nonempty,
+            "tensor_tflops": l1_tf,
+        }
     line = {
         "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -336,13 +374,15 @@ def main():
         "config": workload_config(cfg, world),
         "tflops": tflops, "frac_bf16_peak": tflops / world / peak_tf,
         "kernels_ms": dict(zip(binding.KERNEL_NAMES, kernel_ms)),
-        "linear2_tflops": l2_tf, "dispatch_gbs": disp_gbs, "combine_gbs": comb_gbs,
+        "linear2_tflops": l2_tf, "linear1_gbs": l1_gbs, "linear2_gbs": l2_gbs, "dispatch_gbs": disp_gbs, "combine_gbs": comb_gbs,
         "dispatch_frac_hbm": disp_gbs / float(peaks["hbm_gbs"]), "combine_frac_hbm": comb_gbs / float(peaks["hbm_gbs"]),
         "roofline": roofline,
         "e2e": {"value": tokens / (e2e_ms / args.steps * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": launches, "clocks": clocks, "tuning": [args.burst, args.mode, args.ik],
     }
+    if ffn_trace is not None:
+        line["ffn_trace"] = ffn_trace
     if keep_host:
         rate, dt = oracle_sample_rate(cfg, x_bits, logits, lambda e: host_w[e], args.cpu_baseline_tokens)
         line["cpu_baseline"] = {
@@ -357,25 +397,55 @@ def main():
 
 
 def run_sweep(args, cfg, ctx, binding, bufs, timed, rank):
-    """Store-pacing sweep: burst in {1,2,4,8,16} x {after-mainloop, every-k-iterations k in {1,2,4}}."""
+    """Store-pacing sweep: burst in {1,2,4,8,16} x {after-mainloop, every-k-iterations k in {1,2,4}}.
+
+    The GPU is first brought to its steady power-capped state (about 1.5 s of steps); every point is then
+    timed in two passes (forward and reverse order) so that clock drift shows up as spread, not as a trend.
+    Per point: median/min ms per step, TFLOP/s, algorithmic HBM GB/s, per-kernel times, and from one traced step
+    the Linear-2 per-tile epilogue store span, pacing hold and MMA wait for a free accumulator (SM clocks)."""
     import torch
     x, d_logits, w_gate, w_up, w_down, out, ws = bufs
     points = [(b, 0, 1) for b in (1, 2, 4, 8, 16)] + [(b, 1, ik) for b in (1, 2, 4, 8, 16) for ik in (1, 2, 4)]
+    run = lambda tn: ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tn)
+    t0 = time.time()
+    while time.time() - t0 < 1.5:
+        for _ in range(20):
+            run(None)
+        torch.cuda.synchronize()
     base = None
+    samples = {pt: [] for pt in points}
+    extra = {}
+    R = cfg.R
+    step_bytes = (6 * cfg.E * cfg.H * cfg.F + 2 * (2 * cfg.T * cfg.H + 4 * R * cfg.H + 2 * R * cfg.F))
+    for order in (points, points[::-1]):
+        for pt in order:
+            tn = binding.make_tuning(*pt)
+            ms = timed(lambda: run(tn), args.steps, max(1, args.warmup)) / args.steps
+            samples[pt].append(ms)
+            if pt not in extra:
+                ctx.moe_set_kernel_timing(True)
+                run(tn)
+                km = ctx.moe_get_kernel_times()
+                ctx.moe_set_kernel_timing(False)
+                bits = out.view(torch.int16).clone()
+                if base is None:
+                    base = bits
+                run(binding.make_tuning(*pt, debug_flags=1))
+                tr = ctx.moe_get_ffn_trace().astype(np.float64)
+                l2 = tr[1].mean(axis=0)
+                tiles = max(l2[6], 1.0)
+                extra[pt] = {"linear1_ms": km[4], "linear2_ms": km[5], "identical_bits": bool(torch.equal(bits, base)),
+                             "l2_store_span_clk_per_tile": l2[5] / tiles, "l2_pacing_hold_clk_per_tile": l2[7] / tiles,
+                             "l2_mma_wait_accumulator_clk_per_tile": l2[3] / tiles,
+                             "l2_mma_wait_operands_frac": l2[2] / max(l2[0], 1.0)}
     rows = []
-    ctx.moe_set_kernel_timing(True)
-    for b, mode, ik in points:
-        tn = binding.make_tuning(b, mode, ik)
-        fn = lambda: ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tn)
-        ms = timed(fn, args.steps, max(1, args.warmup)) / args.steps
-        km = ctx.moe_get_kernel_times()
-        bits = out.view(torch.int16).clone()
-        if base is None:
-            base = bits
-        rows.append({"burst": b, "mode": mode, "k": ik, "ms_per_step": ms, "linear1_ms": km[4], "linear2_ms": km[5],
-                     "tflops": cfg.flops / (ms * 1e-3) / 1e12, "identical_bits": bool(torch.equal(bits, base))})
+    for pt in points:
+        ms = statistics.median(samples[pt])
+        rows.append({"burst": pt[0], "mode": pt[1], "k": pt[2], "ms_per_step": ms, "ms_min": min(samples[pt]),
+                     "ms_max": max(samples[pt]), "tflops": cfg.flops / (ms * 1e-3) / 1e12,
+                     "hbm_gbs_algorithmic": step_bytes / (ms * 1e-3) / 1e9, **extra[pt]})
     if rank == 0:
-        print(json.dumps({"sweep": rows, "config": workload_config(cfg, 1)}), flush=True)
+        print(json.dumps({"sweep": rows, "config": workload_config(cfg, 1), "steps_per_sample": args.steps}), flush=True)
 
 
 if __name__ == "__main__":

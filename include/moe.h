@@ -62,7 +62,7 @@ typedef struct {
   int32_t interleave_k;            /* 1, 2 or 4; used when interleave_mode == 1 */
   int32_t schedule;                /* 0 = expert-wave order (Sec. 4.3): all Linear-1 tiles, then Linear-2 */
   int32_t dep_lead_D;              /* reserved for the interleaved schedule (Algorithm 1); must be 0 */
-  int32_t debug_flags;             /* must be 0 */
+  int32_t debug_flags;             /* bit 0: record per-CTA wait counters (moe_get_ffn_trace); other bits 0 */
 } moe_tuning;
 
 /* Byte offsets of the slices of the workspace used by moe_fused_forward (each 256-byte aligned). */
@@ -201,6 +201,20 @@ moe_status moe_last_device_status(moe_ctx* ctx, int32_t* code, int32_t* detail, 
 
 /* Number of kernels the last call on this context launched (host-side count, for benchmarking). */
 int32_t moe_last_launch_count(const moe_ctx* ctx);
+
+/*
+ * Wait counters of the two grouped GEMMs (the instrumentation of Sec. 5.1 / App. A.2: per-tile store spans and
+ * the MMA-side wait for a free accumulator, there read with clock64()).  When a call ran with
+ * tuning->debug_flags bit 0 set, every CTA of Linear-1 and of Linear-2 recorded eight 64-bit counters, in SM
+ * clocks: 0 producer loop span, 1 producer waited for a free shared-memory stage, 2 MMA warp waited for
+ * operands, 3 MMA warp waited for a free accumulator (the epilogue's back-pressure, the paper's tmem_empty
+ * wait), 4 epilogue waited for a finished accumulator, 5 epilogue drain-and-store span, 6 tiles processed
+ * (a count), 7 epilogue held by the pacing gap.  This call synchronises `stream` and copies
+ * counters_host[2][*num_ctas][8] (Linear-1 first) to HOST memory; capacity is in 64-bit elements and must be
+ * at least 16 * (number of SMs).
+ */
+moe_status moe_get_ffn_trace(moe_ctx* ctx, uint64_t* counters_host, int32_t capacity, int32_t* num_ctas,
+                             void* stream);
 
 /*
  * Per-kernel timing (measurement aid; the paper times its kernel with CUDA events, Sec. 5.1).  When

@@ -23,8 +23,11 @@ EXPORTS = (
     "moe_status_string", "moe_create", "moe_destroy", "moe_workspace_bytes", "moe_get_workspace_layout",
     "moe_plan_routing", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_fused_forward",
     "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count", "moe_set_kernel_timing",
-    "moe_get_kernel_times", "moe_plan_routing_static",
+    "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace",
 )
+
+TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
+                "epilogue_wait_accumulator", "epilogue_store_span", "tiles", "epilogue_pacing_gap")
 
 KERNEL_NAMES = ("route_topk_hist", "route_scan", "route_scatter", "dispatch_rows", "expert_gemm_linear1",
                 "expert_gemm_linear2", "combine_rows")
@@ -84,6 +87,7 @@ def load_library() -> C.CDLL:
     lib.moe_last_launch_count.restype = C.c_int32
     lib.moe_set_kernel_timing.argtypes = [vp, C.c_int32]
     lib.moe_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32]
+    lib.moe_get_ffn_trace.argtypes = [vp, C.POINTER(C.c_uint64), C.c_int32, C.POINTER(C.c_int32), vp]
     for name in EXPORTS:
         if name not in ("moe_status_string", "moe_destroy", "moe_workspace_bytes", "moe_last_launch_count"):
             getattr(lib, name).restype = C.c_int
@@ -229,6 +233,16 @@ class Context:
 
     def moe_last_launch_count(self) -> int:
         return self._lib.moe_last_launch_count(self._handle)
+
+    def moe_get_ffn_trace(self, stream=None):
+        """Wait counters of the last traced call as a numpy array [2 (Linear-1, Linear-2), CTAs, 8]."""
+        import numpy as np
+        cap = 2 * 1024 * len(TRACE_FIELDS)
+        buf = (C.c_uint64 * cap)()
+        n = C.c_int32(0)
+        _check(self._lib.moe_get_ffn_trace(self._handle, buf, cap, C.byref(n), _stream(stream)), "moe_get_ffn_trace")
+        a = np.frombuffer(buf, dtype=np.uint64)[: 2 * n.value * len(TRACE_FIELDS)]
+        return a.reshape(2, n.value, len(TRACE_FIELDS)).copy()
 
     def moe_set_kernel_timing(self, enable: bool):
         _check(self._lib.moe_set_kernel_timing(self._handle, 1 if enable else 0), "moe_set_kernel_timing")

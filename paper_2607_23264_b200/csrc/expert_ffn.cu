@@ -11,8 +11,13 @@
 // two 256-column accumulators let the epilogue of tile i overlap the mainloop of tile i+1.
 // Expert row ranges are ragged: a tile may cover rows of the next expert (or past R, zero-filled by
 // TMA); those rows are computed and discarded, stores are masked to the expert's own rows.
-// Tile order is expert-major, then N block, then M block (fastest), so the CTAs running at the same
-// time share one weight tile through L2 and an expert's weights stream from HBM once.
+// Tile order inside an expert is N block, then M block (fastest), so the CTAs running at the same time
+// share one weight tile through L2 and an expert's weights stream from HBM once.  Experts are split into
+// "hot" ones (several 128-row blocks: their tiles are tensor-bound) and "cold" ones (few rows: their
+// tiles only stream weights and are HBM-bound); the global order merges the hot and the cold tile lists
+// at a fixed ratio so that both finish together, and CTAs draw tiles from it dynamically (one atomic
+// counter).  At any time some SMs then keep the tensor pipes busy while others keep HBM busy, instead of
+// the two kinds of work running one after the other.
 #include <cuda_bf16.h>
 
 #include "moe_internal.h"
@@ -32,17 +37,23 @@ constexpr int kThreads = 192;
 constexpr int kMaxExperts = 1024;
 constexpr int kTmemCols = 512;
 constexpr int kChunkCols = 32;     // accumulator columns per tcgen05.ld = columns of one store tile
+constexpr int kRing = 4;           // tile ids the producer may publish ahead of the consumers
+constexpr int kHotBlocks = 2;      // experts with at least this many 128-row blocks count as tensor-bound
 
 struct SharedTail {
   uint64_t full[kStages];
   uint64_t empty[kStages];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
+  uint64_t ring_full[kRing];
+  uint64_t ring_empty[kRing];
+  int32_t ring_tile[kRing];         // tile ids drawn by the producer; -1 = no more tiles
   uint32_t tmem_base;
   volatile int abort_flag;
   volatile uint32_t mma_progress;   // K-blocks issued so far by the MMA warp (pacing clock)
   volatile int mma_idle;            // 1 while the MMA warp waits for an accumulator or has finished
-  int32_t mblk_prefix[kMaxExperts + 1];   // exclusive prefix of 128-row blocks per expert
+  int32_t hot_prefix[kMaxExperts + 1];    // exclusive prefix of 128-row blocks over hot experts (cold count 0)
+  int32_t cold_prefix[kMaxExperts + 1];   // the same over cold experts
 };
 
 constexpr size_t kSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStages) * kStageBytes + sizeof(SharedTail);
@@ -60,6 +71,8 @@ struct FfnParams {
   float* h_dbg;             // Linear-1 only: fp32 copy of h before rounding, or nullptr
   int burst, mode, ik;      // store pacing
   int32_t* status;          // [2]
+  int32_t* sched;           // [2] next tile to draw, CTAs finished; both zero between launches
+  unsigned long long* trace;   // nullptr, or [gridDim.x][kMoeTraceFields] wait counters in SM clocks
   int kernel_id;
 };
 
@@ -70,7 +83,16 @@ struct Tile {
   int w_row0;    // first row of the weight box in the [E*N, K] weight matrix
 };
 
-__device__ __forceinline__ Tile decode_tile(int tile, const int32_t* prefix, const FfnParams& p) {
+// Position `pos` of the merged order -> tile.  Among the first `pos` positions floor(pos*cold/total) are
+// cold tiles; position pos is itself cold when that count steps up at pos+1.
+__device__ __forceinline__ Tile decode_tile(int pos, const SharedTail* st, const FfnParams& p) {
+  const long long hot_tiles = static_cast<long long>(st->hot_prefix[p.E]) * p.n_blocks;
+  const long long cold_tiles = static_cast<long long>(st->cold_prefix[p.E]) * p.n_blocks;
+  const long long total = hot_tiles + cold_tiles;
+  const long long cold_before = (static_cast<long long>(pos) * cold_tiles) / total;
+  const bool is_cold = ((static_cast<long long>(pos) + 1) * cold_tiles) / total > cold_before;
+  const int tile = static_cast<int>(is_cold ? cold_before : pos - cold_before);
+  const int32_t* prefix = is_cold ? st->cold_prefix : st->hot_prefix;
   const int q = tile / p.n_blocks;   // lies in [prefix[e], prefix[e+1]) of the owning expert
   int lo = 0, hi = p.E;              // invariant: prefix[lo] <= q < prefix[hi]
   while (hi - lo > 1) {
@@ -127,28 +149,39 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       ptx::mbar_init(ptx::smem_u32(&st->tmem_full[a]), 1);
       ptx::mbar_init(ptx::smem_u32(&st->tmem_empty[a]), 4);   // one arrival per epilogue warp
     }
+    for (int r = 0; r < kRing; ++r) {
+      ptx::mbar_init(ptx::smem_u32(&st->ring_full[r]), 1);
+      ptx::mbar_init(ptx::smem_u32(&st->ring_empty[r]), 5);   // MMA thread + four epilogue warps
+    }
     st->abort_flag = 0;
     st->mma_progress = 0;
     st->mma_idle = 0;
-    st->mblk_prefix[0] = 0;
+    st->hot_prefix[0] = 0;
+    st->cold_prefix[0] = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async_smem();
   }
   if (warp == 0) {
-    // exclusive prefix of ceil(count/128) over experts, 32 experts per step
-    int32_t run = 0;
+    // exclusive prefixes of ceil(count/128) over experts (hot and cold apart), 32 experts per step
+    int32_t run_hot = 0, run_cold = 0;
     for (int base = 0; base < p.E; base += 32) {
       const int e = base + lane;
       int32_t v = 0;
       if (e < p.E) v = (p.offsets[e + 1] - p.offsets[e] + BM - 1) / BM;
-      int32_t incl = v;
+      int32_t hot = v >= kHotBlocks ? v : 0;
+      int32_t cold = v - hot;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
-        const int32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-        if (lane >= off) incl += o;
+        const int32_t oh = __shfl_up_sync(0xFFFFFFFFu, hot, off);
+        const int32_t oc = __shfl_up_sync(0xFFFFFFFFu, cold, off);
+        if (lane >= off) { hot += oh; cold += oc; }
       }
-      if (e < p.E) st->mblk_prefix[e + 1] = run + incl;
-      run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      if (e < p.E) {
+        st->hot_prefix[e + 1] = run_hot + hot;
+        st->cold_prefix[e + 1] = run_cold + cold;
+      }
+      run_hot += __shfl_sync(0xFFFFFFFFu, hot, 31);
+      run_cold += __shfl_sync(0xFFFFFFFFu, cold, 31);
     }
     if (lane == 0) {
       ptx::prefetch_tensormap(&tm_a);
@@ -165,7 +198,7 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
   ptx::tc_fence_after_sync();
 
   const uint32_t tmem_base = st->tmem_base;
-  const int total_tiles = st->mblk_prefix[p.E] * p.n_blocks;
+  const int total_tiles = (st->hot_prefix[p.E] + st->cold_prefix[p.E]) * p.n_blocks;
   const int k_blocks = (p.K + BK - 1) / BK;
   volatile int* abort_flag = &st->abort_flag;
 
@@ -174,11 +207,27 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
+      int slot = 0;
+      uint32_t ring_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const Tile t = decode_tile(tile, st->mblk_prefix, p);
+      long long w_empty = 0;
+      const long long t_begin = clock64();
+      while (ok) {
+        // draw the next tile and publish it to the MMA and epilogue roles
+        if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_empty[slot]), ring_phase ^ 1u, abort_flag)) {
+          atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
+          atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 5);
+          break;
+        }
+        int pos = atomicAdd(&p.sched[0], 1);
+        if (pos >= total_tiles) pos = -1;
+        st->ring_tile[slot] = pos;
+        ptx::mbar_arrive(ptx::smem_u32(&st->ring_full[slot]));
+        if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
+        if (pos < 0) break;
+        const Tile t = decode_tile(pos, st, p);
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag)) {
+          if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, &w_empty)) {
             atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
             atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 1);
             ok = false;
@@ -193,6 +242,10 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
+      if (p.trace) {
+        p.trace[blockIdx.x * kMoeTraceFields + 0] = static_cast<unsigned long long>(clock64() - t_begin);
+        p.trace[blockIdx.x * kMoeTraceFields + 1] = static_cast<unsigned long long>(w_empty);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -203,10 +256,23 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       int acc = 0;
       uint32_t acc_phase = 0;
       uint32_t progress = 0;
+      int slot = 0;
+      uint32_t ring_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      long long w_full = 0, w_tmem = 0;
+      unsigned long long n_tiles = 0;
+      while (ok) {
         st->mma_idle = 1;
-        if (!ptx::mbar_wait(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) {
+        if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
+          atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
+          atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 6);
+          break;
+        }
+        const int pos = st->ring_tile[slot];
+        ptx::mbar_arrive(ptx::smem_u32(&st->ring_empty[slot]));
+        if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
+        if (pos < 0) break;
+        if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, &w_tmem)) {
           atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
           atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 2);
           break;
@@ -215,7 +281,7 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN_ACC);
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&st->full[stage]), phase, abort_flag)) {
+          if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), phase, abort_flag, &w_full)) {
             atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
             atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 3);
             ok = false;
@@ -239,8 +305,14 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
         ptx::tc_commit(ptx::smem_u32(&st->tmem_full[acc]));    // accumulator complete
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
+        ++n_tiles;
       }
       st->mma_idle = 1;
+      if (p.trace) {
+        p.trace[blockIdx.x * kMoeTraceFields + 2] = static_cast<unsigned long long>(w_full);
+        p.trace[blockIdx.x * kMoeTraceFields + 3] = static_cast<unsigned long long>(w_tmem);
+        p.trace[blockIdx.x * kMoeTraceFields + 6] = n_tiles;
+      }
     }
     __syncwarp();
   } else {
@@ -250,9 +322,24 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
     int acc = 0;
     uint32_t acc_phase = 0;
     const int burst = p.burst;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const Tile t = decode_tile(tile, st->mblk_prefix, p);
-      if (!ptx::mbar_wait(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag)) {
+    int slot = 0;
+    uint32_t ring_phase = 0;
+    long long w_acc = 0, busy = 0, w_gap = 0;
+    while (true) {
+      if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
+        if (lane == 0) {
+          atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
+          atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 7);
+        }
+        break;
+      }
+      const int pos = st->ring_tile[slot];
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->ring_empty[slot]));
+      if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
+      if (pos < 0) break;
+      const Tile t = decode_tile(pos, st, p);
+      if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, &w_acc)) {
         if (lane == 0) {
           atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
           atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 4);
@@ -260,6 +347,7 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
         break;
       }
       ptx::tc_fence_after_sync();
+      const long long t_store = clock64();
       const int row = t.row0 + r_in_tile;
       const bool row_ok = row < t.row_end;
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
@@ -311,7 +399,9 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
           }
         }
         if (p.mode == 1 && ++in_burst >= burst && c + 1 < kChunks) {
+          const long long t_gap = clock64();
           pace_gap(st, gap_start, p.ik);
+          w_gap += clock64() - t_gap;
           gap_start = st->mma_progress;
           in_burst = 0;
         }
@@ -319,8 +409,14 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
+      busy += clock64() - t_store;
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
+    }
+    if (p.trace && warp == 2 && lane == 0) {
+      p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
+      p.trace[blockIdx.x * kMoeTraceFields + 5] = static_cast<unsigned long long>(busy);
+      p.trace[blockIdx.x * kMoeTraceFields + 7] = static_cast<unsigned long long>(w_gap);
     }
   }
 
@@ -333,6 +429,15 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+  // Every CTA has drawn its last tile by now.  The last CTA to leave re-arms the scheduler for the next launch.
+  if (tid == 0) {
+    const int done = atomicAdd(&p.sched[1], 1);
+    if (done == static_cast<int>(gridDim.x) - 1) {
+      p.sched[0] = 0;
+      p.sched[1] = 0;
+      __threadfence();
+    }
   }
 }
 
@@ -389,6 +494,8 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
   p1.mode = tn.interleave_mode;
   p1.ik = tn.interleave_k;
   p1.status = ctx->d_status;
+  p1.sched = ctx->d_sched;
+  p1.trace = (tn.debug_flags & 1) ? ctx->d_trace : nullptr;
   p1.kernel_id = 1;
 
   FfnParams p2 = p1;
@@ -400,6 +507,8 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
   p2.b1_row_shift = 128;
   p2.out = static_cast<__nv_bfloat16*>(y_perm);
   p2.h_dbg = nullptr;
+  p2.sched = ctx->d_sched + 2;
+  p2.trace = p1.trace ? p1.trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
   p2.kernel_id = 2;
 
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)

@@ -26,7 +26,7 @@ moe_status check_tuning(const moe_tuning* t) {
   if (t->interleave_mode != 0 && t->interleave_mode != 1) return MOE_ERR_INVALID_ARG;
   if (!(t->interleave_k == 1 || t->interleave_k == 2 || t->interleave_k == 4)) return MOE_ERR_INVALID_ARG;
   if (t->schedule != 0) return MOE_ERR_UNSUPPORTED;
-  if (t->dep_lead_D != 0 || t->debug_flags != 0) return MOE_ERR_INVALID_ARG;
+  if (t->dep_lead_D != 0 || (t->debug_flags & ~1) != 0) return MOE_ERR_INVALID_ARG;
   return MOE_OK;
 }
 
@@ -136,6 +136,11 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   ok = ok && cudaMalloc(&ctx->d_chunk_base, hist_elems * 4) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_status, 2 * 4) == cudaSuccess;
   ok = ok && cudaMemset(ctx->d_status, 0, 2 * 4) == cudaSuccess;
+  const size_t trace_bytes = static_cast<size_t>(2) * ctx->num_sms * kMoeTraceFields * 8;
+  ok = ok && cudaMalloc(&ctx->d_trace, trace_bytes) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->d_trace, 0, trace_bytes) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_sched, 4 * 4) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->d_sched, 0, 4 * 4) == cudaSuccess;
   ok = ok && moe::prepare_expert_ffn(ctx) == cudaSuccess;
   for (int i = 0; ok && i <= kMoeKernels; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
   if (!ok) {
@@ -151,6 +156,8 @@ void moe_destroy(moe_ctx* ctx) {
   if (ctx->d_chunk_hist) cudaFree(ctx->d_chunk_hist);
   if (ctx->d_chunk_base) cudaFree(ctx->d_chunk_base);
   if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->d_sched) cudaFree(ctx->d_sched);
+  if (ctx->d_trace) cudaFree(ctx->d_trace);
   for (int i = 0; i <= kMoeKernels; ++i)
     if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
   delete ctx;
@@ -303,6 +310,20 @@ moe_status moe_last_device_status(moe_ctx* ctx, int32_t* code, int32_t* detail, 
 }
 
 int32_t moe_last_launch_count(const moe_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+
+moe_status moe_get_ffn_trace(moe_ctx* ctx, uint64_t* counters_host, int32_t capacity, int32_t* num_ctas, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  if (!counters_host || !num_ctas) return MOE_ERR_INVALID_ARG;
+  const int32_t need = 2 * ctx->num_sms * kMoeTraceFields;
+  *num_ctas = ctx->num_sms;
+  if (capacity < need) return MOE_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(counters_host, ctx->d_trace, static_cast<size_t>(need) * 8, cudaMemcpyDeviceToHost, cs) !=
+      cudaSuccess)
+    return MOE_ERR_CUDA;
+  return cudaStreamSynchronize(cs) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
 
 moe_status moe_set_kernel_timing(moe_ctx* ctx, int32_t enable) {
   if (!ctx) return MOE_ERR_INVALID_ARG;

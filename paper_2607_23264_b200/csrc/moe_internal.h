@@ -10,6 +10,11 @@
 constexpr int kRouteThreads = 256;
 // Kernels of one forward, in launch order: top-k+histogram, scan, scatter, dispatch, Linear-1, Linear-2, combine.
 constexpr int kMoeKernels = 7;
+// Wait counters one CTA of a grouped GEMM records when tracing is on (SM clocks unless noted):
+// 0 producer loop span, 1 producer waited for a free stage, 2 MMA waited for data, 3 MMA waited for a free
+// accumulator (the epilogue's back-pressure), 4 epilogue waited for an accumulator, 5 epilogue drain+store span,
+// 6 tiles processed (count), 7 epilogue held by the pacing gap.
+constexpr int kMoeTraceFields = 8;
 
 typedef CUresult (*moe_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -25,6 +30,8 @@ struct moe_ctx {
   int32_t* d_chunk_hist;  // [num_chunks, E] slots of each chunk per expert
   int32_t* d_chunk_base;  // [num_chunks, E] exclusive prefix of d_chunk_hist over chunks
   int32_t* d_status;      // [2] device status word: code, detail
+  int32_t* d_sched;       // [4] tile scheduler of the two grouped GEMMs: {next tile, CTAs done} each; zero when idle
+  unsigned long long* d_trace;   // [2][num_sms][kMoeTraceFields] wait counters of Linear-1 and Linear-2
   moe_encode_tiled_fn encode_tiled;
   int32_t last_launches;
   // Optional per-kernel timing: event i is recorded after kernel i (event 0 before the first kernel).

@@ -62,6 +62,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// Same, adding the clocks spent waiting (zero when the phase had already completed) to *waited.
+__device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                long long* waited) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  *waited += clock64() - t0;
+  return ok;
+}
+
 // ---------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

@@ -217,3 +217,28 @@ def test_host_side_errors_are_synchronous():
     assert ei.value.code == 2
     torch.cuda.synchronize()
     L.check_device_status()
+
+
+def test_ffn_trace_and_kernel_times():
+    """Measurement aids: per-kernel event times and the per-CTA wait counters of the grouped GEMMs."""
+    cfg = SMALL[1]
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
+    L.ctx.moe_set_kernel_timing(True)
+    out2 = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out2, ws,
+                            tuning=binding.make_tuning(1, 1, 2, debug_flags=1))
+    ms = L.ctx.moe_get_kernel_times()
+    L.ctx.moe_set_kernel_timing(False)
+    assert len(ms) == 7 and all(0 < v < 100 for v in ms)
+    tr = L.ctx.moe_get_ffn_trace()
+    assert tr.shape[0] == 2 and tr.shape[2] == 8
+    # every tile is processed exactly once: 128-row blocks per expert x N blocks
+    counts = L.ctx_counts = ws[L.ctx.workspace_layout()["counts"]:][: 4 * cfg.E].view(torch.int32).cpu().numpy()
+    mblocks = int(((counts + 127) // 128).sum())
+    assert tr[0, :, 6].sum() == mblocks * ((cfg.F + 127) // 128)
+    assert tr[1, :, 6].sum() == mblocks * ((cfg.H + 255) // 256)
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16)), "tracing must not change values"
+    L.check_device_status()
