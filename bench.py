@@ -187,17 +187,14 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2607_23264_b200 import binding
+    from paper_2607_23264_b200 import binding, replicas
 
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    replicas.init_process_group(world, "nccl", torch.device(dev))
 
     # every rank gets its own batch (the seeded batch, rows rotated by rank); expert weights are replicated
-    x_bits = gen.make_x(cfg)
-    if rank != 0:
-        x_bits = np.roll(x_bits, rank * 17, axis=0)
+    x_bits = replicas.rank_batch(gen.make_x(cfg), rank)
     logits = gen.make_logits(cfg, x_bits)
 
     to_dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
@@ -223,8 +220,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier(world)
         torch.cuda.synchronize()
 
     def timed(fn, steps, warmup):
@@ -237,12 +233,7 @@ def main():
             fn()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return replicas.max_over_ranks(e0.elapsed_time(e1), world, dev)
 
     if args.sweep:
         run_sweep(args, cfg, ctx, binding, (x, d_logits, w_gate, w_up, w_down, out, ws), timed, rank)
@@ -268,13 +259,9 @@ def main():
         step()
     e1.record(stream)
     barrier()
-    total_ms = e0.elapsed_time(e1)
+    total_ms = replicas.max_over_ranks(e0.elapsed_time(e1), world, dev)
     clocks = sampler.stop() if rank == 0 else None
     launches = ctx.moe_last_launch_count() * args.steps
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
 
     if args.profile:
         if rank == 0:
@@ -327,7 +314,7 @@ def main():
     peaks, peak_kind = load_peaks()
     ms_per_step = total_ms / args.steps
     tokens = cfg.T * world
-    value = tokens / (ms_per_step * 1e-3)
+    value = replicas.job_tokens_per_second(cfg.T, world, args.steps, total_ms)
     tflops = cfg.flops * world / (ms_per_step * 1e-3) / 1e12
     R = cfg.R
     l1_flops = 4 * R * cfg.H * cfg.F

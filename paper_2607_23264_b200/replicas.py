@@ -1,0 +1,49 @@
+"""Host-side logic of a multi-GPU run: independent replicas of the layer, one process per GPU.
+
+Nothing on the data path is sharded and no collective moves activations (EP=1): every rank runs the whole
+layer on its own batch of tokens with replicated expert weights.  torch.distributed is used only to line the
+ranks up (barrier) and to reduce the timing to the slowest rank.  The same functions run on CPU with the
+gloo backend, which is how they are tested.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def rank_batch(x_bits: np.ndarray, rank: int) -> np.ndarray:
+    """The batch of one rank: the seeded batch with its rows rotated by 17*rank, so ranks differ."""
+    return x_bits if rank == 0 else np.roll(x_bits, rank * 17, axis=0)
+
+
+def init_process_group(world: int, backend: str, device=None):
+    """Join the job's process group (rendezvous from the MASTER_* / RANK / WORLD_SIZE environment)."""
+    import torch.distributed as dist
+    if world <= 1:
+        return False
+    if backend == "nccl":
+        dist.init_process_group("nccl", device_id=device)
+    else:
+        dist.init_process_group(backend)
+    return True
+
+
+def barrier(world: int):
+    import torch.distributed as dist
+    if world > 1:
+        dist.barrier()
+
+
+def max_over_ranks(value: float, world: int, device="cpu") -> float:
+    """Slowest rank's figure (e.g. the device time of the timed region)."""
+    import torch
+    import torch.distributed as dist
+    if world <= 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_second(tokens_per_rank: int, world: int, steps: int, slowest_ms: float) -> float:
+    """Whole-job throughput: all ranks' tokens over the slowest rank's time."""
+    return tokens_per_rank * world * steps / (slowest_ms * 1e-3)

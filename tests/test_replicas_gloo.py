@@ -1,0 +1,53 @@
+"""The N>1 path of bench.py on CPU: two gloo ranks, independent replicas, max-over-ranks timing."""
+import os
+import socket
+
+import numpy as np
+import torch.multiprocessing as mp
+
+from paper_2607_23264_b200 import inputs as gen, replicas
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import torch.distributed as dist
+    assert replicas.init_process_group(world, "gloo")
+    cfg = gen.MoEConfig("t", T=64, H=64, F=64, E=4, k=2, seed=3, router="xWr")
+    x = replicas.rank_batch(gen.make_x(cfg), rank)
+    replicas.barrier(world)
+    my_ms = 10.0 + 5.0 * rank                      # rank 1 is the slow one
+    slowest = replicas.max_over_ranks(my_ms, world)
+    q.put((rank, slowest, int(x[:, 0].astype(np.int64).sum()), x[0, :4].tolist()))
+    replicas.barrier(world)
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_report_the_slowest_time_and_distinct_batches():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [g[1] for g in got] == [15.0, 15.0], "every rank sees the slowest rank's time"
+    assert got[0][2] == got[1][2], "same tokens, rotated"
+    assert got[0][3] != got[1][3], "ranks work on different batches"
+    assert replicas.job_tokens_per_second(64, world, steps=10, slowest_ms=15.0) == 64 * 2 * 10 / 0.015
+
+
+def test_single_rank_needs_no_process_group():
+    assert replicas.init_process_group(1, "gloo") is False
+    assert replicas.max_over_ranks(3.5, 1) == 3.5
+    x = np.arange(12, dtype=np.uint16).reshape(4, 3)
+    assert replicas.rank_batch(x, 0) is x
+    assert np.array_equal(replicas.rank_batch(x, 1), np.roll(x, 17, axis=0))
