@@ -168,6 +168,8 @@ def main():
     ap.add_argument("--mode", type=int, default=0)
     ap.add_argument("--ik", type=int, default=1)
     ap.add_argument("--sweep", action="store_true", help="store-pacing sweep (20 points) instead of the bench line")
+    ap.add_argument("--probe-mma", action="store_true",
+                    help="print SM clocks per tcgen05.mma for several tile shapes (tensor-pipe calibration) and exit")
     ap.add_argument("--trace", action="store_true",
                     help="add the grouped GEMMs' per-CTA wait counters (one extra traced step) to the JSON line")
     ap.add_argument("--profile", action="store_true",
@@ -191,6 +193,13 @@ def main():
 
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
+    if args.probe_mma:
+        pctx = binding.Context(128, 64, 64, 1, 1, device=local_rank)
+        rows = [{"M": M, "N": N, "clocks_per_mma": pctx.moe_probe_mma_cycles(M, N)}
+                for M in (128, 64) for N in (16, 32, 64, 128, 256)]
+        print(json.dumps({"probe": "tcgen05.mma kind::f16 MxNx16, one CTA, operands resident in shared memory",
+                          "rows": rows}), flush=True)
+        return
     replicas.init_process_group(world, "nccl", torch.device(dev))
 
     # every rank gets its own batch (the seeded batch, rows rotated by rank); expert weights are replicated

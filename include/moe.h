@@ -217,6 +217,15 @@ moe_status moe_get_ffn_trace(moe_ctx* ctx, uint64_t* counters_host, int32_t capa
                              void* stream);
 
 /*
+ * Calibration probe of the tensor pipe (in the spirit of the paper's independent calibration, Sec. 3.3: measure
+ * the platform parameter alone before using it in a kernel model).  One CTA issues `iters` tcgen05.mma of shape
+ * M x N x 16 (bf16 in, fp32 accumulate; M in {64,128}, N a multiple of 16 up to 256) back to back on operands
+ * resident in shared memory; *cycles_per_mma (HOST) receives the SM clocks per instruction.  Blocking.
+ */
+moe_status moe_probe_mma_cycles(moe_ctx* ctx, int32_t M, int32_t N, int32_t iters, double* cycles_per_mma,
+                                void* stream);
+
+/*
  * Per-kernel timing (measurement aid; the paper times its kernel with CUDA events, Sec. 5.1).  When
  * enabled, each call records a CUDA event on the stream before its first kernel and after every kernel.
  * moe_get_kernel_times waits for the last call's events and writes the seven device durations in

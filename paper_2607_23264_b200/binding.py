@@ -23,7 +23,7 @@ EXPORTS = (
     "moe_status_string", "moe_create", "moe_destroy", "moe_workspace_bytes", "moe_get_workspace_layout",
     "moe_plan_routing", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_fused_forward",
     "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count", "moe_set_kernel_timing",
-    "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace",
+    "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace", "moe_probe_mma_cycles",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -87,6 +87,7 @@ def load_library() -> C.CDLL:
     lib.moe_last_launch_count.restype = C.c_int32
     lib.moe_set_kernel_timing.argtypes = [vp, C.c_int32]
     lib.moe_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32]
+    lib.moe_probe_mma_cycles.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_double), vp]
     lib.moe_get_ffn_trace.argtypes = [vp, C.POINTER(C.c_uint64), C.c_int32, C.POINTER(C.c_int32), vp]
     for name in EXPORTS:
         if name not in ("moe_status_string", "moe_destroy", "moe_workspace_bytes", "moe_last_launch_count"):
@@ -243,6 +244,12 @@ class Context:
         _check(self._lib.moe_get_ffn_trace(self._handle, buf, cap, C.byref(n), _stream(stream)), "moe_get_ffn_trace")
         a = np.frombuffer(buf, dtype=np.uint64)[: 2 * n.value * len(TRACE_FIELDS)]
         return a.reshape(2, n.value, len(TRACE_FIELDS)).copy()
+
+    def moe_probe_mma_cycles(self, M: int, N: int, iters: int = 4096, stream=None) -> float:
+        out = C.c_double(0.0)
+        _check(self._lib.moe_probe_mma_cycles(self._handle, M, N, iters, C.byref(out), _stream(stream)),
+               "moe_probe_mma_cycles")
+        return out.value
 
     def moe_set_kernel_timing(self, enable: bool):
         _check(self._lib.moe_set_kernel_timing(self._handle, 1 if enable else 0), "moe_set_kernel_timing")

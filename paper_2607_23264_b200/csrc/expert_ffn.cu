@@ -441,6 +441,51 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
   }
 }
 
+// Calibration probe: one CTA issues `iters` tcgen05.mma of shape M x N x 16 back to back on resident
+// shared-memory operands and reports the SM clocks from the first issue to the completion of the last.
+__global__ void __launch_bounds__(128, 1) mma_cycle_probe(int M, int N, int iters, long long* out) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ uint64_t bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ volatile int abort_flag;
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+  const uint32_t base = raw + pad;
+  for (int i = threadIdx.x; i < kStageBytes / 4; i += blockDim.x)
+    reinterpret_cast<uint32_t*>(smem_raw + pad)[i] = 0x3c003c00u;   // bf16 values near 0.0078
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  ptx::fence_proxy_async_smem();
+  if (threadIdx.x < 32) {
+    ptx::tmem_alloc(ptx::smem_u32(&tmem_base_s), kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tb = tmem_base_s;
+  if (threadIdx.x == 0) {
+    const uint32_t idesc = ptx::idesc_bf16_f32(M, N);
+    const uint64_t a = ptx::smem_desc_sw128(base), b = ptx::smem_desc_sw128(base + kABytes);
+    const long long t0 = clock64();
+    for (int i = 0; i < iters; ++i) {
+      const uint64_t adv = static_cast<uint64_t>(2 * (i & 3));
+      ptx::tc_mma_bf16(tb, a + adv, b + adv, idesc, i > 0 ? 1u : 0u);
+    }
+    ptx::tc_commit(ptx::smem_u32(&bar));
+    ptx::mbar_wait(ptx::smem_u32(&bar), 0, &abort_flag);
+    out[0] = abort_flag ? -1 : clock64() - t0;
+  }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tb, kTmemCols);
+  }
+}
+
 CUresult encode_2d(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols) {
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * 2};
@@ -452,6 +497,26 @@ CUresult encode_2d(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t ro
 }
 
 }  // namespace
+
+extern "C" moe_status moe_probe_mma_cycles(moe_ctx* ctx, int32_t M, int32_t N, int32_t iters, double* cycles_per_mma,
+                                           void* stream) {
+  if (!ctx || !cycles_per_mma) return MOE_ERR_INVALID_ARG;
+  if (!(M == 64 || M == 128) || N < 16 || N > 256 || N % 16 != 0 || iters < 1 || iters > (1 << 20))
+    return MOE_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  long long* d_out = reinterpret_cast<long long*>(ctx->d_trace);   // reuse the first trace word as the result slot
+  const size_t smem = 1024 + kStageBytes;
+  if (cudaFuncSetAttribute(mma_cycle_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
+      cudaSuccess)
+    return MOE_ERR_CUDA;
+  mma_cycle_probe<<<1, 128, smem, cs>>>(M, N, iters, d_out);
+  long long clocks = 0;
+  if (cudaMemcpyAsync(&clocks, d_out, sizeof(clocks), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return MOE_ERR_CUDA;
+  if (clocks < 0) return MOE_ERR_TIMEOUT;
+  *cycles_per_mma = static_cast<double>(clocks) / iters;
+  return MOE_OK;
+}
 
 namespace moe {
 
