@@ -31,10 +31,10 @@ from paper_2607_23264_b200 import inputs as gen  # noqa: E402
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one expert_gemm_kernel<true> (Linear-1) launch on the
-# C2 workload: the ncu capture of the two-expert case P1 (503.5 MB read + 106.9 MB written, see
+# C2 workload: the ncu capture of the two-expert case P1 (504.1 MB read + 109.2 MB written, see
 # profiles/expert_gemm_P1_ncu_full.md) scaled by 4, since DRAM traffic is per expert and C2 has four times
-# P1's experts at the same rows per expert.
-LINEAR1_DRAM_TRAFFIC_BYTES = {"C2": 4 * (503_479_040 + 106_861_824)}
+# P1's experts at the same rows per expert.  C3: one-pass DRAM counters on the full layer (same file).
+LINEAR1_DRAM_TRAFFIC_BYTES = {"C2": 4 * (504_129_280 + 109_233_664), "C3": 11_263_676_672 + 136_142_592}
 
 
 def load_peaks():
