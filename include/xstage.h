@@ -1,0 +1,78 @@
+/*
+ * xstage.h -- host-side calculator for the paper's X-Stage (Burst-Gap) model, C ABI.
+ *
+ * The model M_X = (T_iss^0, R, Q) (Sec. 3.3): recovered issue floor, effective aggregate drain rate and
+ * effective outstanding capacity of a store path, calibrated by microbenchmarks, then applied to a kernel's
+ * burst sequence {V_n, T_iss,n^0, G_n}.  All functions are pure host arithmetic in double precision; they
+ * allocate nothing and touch no GPU.  Units are the caller's, used consistently: bytes, seconds, bytes/second
+ * in the examples (the paper's GB is 1e9 bytes, its MiB 2^20 bytes).  [z]_+ means max(z, 0).
+ * Pointers are HOST pointers owned by the caller.  Functions returning int return 0 on success and -1 on a bad
+ * argument (null pointer, non-positive rate or period, negative count); value-returning functions return NaN
+ * on a bad argument.
+ */
+#ifndef XSTAGE_B200_H_
+#define XSTAGE_B200_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+  double t_iss0;   /* recovered issue floor T_iss^0 */
+  double rate;     /* drain rate R */
+  double capacity; /* outstanding capacity Q */
+} xstage_params;
+
+/* Eq. 1, the Burst-Gap relation for a periodic pattern of volume V and gap G:
+ *   T_period = max(T_iss^0 + G, V/R),   T_iss = max(T_iss^0, V/R - G). */
+int xstage_burst_gap(const xstage_params* m, double volume, double gap, double* t_period, double* t_iss);
+
+/* Eq. 2, the smallest gap that returns issue to its floor: G* = [V/R - T_iss^0]_+ . */
+double xstage_recovery_gap(const xstage_params* m, double volume);
+
+/* Eq. 6 (first part), occupancy added by one burst issued from a recovered state: b_iso = [V - R T_iss^0]_+ .
+ * With the isolated-burst knee volume as V this is the calibration of Q (Sec. 3.5). */
+double xstage_isolated_occupancy(const xstage_params* m, double volume);
+
+/*
+ * Eqs. 3-6 over a burst sequence (the audit of Sec. 4.1).  For burst n = 0..count-1 with volume[n],
+ * floor[n] (its T_iss,n^0; pass NULL to use m->t_iss0 for every burst) and gap[n]:
+ *   P_n = floor_n + gap_n,  rho_n = V_n / (R P_n),  delta_b_n = V_n - R P_n,
+ *   q_0 = q_initial,  q_{n+1} = [q_n + delta_b_n]_+ ,
+ *   guard_n = (q_n + [V_n - R floor_n]_+ <= Q).
+ * Outputs (each may be NULL): rho[count], delta_b[count], backlog[count + 1] (q_0..q_count),
+ * guard_ok[count] (1 or 0).  Returns the index of the first burst whose guard fails, count if none does,
+ * or -1 on a bad argument (P_n must be positive).
+ */
+int64_t xstage_audit(const xstage_params* m, int64_t count, const double* volume, const double* floor,
+                     const double* gap, double q_initial, double* rho, double* delta_b, double* backlog,
+                     int32_t* guard_ok);
+
+/* Eq. 7, average gap of the interleaved MegaMoE schedule: G_int = T_L2^mma + (n1/n2) T_L1^mma
+ * (the Expert-Wave gap is T_L2^mma alone). */
+double xstage_interleaved_gap(double t_l2_mma, double t_l1_mma, double n1, double n2);
+
+/* Eq. 8, issue overhead left after interleaving: [dT_wave - (n1/n2) T_L1^mma]_+ . */
+double xstage_interleaved_issue_overhead(double overhead_wave, double t_l1_mma, double n1, double n2);
+
+/* Eq. 9, necessary average-rate condition for full recovery:
+ *   n2 V / (n2 (T_iss^0 + T_L2^mma) + n1 T_L1^mma) <= R.   Returns 1, 0, or -1 on a bad argument. */
+int xstage_average_rate_feasible(const xstage_params* m, double volume, double t_l2_mma, double t_l1_mma,
+                                 double n1, double n2);
+
+/* App. A.2, anti-starvation lead knee: D_knee = ceil(b_n K_SM / (2 h_inter)).  -1 on a bad argument. */
+int64_t xstage_lead_knee(int64_t b_n, int64_t k_sm, int64_t h_inter);
+
+/* App. A.2, predicted MMA-side stall: [T_RS - T_cover^mma]_+ . */
+double xstage_mma_stall(double t_remote_store_span, double t_cover_mma);
+
+/* App. C.2, tile-aligned sequence length above which the Q-loop gap (at least sigma per K/V tile) covers the
+ * recovery gap: M_ub = b_n ceil(G* / sigma).  -1 on a bad argument. */
+int64_t xstage_fa_recovery_length(int64_t b_n, double recovery_gap, double sigma);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XSTAGE_B200_H_ */
