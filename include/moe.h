@@ -60,9 +60,17 @@ typedef struct {
   int32_t store_burst_tiles;       /* 1, 2, 4, 8 or 16 (values above the tiles in one output tile act as that count) */
   int32_t interleave_mode;         /* 0 or 1 */
   int32_t interleave_k;            /* 1, 2 or 4; used when interleave_mode == 1 */
-  int32_t schedule;                /* 0 = expert-wave order (Sec. 4.3): all Linear-1 tiles, then Linear-2 */
-  int32_t dep_lead_D;              /* reserved for the interleaved schedule (Algorithm 1); must be 0 */
-  int32_t debug_flags;             /* bit 0: record per-CTA wait counters (moe_get_ffn_trace); other bits 0 */
+  int32_t schedule;                /* 0 = Expert-Wave order (Sec. 4.3): all Linear-1 tiles, then all Linear-2 tiles;
+                                      1 = interleaved order (Algorithm 1): every CTA g of G walks strided cursors
+                                      k1, k2 += G over the row-major Linear-1 / Linear-2 tile lists (a row is one
+                                      128-row block) and emits the Linear-2 tile only while Linear-1 leads by
+                                      dep_lead_D rows; one launch, Linear-2 tiles wait for their row's h.
+                                      Values are bitwise identical for both schedules. */
+  int32_t dep_lead_D;              /* schedule 1: minimum row lead D >= 1 of Linear-1 over Linear-2; 0 = the
+                                      anti-starvation knee ceil(128 * SMs / (2 F)) (App. A.2).  Must be 0 for
+                                      schedule 0. */
+  int32_t debug_flags;             /* bit 0: record per-CTA wait counters (moe_get_ffn_trace); bit 1: run
+                                      schedule 0 as one launch with ready counters instead of two; other bits 0 */
 } moe_tuning;
 
 /* Byte offsets of the slices of the workspace used by moe_fused_forward (each 256-byte aligned). */
@@ -215,6 +223,17 @@ int32_t moe_last_launch_count(const moe_ctx* ctx);
  */
 moe_status moe_get_ffn_trace(moe_ctx* ctx, uint64_t* counters_host, int32_t capacity, int32_t* num_ctas,
                              void* stream);
+
+/*
+ * Tile order of the last one-launch expert FFN that ran with tuning->debug_flags bit 0 set (schedule 1, or
+ * schedule 0 with debug bit 1): the codes each CTA drew, in its own order, so that the emitted schedule can be
+ * checked against Algorithm 1.  A code is (phase << 30) | index, phase 0 = Linear-1, 1 = Linear-2; for
+ * schedule 1 the index is the row-major tile number k (row k / n_blocks, column k % n_blocks, with n_blocks =
+ * ceil(F/128) for Linear-1 and ceil(H/256) for Linear-2); -1 ends a CTA's list.  Synchronises `stream` and copies
+ * codes_host[*num_ctas][*codes_per_cta] (int32, HOST); capacity is in elements and must cover that.
+ */
+moe_status moe_get_ffn_order(moe_ctx* ctx, int32_t* codes_host, int32_t capacity, int32_t* num_ctas,
+                             int32_t* codes_per_cta, void* stream);
 
 /*
  * Calibration probe of the tensor pipe (in the spirit of the paper's independent calibration, Sec. 3.3: measure

@@ -24,6 +24,7 @@ EXPORTS = (
     "moe_plan_routing", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_fused_forward",
     "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count", "moe_set_kernel_timing",
     "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace", "moe_probe_mma_cycles",
+    "moe_get_ffn_order",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -88,6 +89,7 @@ def load_library() -> C.CDLL:
     lib.moe_set_kernel_timing.argtypes = [vp, C.c_int32]
     lib.moe_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32]
     lib.moe_probe_mma_cycles.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_double), vp]
+    lib.moe_get_ffn_order.argtypes = [vp, C.POINTER(C.c_int32), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_get_ffn_trace.argtypes = [vp, C.POINTER(C.c_uint64), C.c_int32, C.POINTER(C.c_int32), vp]
     for name in EXPORTS:
         if name not in ("moe_status_string", "moe_destroy", "moe_workspace_bytes", "moe_last_launch_count"):
@@ -244,6 +246,25 @@ class Context:
         _check(self._lib.moe_get_ffn_trace(self._handle, buf, cap, C.byref(n), _stream(stream)), "moe_get_ffn_trace")
         a = np.frombuffer(buf, dtype=np.uint64)[: 2 * n.value * len(TRACE_FIELDS)]
         return a.reshape(2, n.value, len(TRACE_FIELDS)).copy()
+
+    def moe_get_ffn_order(self, stream=None):
+        """Tile codes each CTA drew in the last traced one-launch run: list (per CTA) of lists of
+        (phase, index), the terminating -1 dropped."""
+        cap = 1024 * 512
+        buf = (C.c_int32 * cap)()
+        n, per = C.c_int32(0), C.c_int32(0)
+        _check(self._lib.moe_get_ffn_order(self._handle, buf, cap, C.byref(n), C.byref(per), _stream(stream)),
+               "moe_get_ffn_order")
+        out = []
+        for g in range(n.value):
+            seq = []
+            for i in range(per.value):
+                code = buf[g * per.value + i]
+                if code < 0:
+                    break
+                seq.append((code >> 30, code & ((1 << 30) - 1)))
+            out.append(seq)
+        return out
 
     def moe_probe_mma_cycles(self, M: int, N: int, iters: int = 4096, stream=None) -> float:
         out = C.c_double(0.0)

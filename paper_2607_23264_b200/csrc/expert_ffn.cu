@@ -1,24 +1,34 @@
 // Grouped expert GEMMs for sm_100a: Linear-1 (gate/up projections with the SiLU*mul epilogue) and
-// Linear-2 (down projection), both as one persistent, warp-specialised tcgen05 kernel template.
+// Linear-2 (down projection) in one persistent, warp-specialised tcgen05 kernel.
 //
 // Tile: 128 rows of the expert-contiguous buffer x 256 fp32 accumulator columns in tensor memory.
 //   Linear-1: columns 0..127 are gate outputs f0..f0+127, columns 128..255 the matching up outputs, so
 //             the epilogue holds both halves of silu(g)*u for 128 h columns.
 //   Linear-2: 256 output columns of y_perm.
 // K is consumed in blocks of 64 bf16 (one 128-byte swizzle row); each block is 4 tcgen05.mma of K=16.
-// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue
-// (warp w reads TMEM lanes 32*(w%4)..+31, i.e. tile rows).  A 4-stage shared-memory ring feeds the MMA;
-// two 256-column accumulators let the epilogue of tile i overlap the mainloop of tile i+1.
+// Roles (192 threads): warp 0 = TMA producer and tile scheduler, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4)..+31, i.e. tile rows).  A 4-stage
+// shared-memory ring feeds the MMA; two 256-column accumulators let the epilogue of tile i overlap the
+// mainloop of tile i+1.  The producer publishes the tiles it draws to the other roles through a small
+// ring of tile codes.
 // Expert row ranges are ragged: a tile may cover rows of the next expert (or past R, zero-filled by
 // TMA); those rows are computed and discarded, stores are masked to the expert's own rows.
-// Tile order inside an expert is N block, then M block (fastest), so the CTAs running at the same time
-// share one weight tile through L2 and an expert's weights stream from HBM once.  Experts are split into
-// "hot" ones (several 128-row blocks: their tiles are tensor-bound) and "cold" ones (few rows: their
-// tiles only stream weights and are HBM-bound); the global order merges the hot and the cold tile lists
-// at a fixed ratio so that both finish together, and CTAs draw tiles from it dynamically (one atomic
-// counter).  At any time some SMs then keep the tensor pipes busy while others keep HBM busy, instead of
-// the two kinds of work running one after the other.
+//
+// Tile orders (moe_tuning.schedule):
+//   0  Expert-Wave: all Linear-1 tiles, then all Linear-2 tiles.  Inside a GEMM the order within an expert is
+//      N block, then M block (fastest), so the CTAs running at the same time share one weight tile through L2
+//      and an expert's weights stream from HBM once.  Experts are split into "hot" ones (several 128-row
+//      blocks: tensor-bound tiles) and "cold" ones (one block: their tiles only stream weights, HBM-bound);
+//      the order merges the hot and the cold tile lists at a fixed ratio so that both finish together, and
+//      CTAs draw tiles dynamically from one atomic counter.  Run as two launches (the kernel boundary is the
+//      Linear-1 -> Linear-2 dependency) or as one launch with per-block ready counters.
+//   1  Interleaved (Algorithm 1 of the paper): each CTA g of G walks two strided cursors k1, k2 over the
+//      row-major Linear-1 and Linear-2 tile lists (row = one 128-row block) and emits the Linear-2 tile only
+//      while Linear-1 leads by D rows, else the next Linear-1 tile.  One launch; a Linear-2 tile waits (bounded)
+//      until all Linear-1 tiles of its row have published their h rows.
 #include <cuda_bf16.h>
+
+#include <climits>
 
 #include "moe_internal.h"
 #include "ptx_sm100.cuh"
@@ -37,8 +47,9 @@ constexpr int kThreads = 192;
 constexpr int kMaxExperts = 1024;
 constexpr int kTmemCols = 512;
 constexpr int kChunkCols = 32;     // accumulator columns per tcgen05.ld = columns of one store tile
-constexpr int kRing = 4;           // tile ids the producer may publish ahead of the consumers
+constexpr int kRing = 4;           // tile codes the producer may publish ahead of the consumers
 constexpr int kHotBlocks = 2;      // experts with at least this many 128-row blocks count as tensor-bound
+constexpr int kPhaseShift = 30;    // tile code = phase << 30 | index in the phase's tile list; -1 = no more tiles
 
 struct SharedTail {
   uint64_t full[kStages];
@@ -47,7 +58,7 @@ struct SharedTail {
   uint64_t tmem_empty[2];
   uint64_t ring_full[kRing];
   uint64_t ring_empty[kRing];
-  int32_t ring_tile[kRing];         // tile ids drawn by the producer; -1 = no more tiles
+  int32_t ring_tile[kRing];
   uint32_t tmem_base;
   volatile int abort_flag;
   volatile uint32_t mma_progress;   // K-blocks issued so far by the MMA warp (pacing clock)
@@ -58,58 +69,93 @@ struct SharedTail {
 
 constexpr size_t kSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStages) * kStageBytes + sizeof(SharedTail);
 
+struct PhaseDesc {          // one of the two GEMMs
+  int N;                    // output columns per row (F for Linear-1, H for Linear-2) = weight rows per expert
+  int K;                    // reduction length (H for Linear-1, F for Linear-2)
+  int n_blocks;             // tiles along N
+  int k_blocks;             // 64-deep K blocks
+  int out_cols_per_tile;    // 128 (Linear-1) or 256 (Linear-2)
+  int b1_row_shift;         // row offset of the second weight box: 0 (up matrix) or 128 (same matrix)
+  __nv_bfloat16* out;       // [R, N]
+};
+
 struct FfnParams {
   const int32_t* offsets;   // [E+1]
   int E;
-  int N;                    // output columns of this GEMM per row (F for Linear-1, H for Linear-2)
-  int K;                    // reduction length (H for Linear-1, F for Linear-2)
-  int n_blocks;             // tiles along N
-  int out_cols_per_tile;    // 128 (Linear-1) or 256 (Linear-2)
-  int w_rows_per_expert;    // rows of the weight matrix per expert (= N)
-  int b1_row_shift;         // row offset of the second weight box: 0 (up matrix) or 128 (same matrix)
-  __nv_bfloat16* out;       // [R, N]
-  float* h_dbg;             // Linear-1 only: fp32 copy of h before rounding, or nullptr
+  PhaseDesc ph[2];
+  float* h_dbg;             // fp32 copy of h before rounding, or nullptr
   int burst, mode, ik;      // store pacing
   int32_t* status;          // [2]
   int32_t* sched;           // [2] next tile to draw, CTAs finished; both zero between launches
+  int32_t* ready;           // [128-row blocks] Linear-1 warps that published their part of the block's h rows
   unsigned long long* trace;   // nullptr, or [gridDim.x][kMoeTraceFields] wait counters in SM clocks
+  int32_t* order_log;       // nullptr, or [gridDim.x][kMoeOrderLogCap] tile codes in the order this CTA drew them
+  int phase_lo, phase_hi;   // GEMMs in this launch: [0,1) Linear-1, [1,2) Linear-2, [0,2) both
+  int schedule;             // 0 merged order drawn dynamically, 1 Algorithm 1
+  int lead_D;               // Algorithm 1: minimum row lead of Linear-1 over Linear-2 (>= 1)
   int kernel_id;
 };
 
 struct Tile {
+  int phase;     // 0 Linear-1, 1 Linear-2
   int row0;      // first row in the expert-contiguous buffer
   int row_end;   // end of the expert's rows (exclusive)
   int n0;        // first output column
   int w_row0;    // first row of the weight box in the [E*N, K] weight matrix
+  int block;     // global index of the 128-row block (ready counter)
 };
 
-// Position `pos` of the merged order -> tile.  Among the first `pos` positions floor(pos*cold/total) are
-// cold tiles; position pos is itself cold when that count steps up at pos+1.
-__device__ __forceinline__ Tile decode_tile(int pos, const SharedTail* st, const FfnParams& p) {
-  const long long hot_tiles = static_cast<long long>(st->hot_prefix[p.E]) * p.n_blocks;
-  const long long cold_tiles = static_cast<long long>(st->cold_prefix[p.E]) * p.n_blocks;
-  const long long total = hot_tiles + cold_tiles;
-  const long long cold_before = (static_cast<long long>(pos) * cold_tiles) / total;
-  const bool is_cold = ((static_cast<long long>(pos) + 1) * cold_tiles) / total > cold_before;
-  const int tile = static_cast<int>(is_cold ? cold_before : pos - cold_before);
-  const int32_t* prefix = is_cold ? st->cold_prefix : st->hot_prefix;
-  const int q = tile / p.n_blocks;   // lies in [prefix[e], prefix[e+1]) of the owning expert
-  int lo = 0, hi = p.E;              // invariant: prefix[lo] <= q < prefix[hi]
+// Largest e with prefix(e) <= q, prefix non-decreasing with prefix(0) = 0 and q < prefix(E).
+template <class F>
+__device__ __forceinline__ int find_expert(F prefix, int q, int E) {
+  int lo = 0, hi = E;   // invariant: prefix(lo) <= q < prefix(hi)
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
-    if (prefix[mid] <= q) lo = mid; else hi = mid;
+    if (prefix(mid) <= q) lo = mid; else hi = mid;
   }
-  const int e = lo;
-  const int mb = prefix[e + 1] - prefix[e];
-  const int local = tile - p.n_blocks * prefix[e];
-  const int n_blk = local / mb;
-  const int m_blk = local - n_blk * mb;
+  return lo;
+}
+
+__device__ __forceinline__ Tile make_tile(int phase, int e, int m_blk, int n_blk, const SharedTail* st,
+                                          const FfnParams& p) {
+  const PhaseDesc& d = p.ph[phase];
   Tile t;
+  t.phase = phase;
   t.row0 = p.offsets[e] + m_blk * BM;
   t.row_end = p.offsets[e + 1];
-  t.n0 = n_blk * p.out_cols_per_tile;
-  t.w_row0 = e * p.w_rows_per_expert + t.n0;
+  t.n0 = n_blk * d.out_cols_per_tile;
+  t.w_row0 = e * d.N + t.n0;
+  t.block = st->hot_prefix[e] + st->cold_prefix[e] + m_blk;
   return t;
+}
+
+// Tile code -> tile.
+//  schedule 0: index = position in the merged hot/cold order of the phase.  Among the first `pos` positions
+//              floor(pos*cold/total) are cold tiles; position pos is itself cold when that count steps up at
+//              pos+1.  Inside a class the order is expert, N block, M block (fastest).
+//  schedule 1: index = row-major tile number k: row k / n_blocks (a global 128-row block), column k % n_blocks.
+__device__ __forceinline__ Tile decode_tile(int code, const SharedTail* st, const FfnParams& p) {
+  const int phase = code >> kPhaseShift;
+  const int idx = code & ((1 << kPhaseShift) - 1);
+  const int nb = p.ph[phase].n_blocks;
+  if (p.schedule == 1) {
+    const int row = idx / nb;
+    const int n_blk = idx - row * nb;
+    const int e = find_expert([&](int i) { return st->hot_prefix[i] + st->cold_prefix[i]; }, row, p.E);
+    return make_tile(phase, e, row - (st->hot_prefix[e] + st->cold_prefix[e]), n_blk, st, p);
+  }
+  const long long hot_tiles = static_cast<long long>(st->hot_prefix[p.E]) * nb;
+  const long long cold_tiles = static_cast<long long>(st->cold_prefix[p.E]) * nb;
+  const long long total = hot_tiles + cold_tiles;
+  const long long cold_before = (static_cast<long long>(idx) * cold_tiles) / total;
+  const bool is_cold = ((static_cast<long long>(idx) + 1) * cold_tiles) / total > cold_before;
+  const int tile = static_cast<int>(is_cold ? cold_before : idx - cold_before);
+  const int32_t* prefix = is_cold ? st->cold_prefix : st->hot_prefix;
+  const int e = find_expert([&](int i) { return prefix[i]; }, tile / nb, p.E);
+  const int mb = prefix[e + 1] - prefix[e];
+  const int local = tile - nb * prefix[e];
+  const int n_blk = local / mb;
+  return make_tile(phase, e, local - n_blk * mb, n_blk, st, p);
 }
 
 __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
@@ -117,6 +163,11 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+__device__ __forceinline__ void report_timeout(const FfnParams& p, int role) {
+  atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
+  atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + role);
 }
 
 // Hold the epilogue until the MMA warp has issued `ik` more K-blocks than at `start`, or cannot advance.
@@ -127,10 +178,91 @@ __device__ __forceinline__ void pace_gap(SharedTail* st, uint32_t start, int ik)
   }
 }
 
+// Bounded wait until `*counter` (written by other CTAs with release ordering) reaches `target`.
+__device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, volatile int* abort_flag) {
+  const long long t0 = clock64();
+  for (uint32_t it = 0;; ++it) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) return true;
+    if ((it & 0xFu) == 0xFu) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > ptx::kWaitClockBudget) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+    __nanosleep(100);
+  }
+}
+
+// Drain one finished accumulator: rows of this thread's TMEM lane, kGated ? silu(g)*u of 128 columns
+// : 256 plain columns, written as bf16 with 16-byte stores masked to the expert's rows and to N.
 template <bool kGated>
+__device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams& p, SharedTail* st, uint32_t t_addr,
+                                                  int row, long long* w_gap) {
+  const PhaseDesc& d = p.ph[kGated ? 0 : 1];
+  const bool row_ok = row < t.row_end;
+  __nv_bfloat16* out_row = d.out + static_cast<size_t>(row) * d.N + t.n0;
+  constexpr int kChunks = kGated ? (128 / kChunkCols) : (BN_ACC / kChunkCols);
+  int in_burst = 0;
+  uint32_t gap_start = st->mma_progress;
+#pragma unroll 1
+  for (int c = 0; c < kChunks; ++c) {
+    uint32_t v[32];
+    float o[32];
+    if constexpr (kGated) {
+      uint32_t u[32];
+      ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
+      ptx::tmem_ld_32x32(t_addr + 128 + c * kChunkCols, u);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[i] = silu_mul(__uint_as_float(v[i]), __uint_as_float(u[i]));
+    } else {
+      ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
+    }
+    const int col0 = t.n0 + c * kChunkCols;
+    if (row_ok) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (col0 + q * 8 < d.N) {     // N is a multiple of 8: a 16-byte vector is inside or outside
+          uint4 w;
+          w.x = pack_bf16(o[q * 8 + 0], o[q * 8 + 1]);
+          w.y = pack_bf16(o[q * 8 + 2], o[q * 8 + 3]);
+          w.z = pack_bf16(o[q * 8 + 4], o[q * 8 + 5]);
+          w.w = pack_bf16(o[q * 8 + 6], o[q * 8 + 7]);
+          *reinterpret_cast<uint4*>(out_row + c * kChunkCols + q * 8) = w;
+        }
+      }
+      if constexpr (kGated) {
+        if (p.h_dbg != nullptr) {
+          float* dbg = p.h_dbg + static_cast<size_t>(row) * d.N + col0;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            if (col0 + q * 4 < d.N) {
+              *reinterpret_cast<float4*>(dbg + q * 4) = make_float4(o[q * 4], o[q * 4 + 1], o[q * 4 + 2], o[q * 4 + 3]);
+            }
+          }
+        }
+      }
+    }
+    if (p.mode == 1 && ++in_burst >= p.burst && c + 1 < kChunks) {
+      const long long t_gap = clock64();
+      pace_gap(st, gap_start, p.ik);
+      *w_gap += clock64() - t_gap;
+      gap_start = st->mma_progress;
+      in_burst = 0;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
-                   const __grid_constant__ CUtensorMap tm_b1, const FfnParams p) {
+expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wg,
+                  const __grid_constant__ CUtensorMap tm_wu, const __grid_constant__ CUtensorMap tm_h,
+                  const __grid_constant__ CUtensorMap tm_wd, const FfnParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -184,9 +316,11 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       run_cold += __shfl_sync(0xFFFFFFFFu, cold, 31);
     }
     if (lane == 0) {
-      ptx::prefetch_tensormap(&tm_a);
-      ptx::prefetch_tensormap(&tm_b0);
-      ptx::prefetch_tensormap(&tm_b1);
+      ptx::prefetch_tensormap(&tm_x);
+      ptx::prefetch_tensormap(&tm_wg);
+      ptx::prefetch_tensormap(&tm_wu);
+      ptx::prefetch_tensormap(&tm_h);
+      ptx::prefetch_tensormap(&tm_wd);
     }
   }
   if (warp == 1) {
@@ -198,12 +332,14 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
   ptx::tc_fence_after_sync();
 
   const uint32_t tmem_base = st->tmem_base;
-  const int total_tiles = (st->hot_prefix[p.E] + st->cold_prefix[p.E]) * p.n_blocks;
-  const int k_blocks = (p.K + BK - 1) / BK;
+  const int total_blocks = st->hot_prefix[p.E] + st->cold_prefix[p.E];
+  const int tiles1 = p.phase_lo == 0 ? total_blocks * p.ph[0].n_blocks : 0;   // Linear-1 tiles of this launch
+  const int tiles2 = p.phase_hi == 2 ? total_blocks * p.ph[1].n_blocks : 0;   // Linear-2 tiles of this launch
+  const bool chained = tiles1 > 0 && tiles2 > 0;   // Linear-2 tiles depend on Linear-1 tiles of the same launch
   volatile int* abort_flag = &st->abort_flag;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ tile scheduler + TMA producer
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
@@ -211,34 +347,63 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       uint32_t ring_phase = 0;
       bool ok = true;
       long long w_empty = 0;
+      int k1 = blockIdx.x, k2 = blockIdx.x;   // Algorithm 1 cursors of scheduler instance g = blockIdx.x
+      int n_drawn = 0;
       const long long t_begin = clock64();
       while (ok) {
-        // draw the next tile and publish it to the MMA and epilogue roles
         if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_empty[slot]), ring_phase ^ 1u, abort_flag)) {
-          atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
-          atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 5);
+          report_timeout(p, 5);
           break;
         }
-        int pos = atomicAdd(&p.sched[0], 1);
-        if (pos >= total_tiles) pos = -1;
-        st->ring_tile[slot] = pos;
+        // ---- next tile of this CTA
+        int code = -1;
+        if (p.schedule == 1) {
+          if (k1 < tiles1 || k2 < tiles2) {
+            const int p1 = k1 < tiles1 ? k1 / p.ph[0].n_blocks : INT_MAX;   // row of the next Linear-1 tile
+            const int p2 = k2 / p.ph[1].n_blocks;
+            if (k2 < tiles2 && p2 <= p1 - p.lead_D) {
+              code = (1 << kPhaseShift) | k2;
+              k2 += gridDim.x;
+            } else {
+              code = k1;
+              k1 += gridDim.x;
+            }
+          }
+        } else {
+          const int pos = atomicAdd(&p.sched[0], 1);
+          if (pos < tiles1) code = pos;
+          else if (pos < tiles1 + tiles2) code = (1 << kPhaseShift) | (pos - tiles1);
+        }
+        if (p.order_log && n_drawn < kMoeOrderLogCap) p.order_log[blockIdx.x * kMoeOrderLogCap + n_drawn++] = code;
+        st->ring_tile[slot] = code;
         ptx::mbar_arrive(ptx::smem_u32(&st->ring_full[slot]));
         if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
-        if (pos < 0) break;
-        const Tile t = decode_tile(pos, st, p);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        if (code < 0) break;
+        const Tile t = decode_tile(code, st, p);
+        const PhaseDesc& d = p.ph[t.phase];
+        const CUtensorMap* ma = t.phase == 0 ? &tm_x : &tm_h;
+        const CUtensorMap* mb0 = t.phase == 0 ? &tm_wg : &tm_wd;
+        const CUtensorMap* mb1 = t.phase == 0 ? &tm_wu : &tm_wd;
+        if (chained && t.phase == 1) {
+          // every Linear-1 tile of this row (n_blocks tiles x 4 epilogue warps) must have published its h rows
+          if (!wait_counter(&p.ready[t.block], 4 * p.ph[0].n_blocks, abort_flag)) {
+            report_timeout(p, 8);
+            break;
+          }
+          ptx::fence_proxy_async_all();   // h was written through the generic proxy, TMA reads through the async one
+        }
+        for (int kb = 0; kb < d.k_blocks; ++kb) {
           if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, &w_empty)) {
-            atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
-            atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 1);
+            report_timeout(p, 1);
             ok = false;
             break;
           }
           const uint32_t full = ptx::smem_u32(&st->full[stage]);
           const uint32_t sa = stage_u32 + stage * kStageBytes;
           ptx::mbar_expect_tx(full, kStageBytes);
-          ptx::tma_load_2d(sa, &tm_a, full, kb * BK, t.row0);
-          ptx::tma_load_2d(sa + kABytes, &tm_b0, full, kb * BK, t.w_row0);
-          ptx::tma_load_2d(sa + kABytes + kBHalfBytes, &tm_b1, full, kb * BK, t.w_row0 + p.b1_row_shift);
+          ptx::tma_load_2d(sa, ma, full, kb * BK, t.row0);
+          ptx::tma_load_2d(sa + kABytes, mb0, full, kb * BK, t.w_row0);
+          ptx::tma_load_2d(sa + kABytes + kBHalfBytes, mb1, full, kb * BK, t.w_row0 + d.b1_row_shift);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -264,17 +429,16 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       while (ok) {
         st->mma_idle = 1;
         if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
-          atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
-          atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 6);
+          report_timeout(p, 6);
           break;
         }
-        const int pos = st->ring_tile[slot];
+        const int code = st->ring_tile[slot];
         ptx::mbar_arrive(ptx::smem_u32(&st->ring_empty[slot]));
         if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
-        if (pos < 0) break;
+        if (code < 0) break;
+        const int k_blocks = p.ph[code >> kPhaseShift].k_blocks;
         if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, &w_tmem)) {
-          atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
-          atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 2);
+          report_timeout(p, 2);
           break;
         }
         st->mma_idle = 0;
@@ -282,8 +446,7 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN_ACC);
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), phase, abort_flag, &w_full)) {
-            atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
-            atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 3);
+            report_timeout(p, 3);
             ok = false;
             break;
           }
@@ -321,94 +484,41 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
     const int r_in_tile = quarter * 32 + lane;
     int acc = 0;
     uint32_t acc_phase = 0;
-    const int burst = p.burst;
     int slot = 0;
     uint32_t ring_phase = 0;
     long long w_acc = 0, busy = 0, w_gap = 0;
     while (true) {
       if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
-        if (lane == 0) {
-          atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
-          atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 7);
-        }
+        if (lane == 0) report_timeout(p, 7);
         break;
       }
-      const int pos = st->ring_tile[slot];
+      const int code = st->ring_tile[slot];
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->ring_empty[slot]));
       if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
-      if (pos < 0) break;
-      const Tile t = decode_tile(pos, st, p);
+      if (code < 0) break;
+      const Tile t = decode_tile(code, st, p);
       if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, &w_acc)) {
-        if (lane == 0) {
-          atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
-          atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + 4);
-        }
+        if (lane == 0) report_timeout(p, 4);
         break;
       }
       ptx::tc_fence_after_sync();
       const long long t_store = clock64();
-      const int row = t.row0 + r_in_tile;
-      const bool row_ok = row < t.row_end;
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               static_cast<uint32_t>(acc * BN_ACC);
-      __nv_bfloat16* out_row = p.out + static_cast<size_t>(row) * p.N + t.n0;
-      constexpr int kChunks = kGated ? (128 / kChunkCols) : (BN_ACC / kChunkCols);
-      int in_burst = 0;
-      uint32_t gap_start = st->mma_progress;
-#pragma unroll 1
-      for (int c = 0; c < kChunks; ++c) {
-        uint32_t v[32];
-        float o[32];
-        if constexpr (kGated) {
-          uint32_t u[32];
-          ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
-          ptx::tmem_ld_32x32(t_addr + 128 + c * kChunkCols, u);
-          ptx::tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = silu_mul(__uint_as_float(v[i]), __uint_as_float(u[i]));
-        } else {
-          ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
-          ptx::tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
-        }
-        const int col0 = t.n0 + c * kChunkCols;
-        if (row_ok) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            if (col0 + q * 8 < p.N) {     // N is a multiple of 8: a 16-byte vector is inside or outside
-              uint4 w;
-              w.x = pack_bf16(o[q * 8 + 0], o[q * 8 + 1]);
-              w.y = pack_bf16(o[q * 8 + 2], o[q * 8 + 3]);
-              w.z = pack_bf16(o[q * 8 + 4], o[q * 8 + 5]);
-              w.w = pack_bf16(o[q * 8 + 6], o[q * 8 + 7]);
-              *reinterpret_cast<uint4*>(out_row + c * kChunkCols + q * 8) = w;
-            }
-          }
-          if constexpr (kGated) {
-            if (p.h_dbg != nullptr) {
-              float* dbg = p.h_dbg + static_cast<size_t>(row) * p.N + col0;
-#pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                if (col0 + q * 4 < p.N) {
-                  *reinterpret_cast<float4*>(dbg + q * 4) = make_float4(o[q * 4], o[q * 4 + 1], o[q * 4 + 2], o[q * 4 + 3]);
-                }
-              }
-            }
-          }
-        }
-        if (p.mode == 1 && ++in_burst >= burst && c + 1 < kChunks) {
-          const long long t_gap = clock64();
-          pace_gap(st, gap_start, p.ik);
-          w_gap += clock64() - t_gap;
-          gap_start = st->mma_progress;
-          in_burst = 0;
-        }
-      }
+      if (t.phase == 0) drain_accumulator<true>(t, p, st, t_addr, t.row0 + r_in_tile, &w_gap);
+      else drain_accumulator<false>(t, p, st, t_addr, t.row0 + r_in_tile, &w_gap);
       ptx::tc_fence_before_sync();
+      if (chained && t.phase == 0) {
+        // publish this warp's 32 rows x 128 columns of h to the Linear-2 tiles of the block
+        __threadfence();
+        ptx::fence_proxy_async_all();
+      }
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
+      if (lane == 0) {
+        ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
+        if (chained && t.phase == 0) atomicAdd(&p.ready[t.block], 1);
+      }
       busy += clock64() - t_store;
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
@@ -430,14 +540,19 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
-  // Every CTA has drawn its last tile by now.  The last CTA to leave re-arms the scheduler for the next launch.
-  if (tid == 0) {
-    const int done = atomicAdd(&p.sched[1], 1);
-    if (done == static_cast<int>(gridDim.x) - 1) {
+  // Every CTA has drawn its last tile by now.  The last CTA to leave re-arms the scheduler and, after a
+  // chained launch, the ready counters for the next launch.
+  __shared__ int s_last;
+  if (tid == 0) s_last = atomicAdd(&p.sched[1], 1) == static_cast<int>(gridDim.x) - 1;
+  __syncthreads();
+  if (s_last) {
+    if (chained)
+      for (int i = tid; i < total_blocks; i += kThreads) p.ready[i] = 0;
+    if (tid == 0) {
       p.sched[0] = 0;
       p.sched[1] = 0;
-      __threadfence();
     }
+    __threadfence();
   }
 }
 
@@ -521,10 +636,7 @@ extern "C" moe_status moe_probe_mma_cycles(moe_ctx* ctx, int32_t M, int32_t N, i
 namespace moe {
 
 cudaError_t prepare_expert_ffn(moe_ctx*) {
-  cudaError_t e = cudaFuncSetAttribute(expert_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kSmemBytes));
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(expert_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  return cudaFuncSetAttribute(expert_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(kSmemBytes));
 }
 
@@ -544,44 +656,52 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
   if (encode_2d(ctx, &tm_h, h_ws, R, s.F) != CUDA_SUCCESS) return MOE_ERR_CUDA;
   if (encode_2d(ctx, &tm_wd, w_down, static_cast<uint64_t>(s.E) * s.H, s.F) != CUDA_SUCCESS) return MOE_ERR_CUDA;
 
-  FfnParams p1{};
-  p1.offsets = offsets;
-  p1.E = s.E;
-  p1.N = s.F;
-  p1.K = s.H;
-  p1.n_blocks = (s.F + 127) / 128;
-  p1.out_cols_per_tile = 128;
-  p1.w_rows_per_expert = s.F;
-  p1.b1_row_shift = 0;
-  p1.out = static_cast<__nv_bfloat16*>(h_ws);
-  p1.h_dbg = h_fp32_debug;
-  p1.burst = tn.store_burst_tiles;
-  p1.mode = tn.interleave_mode;
-  p1.ik = tn.interleave_k;
-  p1.status = ctx->d_status;
-  p1.sched = ctx->d_sched;
-  p1.trace = (tn.debug_flags & 1) ? ctx->d_trace : nullptr;
-  p1.kernel_id = 1;
-
-  FfnParams p2 = p1;
-  p2.N = s.H;
-  p2.K = s.F;
-  p2.n_blocks = (s.H + 255) / 256;
-  p2.out_cols_per_tile = 256;
-  p2.w_rows_per_expert = s.H;
-  p2.b1_row_shift = 128;
-  p2.out = static_cast<__nv_bfloat16*>(y_perm);
-  p2.h_dbg = nullptr;
-  p2.sched = ctx->d_sched + 2;
-  p2.trace = p1.trace ? p1.trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
-  p2.kernel_id = 2;
-
+  FfnParams p{};
+  p.offsets = offsets;
+  p.E = s.E;
+  p.ph[0] = PhaseDesc{s.F, s.H, (s.F + 127) / 128, (s.H + BK - 1) / BK, 128, 0, static_cast<__nv_bfloat16*>(h_ws)};
+  p.ph[1] = PhaseDesc{s.H, s.F, (s.H + 255) / 256, (s.F + BK - 1) / BK, 256, 128, static_cast<__nv_bfloat16*>(y_perm)};
+  p.h_dbg = h_fp32_debug;
+  p.burst = tn.store_burst_tiles;
+  p.mode = tn.interleave_mode;
+  p.ik = tn.interleave_k;
+  p.status = ctx->d_status;
+  p.ready = ctx->d_ready;
+  p.schedule = tn.schedule;
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
-  expert_gemm_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, p1);
-  moe_mark(ctx, 5, stream);
-  expert_gemm_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(tm_h, tm_wd, tm_wd, p2);
-  moe_mark(ctx, 6, stream);
-  ctx->last_launches += 2;
+  // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
+  p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);
+  const bool trace = (tn.debug_flags & 1) != 0;
+  const bool one_launch = tn.schedule == 1 || (tn.debug_flags & 2) != 0;
+
+  if (one_launch) {
+    p.phase_lo = 0;
+    p.phase_hi = 2;
+    p.sched = ctx->d_sched;
+    p.trace = trace ? ctx->d_trace : nullptr;
+    p.order_log = trace ? ctx->d_order : nullptr;
+    p.kernel_id = 3;
+    expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+    moe_mark(ctx, 5, stream);
+    moe_mark(ctx, 6, stream);
+    ctx->last_launches += 1;
+  } else {
+    p.phase_lo = 0;
+    p.phase_hi = 1;
+    p.sched = ctx->d_sched;
+    p.trace = trace ? ctx->d_trace : nullptr;
+    p.kernel_id = 1;
+    expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+    moe_mark(ctx, 5, stream);
+    p.phase_lo = 1;
+    p.phase_hi = 2;
+    p.sched = ctx->d_sched + 2;
+    p.trace = trace ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
+    p.kernel_id = 2;
+    expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+    moe_mark(ctx, 6, stream);
+    ctx->last_launches += 2;
+  }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

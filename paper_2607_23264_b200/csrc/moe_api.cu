@@ -25,8 +25,9 @@ moe_status check_tuning(const moe_tuning* t) {
   if (!(b == 1 || b == 2 || b == 4 || b == 8 || b == 16)) return MOE_ERR_INVALID_ARG;
   if (t->interleave_mode != 0 && t->interleave_mode != 1) return MOE_ERR_INVALID_ARG;
   if (!(t->interleave_k == 1 || t->interleave_k == 2 || t->interleave_k == 4)) return MOE_ERR_INVALID_ARG;
-  if (t->schedule != 0) return MOE_ERR_UNSUPPORTED;
-  if (t->dep_lead_D != 0 || (t->debug_flags & ~1) != 0) return MOE_ERR_INVALID_ARG;
+  if (t->schedule != 0 && t->schedule != 1) return MOE_ERR_UNSUPPORTED;
+  if (t->dep_lead_D < 0 || (t->schedule == 0 && t->dep_lead_D != 0) || (t->debug_flags & ~3) != 0)
+    return MOE_ERR_INVALID_ARG;
   return MOE_OK;
 }
 
@@ -139,6 +140,12 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   const size_t trace_bytes = static_cast<size_t>(2) * ctx->num_sms * kMoeTraceFields * 8;
   ok = ok && cudaMalloc(&ctx->d_trace, trace_bytes) == cudaSuccess;
   ok = ok && cudaMemset(ctx->d_trace, 0, trace_bytes) == cudaSuccess;
+  const size_t order_bytes = static_cast<size_t>(ctx->num_sms) * kMoeOrderLogCap * 4;
+  ok = ok && cudaMalloc(&ctx->d_order, order_bytes) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->d_order, 0xFF, order_bytes) == cudaSuccess;
+  const size_t ready_bytes = (static_cast<size_t>(shape->T) * shape->k / 128 + shape->E + 1) * 4;
+  ok = ok && cudaMalloc(&ctx->d_ready, ready_bytes) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->d_ready, 0, ready_bytes) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_sched, 4 * 4) == cudaSuccess;
   ok = ok && cudaMemset(ctx->d_sched, 0, 4 * 4) == cudaSuccess;
   ok = ok && moe::prepare_expert_ffn(ctx) == cudaSuccess;
@@ -158,6 +165,8 @@ void moe_destroy(moe_ctx* ctx) {
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->d_sched) cudaFree(ctx->d_sched);
   if (ctx->d_trace) cudaFree(ctx->d_trace);
+  if (ctx->d_ready) cudaFree(ctx->d_ready);
+  if (ctx->d_order) cudaFree(ctx->d_order);
   for (int i = 0; i <= kMoeKernels; ++i)
     if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
   delete ctx;
@@ -321,6 +330,21 @@ moe_status moe_get_ffn_trace(moe_ctx* ctx, uint64_t* counters_host, int32_t capa
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   if (cudaMemcpyAsync(counters_host, ctx->d_trace, static_cast<size_t>(need) * 8, cudaMemcpyDeviceToHost, cs) !=
       cudaSuccess)
+    return MOE_ERR_CUDA;
+  return cudaStreamSynchronize(cs) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_get_ffn_order(moe_ctx* ctx, int32_t* codes_host, int32_t capacity, int32_t* num_ctas,
+                             int32_t* codes_per_cta, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  if (!codes_host || !num_ctas || !codes_per_cta) return MOE_ERR_INVALID_ARG;
+  const int32_t need = ctx->num_sms * kMoeOrderLogCap;
+  *num_ctas = ctx->num_sms;
+  *codes_per_cta = kMoeOrderLogCap;
+  if (capacity < need) return MOE_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(codes_host, ctx->d_order, static_cast<size_t>(need) * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
     return MOE_ERR_CUDA;
   return cudaStreamSynchronize(cs) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

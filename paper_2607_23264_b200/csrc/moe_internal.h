@@ -15,6 +15,8 @@ constexpr int kMoeKernels = 7;
 // accumulator (the epilogue's back-pressure), 4 epilogue waited for an accumulator, 5 epilogue drain+store span,
 // 6 tiles processed (count), 7 epilogue held by the pacing gap.
 constexpr int kMoeTraceFields = 8;
+// Tile codes (phase << 30 | index in the phase's tile list, -1 = end) a CTA logs when tracing a one-launch run.
+constexpr int kMoeOrderLogCap = 512;
 
 typedef CUresult (*moe_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -31,6 +33,8 @@ struct moe_ctx {
   int32_t* d_chunk_base;  // [num_chunks, E] exclusive prefix of d_chunk_hist over chunks
   int32_t* d_status;      // [2] device status word: code, detail
   int32_t* d_sched;       // [4] tile scheduler of the two grouped GEMMs: {next tile, CTAs done} each; zero when idle
+  int32_t* d_ready;       // [T*k/128 + E + 1] per 128-row block: Linear-1 warps that published its h rows; zero when idle
+  int32_t* d_order;       // [num_sms][kMoeOrderLogCap] tile codes drawn by each CTA in the last traced one-launch run
   unsigned long long* d_trace;   // [2][num_sms][kMoeTraceFields] wait counters of Linear-1 and Linear-2
   moe_encode_tiled_fn encode_tiled;
   int32_t last_launches;

@@ -177,6 +177,39 @@ def test_pacing_points_are_bitwise_identical():
     L.check_device_status()
 
 
+@pytest.mark.parametrize("cfg", [SMALL[0], SMALL[1], SMALL[5], SMALL[7],
+                                 gen.MoEConfig("waves", T=1500, H=512, F=512, E=6, k=2, seed=51, router="xWr")],
+                         ids=lambda c: c.name)
+def test_schedules_are_bitwise_identical(cfg):
+    """Expert-Wave as two launches, Expert-Wave as one launch with ready counters, and the interleaved order
+    (Algorithm 1) for several leads compute the same bits: only the order of tiles changes."""
+    L = Layer(cfg)
+    lay = L.ctx.workspace_layout()
+    ws = torch.empty(lay["total"], dtype=torch.uint8, device=DEV)
+    base = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, base, ws)
+    torch.cuda.synchronize()
+    assert L.ctx.moe_last_launch_count() == 7
+    ref = oracle_for(L)
+    assert_out_close(dev_bf16_to_f64(base), ref["out"], f"out[{cfg.name}]")
+    R = cfg.R
+    h_base = ws[lay["h"]:lay["h"] + R * cfg.F * 2].clone()
+    variants = [binding.make_tuning(1, 0, 1, debug_flags=2)] + \
+               [binding.make_tuning(1, 0, 1, schedule=1, dep_lead_D=D) for D in (0, 1, 2, 7, 1000)] + \
+               [binding.make_tuning(2, 1, 2, schedule=1, dep_lead_D=1)]
+    for tn in variants:
+        ws[lay["h"]:lay["h"] + R * cfg.F * 2].fill_(0xFF)          # stale h must not be read before it is rewritten
+        out = L.nan_bf16(cfg.T, cfg.H)
+        for _ in range(2):                                          # twice: the ready counters re-arm themselves
+            L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws, tuning=tn)
+        torch.cuda.synchronize()
+        assert L.ctx.moe_last_launch_count() == 6
+        what = (tn.schedule, tn.dep_lead_D, tn.debug_flags)
+        assert torch.equal(ws[lay["h"]:lay["h"] + R * cfg.F * 2], h_base), what
+        assert torch.equal(out.view(torch.int16), base.view(torch.int16)), what
+    L.check_device_status()
+
+
 def test_zero_tokens_is_a_no_op():
     ctx = binding.Context(0, 128, 128, 4, 2)
     counts = torch.full((4,), -1, dtype=torch.int32, device=DEV)
@@ -209,8 +242,8 @@ def test_host_side_errors_are_synchronous():
         with pytest.raises(binding.MoeError) as ei:
             L.ctx.moe_fused_forward(L.x, L.d_logits, w, w, w, out, ws, tuning=bad)
         assert ei.value.code == 1
-    with pytest.raises(binding.MoeError) as ei:       # interleaved schedule not built
-        L.ctx.moe_fused_forward(L.x, L.d_logits, w, w, w, out, ws, tuning=binding.make_tuning(1, 0, 1, schedule=1))
+    with pytest.raises(binding.MoeError) as ei:       # unknown schedule
+        L.ctx.moe_fused_forward(L.x, L.d_logits, w, w, w, out, ws, tuning=binding.make_tuning(1, 0, 1, schedule=2))
     assert ei.value.code == 7
     with pytest.raises(binding.MoeError) as ei:
         binding.Context(8, 100, 128, 4, 2)
