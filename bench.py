@@ -167,6 +167,9 @@ def main():
     ap.add_argument("--burst", type=int, default=1)
     ap.add_argument("--mode", type=int, default=0)
     ap.add_argument("--ik", type=int, default=1)
+    ap.add_argument("--schedule", type=int, default=0, help="0 Expert-Wave order, 1 interleaved order (Algorithm 1)")
+    ap.add_argument("--lead", type=int, default=0, help="schedule 1: row lead D (0 = the anti-starvation knee)")
+    ap.add_argument("--one-launch", action="store_true", help="schedule 0 as one launch with ready counters")
     ap.add_argument("--sweep", action="store_true", help="store-pacing sweep (20 points) instead of the bench line")
     ap.add_argument("--probe-mma", action="store_true",
                     help="print SM clocks per tcgen05.mma for several tile shapes (tensor-pipe calibration) and exit")
@@ -248,7 +251,9 @@ def main():
         run_sweep(args, cfg, ctx, binding, (x, d_logits, w_gate, w_up, w_down, out, ws), timed, rank)
         return
 
-    tuning = binding.make_tuning(args.burst, args.mode, args.ik)
+    dbg = 2 if args.one_launch else 0
+    tuning = binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule, dep_lead_D=args.lead,
+                                 debug_flags=dbg)
     step = lambda: ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tuning)
 
     # ---- device-resident throughput, with per-kernel events, clocks sampled during the timed region
@@ -289,7 +294,8 @@ def main():
 
     ffn_trace = None
     if args.trace:
-        ttn = binding.make_tuning(args.burst, args.mode, args.ik, debug_flags=1)
+        ttn = binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule, dep_lead_D=args.lead,
+                                  debug_flags=dbg | 1)
         ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=ttn)
         tr = ctx.moe_get_ffn_trace().astype(np.float64)          # [2, CTAs, 8]
         ffn_trace = {}
@@ -328,8 +334,11 @@ def main():
     R = cfg.R
     l1_flops = 4 * R * cfg.H * cfg.F
     l2_flops = 2 * R * cfg.H * cfg.F
+    one_launch = args.schedule == 1 or args.one_launch     # both GEMMs in one kernel: its time is in slot 4
+    if one_launch:
+        l1_flops, l2_flops = l1_flops + l2_flops, 0
     l1_tf = l1_flops / (kernel_ms[4] * 1e-3) / 1e12
-    l2_tf = l2_flops / (kernel_ms[5] * 1e-3) / 1e12
+    l2_tf = 0.0 if one_launch else l2_flops / (kernel_ms[5] * 1e-3) / 1e12
     move_bytes = 2 * cfg.H * (cfg.T + R)
     disp_gbs = move_bytes / (kernel_ms[3] * 1e-3) / 1e9
     comb_gbs = (move_bytes + 8 * R) / (kernel_ms[6] * 1e-3) / 1e9
@@ -341,25 +350,30 @@ def main():
     # algorithmic bytes of one Linear-1 launch: gate+up weights of the non-empty experts, x_perm read, h written
     l1_bytes = nonempty * 2 * cfg.F * cfg.H * 2 + R * cfg.H * 2 + R * cfg.F * 2
     l2_bytes = nonempty * cfg.F * cfg.H * 2 + R * cfg.F * 2 + R * cfg.H * 2
+    if one_launch:
+        l1_bytes, l2_bytes = l1_bytes + l2_bytes, 0
     l1_gbs = l1_bytes / (kernel_ms[4] * 1e-3) / 1e9
-    l2_gbs = l2_bytes / (kernel_ms[5] * 1e-3) / 1e9
+    l2_gbs = 0.0 if one_launch else l2_bytes / (kernel_ms[5] * 1e-3) / 1e9
+    gemm_name = ("expert_ffn_kernel (Linear-1 + SiLU*mul + Linear-2, one launch)" if one_launch
+                 else "expert_ffn_kernel, Linear-1 + SiLU*mul launch")
     # the roofline that binds Linear-1: tensor time at the measured GEMM peak vs HBM time at the measured copy rate
     t_tensor = l1_flops / (peak_tf * 1e12)
     t_hbm = l1_bytes / (peak_hbm * 1e9)
     if t_tensor >= t_hbm:
         roofline = {
-            "kernel": "expert_gemm_kernel<gated> (Linear-1 + SiLU*mul)", "bound": "tensor", "achieved": l1_tf,
+            "kernel": gemm_name, "bound": "tensor", "achieved": l1_tf,
             "peak": peak_tf, "unit": "TFLOP/s", "frac": l1_tf / peak_tf,
-            "traffic": LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name),
+            "traffic": None if one_launch else LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name),
             "peak_source": f"{peak_kind} bf16_tflops (burst)",
             "frac_of_sustained": l1_tf / float(peaks.get("bf16_tflops_sustained", peak_tf)),
             "flops_per_launch": l1_flops, "ms_per_launch": kernel_ms[4],
         }
     else:
         roofline = {
-            "kernel": "expert_gemm_kernel<gated> (Linear-1 + SiLU*mul)", "bound": "hbm", "achieved": l1_gbs,
+            "kernel": gemm_name, "bound": "hbm", "achieved": l1_gbs,
             "peak": peak_hbm, "unit": "GB/s", "frac": l1_gbs / peak_hbm,
-            "traffic": LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name), "peak_source": f"{peak_kind} hbm_gbs (copy)",
+            "traffic": None if one_launch else LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name),
+            "peak_source": f"{peak_kind} hbm_gbs (copy)",
             "bytes_per_launch": l1_bytes, "ms_per_launch": kernel_ms[4], "nonempty_experts": nonempty,
             "tensor_tflops": l1_tf,
         }
@@ -376,6 +390,7 @@ def main():
         "e2e": {"value": tokens / (e2e_ms / args.steps * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": launches, "clocks": clocks, "tuning": [args.burst, args.mode, args.ik],
+        "schedule": {"schedule": args.schedule, "lead_D": args.lead, "one_launch": one_launch},
     }
     if ffn_trace is not None:
         line["ffn_trace"] = ffn_trace

@@ -70,7 +70,8 @@ typedef struct {
                                       anti-starvation knee ceil(128 * SMs / (2 F)) (App. A.2).  Must be 0 for
                                       schedule 0. */
   int32_t debug_flags;             /* bit 0: record per-CTA wait counters (moe_get_ffn_trace); bit 1: run
-                                      schedule 0 as one launch with ready counters instead of two; other bits 0 */
+                                      schedule 0 as one launch with ready counters instead of two (layers whose
+                                      tiles fit in about one wave of CTAs always do); other bits 0 */
 } moe_tuning;
 
 /* Byte offsets of the slices of the workspace used by moe_fused_forward (each 256-byte aligned). */

@@ -30,8 +30,8 @@ EXPORTS = (
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
                 "epilogue_wait_accumulator", "epilogue_store_span", "tiles", "epilogue_pacing_gap")
 
-KERNEL_NAMES = ("route_topk_hist", "route_scan", "route_scatter", "dispatch_rows", "expert_gemm_linear1",
-                "expert_gemm_linear2", "combine_rows")
+KERNEL_NAMES = ("route_topk_hist", "route_scan", "route_scatter", "dispatch_rows", "expert_ffn_linear1",
+                "expert_ffn_linear2", "combine_rows")
 
 
 class MoeError(RuntimeError):

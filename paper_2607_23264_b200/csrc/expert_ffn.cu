@@ -672,7 +672,10 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
   // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
   p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);
   const bool trace = (tn.debug_flags & 1) != 0;
-  const bool one_launch = tn.schedule == 1 || (tn.debug_flags & 2) != 0;
+  // Launch-latency-bound layers (every tile fits in about one wave of CTAs) run both GEMMs in one launch.
+  const long long max_blocks = static_cast<long long>(R / 128) + s.E;
+  const bool tiny = max_blocks * (p.ph[0].n_blocks + p.ph[1].n_blocks) <= 2LL * grid;
+  const bool one_launch = tn.schedule == 1 || (tn.debug_flags & 2) != 0 || tiny;
 
   if (one_launch) {
     p.phase_lo = 0;

@@ -10,6 +10,7 @@ import torch
 
 from oracle import moe_oracle as orc
 from paper_2607_23264_b200 import inputs as gen
+from paper_2607_23264_b200 import binding
 from moe_testlib import (DEV, TOL_FRO, Layer, assert_out_close, assert_plan_matches, dev_bf16_to_f64, dev_to_bits,
                          rel_fro, sample_tokens)
 
@@ -57,6 +58,14 @@ def run_sampled(cfg, n_random, max_boundary):
     out_np = dev_bf16_to_f64(out)
     assert np.isfinite(out_np).all(), "every token row must be written"
     assert_out_close(out_np[toks], ref["out"], f"out[{cfg.name}] on {len(toks)} sampled tokens")
+
+    # the interleaved order (Algorithm 1, one launch with ready counters) must give the same bits at full size
+    out1 = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out1, ws,
+                            tuning=binding.make_tuning(1, 0, 1, schedule=1, dep_lead_D=8))
+    torch.cuda.synchronize()
+    L.check_device_status()
+    assert torch.equal(out1.view(torch.int16), out.view(torch.int16)), "schedule 1 differs from schedule 0"
     return L, plan
 
 

@@ -76,7 +76,7 @@ def test_expert_ffn_parity(cfg):
     L.ctx.moe_expert_ffn(x_perm, offsets, L.w_gate, L.w_up, L.w_down, h, y, h_fp32_debug=h32)
     torch.cuda.synchronize()
     L.check_device_status()
-    assert L.ctx.moe_last_launch_count() == 2
+    assert L.ctx.moe_last_launch_count() in (1, 2)      # tiny layers run both GEMMs in one launch
     h32_np = h32.cpu().numpy().astype(np.float64)
     assert np.isfinite(h32_np).all(), "every row of h belongs to an expert and must be written"
     assert rel_fro(h32_np, ref["h"]) <= TOL_FRO
@@ -119,7 +119,7 @@ def test_fused_forward_parity(cfg):
     L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
     torch.cuda.synchronize()
     L.check_device_status()
-    assert L.ctx.moe_last_launch_count() == 7
+    assert L.ctx.moe_last_launch_count() in (6, 7)
 
     def sl(name, count, dtype):
         nbytes = count * torch.empty((), dtype=dtype).element_size()
@@ -189,7 +189,7 @@ def test_schedules_are_bitwise_identical(cfg):
     base = L.nan_bf16(cfg.T, cfg.H)
     L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, base, ws)
     torch.cuda.synchronize()
-    assert L.ctx.moe_last_launch_count() == 7
+    assert L.ctx.moe_last_launch_count() in (6, 7)
     ref = oracle_for(L)
     assert_out_close(dev_bf16_to_f64(base), ref["out"], f"out[{cfg.name}]")
     R = cfg.R
@@ -254,7 +254,7 @@ def test_host_side_errors_are_synchronous():
 
 def test_ffn_trace_and_kernel_times():
     """Measurement aids: per-kernel event times and the per-CTA wait counters of the grouped GEMMs."""
-    cfg = SMALL[1]
+    cfg = gen.MoEConfig("traced", T=4000, H=512, F=384, E=6, k=2, seed=61, router="xWr")   # two launches
     L = Layer(cfg)
     ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
     out = L.nan_bf16(cfg.T, cfg.H)
