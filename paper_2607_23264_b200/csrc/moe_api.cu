@@ -120,7 +120,11 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
     delete ctx;
     return MOE_ERR_CUDA;
   }
-  ctx->tokens_per_chunk = kRouteThreads / shape->k;   // k <= 32, so at least 8 tokens
+  // A routing chunk holds at most 256 slots (k <= 32, so at least 8 tokens).  Small batches use smaller chunks,
+  // down to one token per warp, so that the top-k work spreads over about two CTAs per SM.
+  ctx->tokens_per_chunk = kRouteThreads / shape->k;
+  const int spread = (shape->T + 2 * ctx->num_sms - 1) / (2 * ctx->num_sms);
+  if (spread < ctx->tokens_per_chunk) ctx->tokens_per_chunk = spread < 8 ? 8 : spread;
   ctx->num_chunks = shape->T ? (shape->T + ctx->tokens_per_chunk - 1) / ctx->tokens_per_chunk : 0;
   const size_t hist_elems = static_cast<size_t>(ctx->num_chunks ? ctx->num_chunks : 1) * shape->E;
 

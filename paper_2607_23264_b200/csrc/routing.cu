@@ -86,7 +86,19 @@ route_scan(const int32_t* __restrict__ chunk_hist, int32_t* __restrict__ chunk_b
   const int e = threadIdx.x, lane = e & 31, warp = e >> 5;
   int32_t total = 0;
   if (e < E) {
-    for (int c = 0; c < num_chunks; ++c) {
+    // eight chunks per step: the loads are independent, only the running sum is serial
+    int c = 0;
+    for (; c + 8 <= num_chunks; c += 8) {
+      int32_t v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = chunk_hist[static_cast<size_t>(c + u) * E + e];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        chunk_base[static_cast<size_t>(c + u) * E + e] = total;
+        total += v[u];
+      }
+    }
+    for (; c < num_chunks; ++c) {
       const size_t i = static_cast<size_t>(c) * E + e;
       const int32_t v = chunk_hist[i];
       chunk_base[i] = total;
