@@ -173,6 +173,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="store-pacing sweep (20 points) instead of the bench line")
     ap.add_argument("--probe-mma", action="store_true",
                     help="print SM clocks per tcgen05.mma for several tile shapes (tensor-pipe calibration) and exit")
+    ap.add_argument("--xstage-probe", action="store_true",
+                    help="run the burst/gap store microbenchmark on local HBM, print the rows and the calibration, exit")
     ap.add_argument("--trace", action="store_true",
                     help="add the grouped GEMMs' per-CTA wait counters (one extra traced step) to the JSON line")
     ap.add_argument("--profile", action="store_true",
@@ -202,6 +204,9 @@ def main():
                 for M in (128, 64) for N in (16, 32, 64, 128, 256)]
         print(json.dumps({"probe": "tcgen05.mma kind::f16 MxNx16, one CTA, operands resident in shared memory",
                           "rows": rows}), flush=True)
+        return
+    if args.xstage_probe:
+        run_xstage_probe(dev)
         return
     replicas.init_process_group(world, "nccl", torch.device(dev))
 
@@ -405,6 +410,54 @@ def main():
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_xstage_probe(dev):
+    """Periodic-burst gap sweep, zero-gap decompositions and isolated bursts on this GPU's own HBM."""
+    import torch
+    from paper_2607_23264_b200 import xstage
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    buf = torch.empty(1 << 30, dtype=torch.uint8, device=dev)          # 1 GiB: slices of 7 MB per producer, far above L2
+    KiB = 1024
+    med = lambda xs: statistics.median(xs)
+    out = {"probe": "xstage_store_probe: K producers x B bytes of 16-byte stores, gap G, local HBM", "sms": sms}
+    xstage.xstage_store_probe(sms, 8 * KiB, 0, 50, buf)                # warm-up
+    periodic = []
+    for B in (8 * KiB, 32 * KiB, 128 * KiB):
+        for gap in (0, 250, 500, 1000, 2000, 4000, 8000, 16000, 32000):
+            r = xstage.xstage_store_probe(sms, B, gap, 300, buf)
+            tail = slice(100, 300)
+            periodic.append({"producers": sms, "bytes_per_producer": B, "volume": sms * B, "gap": gap,
+                             "t_iss": med(r["issue_mean"][tail]), "t_iss_max": med(r["issue_max"][tail]),
+                             "t_period": med(r["period_mean"][tail]), "clocks_per_us": r["clocks_per_us"]})
+    out["periodic"] = periodic
+    decomp = []
+    for K, B in ((sms, 32 * KiB), (sms // 2, 64 * KiB), (sms // 4, 128 * KiB)):
+        r = xstage.xstage_store_probe(K, B, 0, 300, buf)
+        tp = med(r["period_mean"][100:300])
+        decomp.append({"producers": K, "bytes_per_producer": B, "volume": K * B, "t_period": tp,
+                       "bytes_per_clock": K * B / tp, "gb_per_s": K * B / tp * r["clocks_per_us"] / 1e3})
+    out["zero_gap_decompositions"] = decomp
+    isolated = []
+    sizes = [b * KiB for b in (1, 2, 4, 8, 12, 16, 20, 24, 28, 32, 40, 48, 64, 96, 128, 256, 512, 1024, 2048, 4096)]
+    for B in sizes:
+        runs = [xstage.xstage_store_probe(sms, B, 0, 1, buf) for _ in range(9)]
+        isolated.append({"producers": sms, "bytes_per_producer": B, "volume": sms * B,
+                         "t_iss": med([x["issue_mean"][0] for x in runs]), "t_iss_max": med([x["issue_max"][0] for x in runs])})
+    out["isolated"] = isolated
+    cal = {}
+    for B in (8 * KiB, 32 * KiB, 128 * KiB):
+        rows = [r for r in periodic if r["bytes_per_producer"] == B]
+        c = xstage.calibrate(rows, isolated)
+        cpu = med([r["clocks_per_us"] for r in rows])
+        c["clocks_per_us"] = cpu
+        c["rate_gb_per_s"] = c["rate"] * cpu / 1e3 if c["rate"] else None
+        c["t_iss0_us"] = c["t_iss0"] / cpu
+        if c["rate"]:
+            c["recovery_gap_clocks"] = xstage.xstage_recovery_gap(c["t_iss0"], c["rate"], sms * B)
+        cal[str(B)] = c
+    out["calibration_by_bytes_per_producer"] = cal
+    print(json.dumps(out), flush=True)
 
 
 def run_sweep(args, cfg, ctx, binding, bufs, timed, rank):

@@ -4,7 +4,7 @@
  * The model M_X = (T_iss^0, R, Q) (Sec. 3.3): recovered issue floor, effective aggregate drain rate and
  * effective outstanding capacity of a store path, calibrated by microbenchmarks, then applied to a kernel's
  * burst sequence {V_n, T_iss,n^0, G_n}.  All functions are pure host arithmetic in double precision; they
- * allocate nothing and touch no GPU.  Units are the caller's, used consistently: bytes, seconds, bytes/second
+ * allocate nothing and touch no GPU (the one exception, the store microbenchmark at the end, says so).  Units are the caller's, used consistently: bytes, seconds, bytes/second
  * in the examples (the paper's GB is 1e9 bytes, its MiB 2^20 bytes).  [z]_+ means max(z, 0).
  * Pointers are HOST pointers owned by the caller.  Functions returning int return 0 on success and -1 on a bad
  * argument (null pointer, non-positive rate or period, negative count); value-returning functions return NaN
@@ -71,6 +71,25 @@ double xstage_mma_stall(double t_remote_store_span, double t_cover_mma);
 /* App. C.2, tile-aligned sequence length above which the Q-loop gap (at least sigma per K/V tile) covers the
  * recovery gap: M_ub = b_n ceil(G* / sigma).  -1 on a bad argument. */
 int64_t xstage_fa_recovery_length(int64_t b_n, double recovery_gap, double sigma);
+
+/*
+ * Store microbenchmark on this GPU's own memory (Sec. 3.1's periodic-burst and isolated-burst patterns, run as the
+ * paper's local-memory control: same producer count, store width, address generation and loop structure, local
+ * destination).  `producers` CTAs of 128 threads, one per SM (producers <= SM count), start together; each
+ * repeats `periods` times: issue bytes_per_burst bytes (a multiple of 16) as 16-byte stores into its own slice of
+ * device_buffer (DEVICE pointer, 16-byte aligned, buffer_bytes / producers >= bytes_per_burst; slices are walked
+ * and wrap, so a buffer well above the L2 size keeps the stores going to HBM), then spin gap_clocks SM clocks
+ * without storing.  periods = 1 with gap 0 is an isolated burst from a recovered state.
+ * Results, HOST arrays of `periods` doubles, in SM clocks: issue_mean_clocks / issue_max_clocks (may be NULL) =
+ * mean / maximum over producers of the sender-visible issue span of burst n (first store issued to last store
+ * issued, not completion); period_mean_clocks = mean period n (issue + gap).  *clocks_per_us (may be NULL) = SM
+ * clocks per microsecond during the run (clock64 against globaltimer).  Allocates and frees a small device result
+ * buffer, runs on the current device, synchronises `stream`.  Returns 0, -1 bad argument, -2 CUDA error,
+ * -3 the producers could not be started together within the wait budget.
+ */
+int xstage_store_probe(int32_t producers, int64_t bytes_per_burst, int64_t gap_clocks, int32_t periods,
+                       void* device_buffer, uint64_t buffer_bytes, double* issue_mean_clocks,
+                       double* issue_max_clocks, double* period_mean_clocks, double* clocks_per_us, void* stream);
 
 #ifdef __cplusplus
 }

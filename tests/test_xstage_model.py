@@ -164,3 +164,53 @@ def test_every_declared_function_is_exported():
     lib = xstage._lib()
     for n in names:
         assert hasattr(lib, n)
+
+
+def test_calibrate_recovers_model_parameters_from_synthetic_rows():
+    """Rows generated from the oracle's Burst-Gap law and capacity guard give back T0, R and a capacity
+    estimate that brackets Q."""
+    T0, R, Q = 800.0, 3000.0, 12.0e6           # clocks, bytes per clock, bytes
+    V = 148 * 32768
+    periodic = []
+    for gap in (0, 250, 500, 1000, 2000, 4000, 8000, 16000, 32000):
+        tp, ti = xo.burst_gap(T0, R, V, gap)
+        periodic.append(dict(volume=V, gap=gap, t_iss=ti, t_period=tp))
+    floor = 150.0                              # a recovered burst is absorbed at a constant issue floor ...
+    isolated = []
+    for b in (2048 * i for i in range(1, 80)):
+        v = 148 * b
+        over = xo.pos(xo.isolated_occupancy(floor, R, v) - Q)      # ... until its occupancy exceeds Q (Eq. 6)
+        isolated.append(dict(volume=v, t_iss=floor + over / R))    # then issue stretches until the excess drains
+    c = xstage.calibrate(periodic, isolated)
+    assert c["t_iss0"] == pytest.approx(T0)
+    assert c["rate"] == pytest.approx(R)                      # zero gap: T_period = V / R
+    assert c["floor_intercept"] == pytest.approx(floor) and abs(c["floor_per_byte"]) < 1e-12
+    step = 148 * 2048
+    # the knee is the last volume on the floor: Q lies within a few sweep steps above the estimate
+    assert c["capacity"] <= Q + R * floor and Q - c["capacity"] < 3 * step
+    flat = xstage.calibrate(periodic, [dict(volume=r["volume"], t_iss=floor) for r in isolated])
+    assert flat["capacity"] is None and flat["knee_volume"] is None, "no knee, no capacity estimate"
+
+
+@pytest.mark.gpu
+def test_store_probe_runs_and_reports_consistent_spans():
+    import torch
+    buf = torch.zeros(256 << 20, dtype=torch.uint8, device="cuda:0")
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    r = xstage.xstage_store_probe(sms, 8192, 2000, 40, buf)
+    assert 0.5e3 < r["clocks_per_us"] < 2.5e3
+    for n in range(40):
+        assert 0 < r["issue_mean"][n] <= r["issue_max"][n]
+        assert r["period_mean"][n] >= r["issue_mean"][n] + 2000 - 1
+    torch.cuda.synchronize()
+    # every producer wrote its own slice: burst 0 of producer p starts at p * slice with (n=0, producer=p, tid, tag)
+    words = buf.view(torch.int32)
+    slice_words = (buf.numel() // 16 // sms) * 4
+    for p in (0, 1, sms - 1):
+        assert words[p * slice_words + 1].item() == p and words[p * slice_words + 3].item() == 0x5A5A5A5A
+    iso = xstage.xstage_store_probe(sms, 1 << 20, 0, 1, buf)
+    assert iso["issue_mean"][0] > r["issue_mean"][5], "a 1 MiB burst per producer takes longer to issue than 8 KiB"
+    with pytest.raises(RuntimeError):
+        xstage.xstage_store_probe(sms + 1, 8192, 0, 1, buf)
+    with pytest.raises(RuntimeError):
+        xstage.xstage_store_probe(sms, 24, 0, 1, buf)
