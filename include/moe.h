@@ -71,7 +71,10 @@ typedef struct {
                                       schedule 0. */
   int32_t debug_flags;             /* bit 0: record per-CTA wait counters (moe_get_ffn_trace); bit 1: run
                                       schedule 0 as one launch with ready counters instead of two (layers whose
-                                      tiles fit in about one wave of CTAs always do); other bits 0 */
+                                      tiles fit in about one wave of CTAs always do); bit 2: failure drill, requested
+                                      by the host: runs as one launch in which Linear-1 never publishes its rows, so
+                                      every Linear-2 wait expires (after about 0.1 s), the kernel unwinds and the
+                                      status word reads MOE_ERR_TIMEOUT; outputs are then undefined; other bits 0 */
 } moe_tuning;
 
 /* Byte offsets of the slices of the workspace used by moe_fused_forward (each 256-byte aligned). */

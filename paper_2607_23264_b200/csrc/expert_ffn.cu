@@ -93,6 +93,8 @@ struct FfnParams {
   int phase_lo, phase_hi;   // GEMMs in this launch: [0,1) Linear-1, [1,2) Linear-2, [0,2) both
   int schedule;             // 0 merged order drawn dynamically, 1 Algorithm 1
   int lead_D;               // Algorithm 1: minimum row lead of Linear-1 over Linear-2 (>= 1)
+  int withhold_ready;       // host-requested failure drill: Linear-1 never publishes its rows (one-launch runs)
+  long long wait_budget;    // clocks a cross-CTA wait may last before it gives up
   int kernel_id;
 };
 
@@ -179,7 +181,8 @@ __device__ __forceinline__ void pace_gap(SharedTail* st, uint32_t start, int ik)
 }
 
 // Bounded wait until `*counter` (written by other CTAs with release ordering) reaches `target`.
-__device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, volatile int* abort_flag,
+                                             long long budget) {
   const long long t0 = clock64();
   for (uint32_t it = 0;; ++it) {
     int v;
@@ -187,7 +190,7 @@ __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target,
     if (v >= target) return true;
     if ((it & 0xFu) == 0xFu) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > ptx::kWaitClockBudget) {
+      if (clock64() - t0 > budget) {
         *abort_flag = 1;
         return false;
       }
@@ -386,7 +389,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         const CUtensorMap* mb1 = t.phase == 0 ? &tm_wu : &tm_wd;
         if (chained && t.phase == 1) {
           // every Linear-1 tile of this row (n_blocks tiles x 4 epilogue warps) must have published its h rows
-          if (!wait_counter(&p.ready[t.block], 4 * p.ph[0].n_blocks, abort_flag)) {
+          if (!wait_counter(&p.ready[t.block], 4 * p.ph[0].n_blocks, abort_flag, p.wait_budget)) {
             report_timeout(p, 8);
             break;
           }
@@ -517,7 +520,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       __syncwarp();
       if (lane == 0) {
         ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
-        if (chained && t.phase == 0) atomicAdd(&p.ready[t.block], 1);
+        if (chained && t.phase == 0 && !p.withhold_ready) atomicAdd(&p.ready[t.block], 1);
       }
       busy += clock64() - t_store;
       acc ^= 1;
@@ -671,11 +674,13 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
   // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
   p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);
+  p.withhold_ready = (tn.debug_flags & 4) != 0;
+  p.wait_budget = p.withhold_ready ? 200000000LL : ptx::kWaitClockBudget;   // the drill gives up after ~0.1 s
   const bool trace = (tn.debug_flags & 1) != 0;
   // Launch-latency-bound layers (every tile fits in about one wave of CTAs) run both GEMMs in one launch.
   const long long max_blocks = static_cast<long long>(R / 128) + s.E;
   const bool tiny = max_blocks * (p.ph[0].n_blocks + p.ph[1].n_blocks) <= 2LL * grid;
-  const bool one_launch = tn.schedule == 1 || (tn.debug_flags & 2) != 0 || tiny;
+  const bool one_launch = tn.schedule == 1 || (tn.debug_flags & 6) != 0 || tiny;
 
   if (one_launch) {
     p.phase_lo = 0;

@@ -275,3 +275,28 @@ def test_ffn_trace_and_kernel_times():
     assert tr[1, :, 6].sum() == mblocks * ((cfg.H + 255) // 256)
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16)), "tracing must not change values"
     L.check_device_status()
+
+
+def test_expired_wait_is_reported_not_hung():
+    """Failure path without a GPU fault: the host asks Linear-1 to withhold its ready counts, so every bounded
+    Linear-2 wait runs out; the kernel must unwind by itself, report MOE_ERR_TIMEOUT in the status word, and the
+    context must stay usable (the next run is correct)."""
+    import time
+    cfg = gen.MoEConfig("drill", T=600, H=256, F=256, E=4, k=2, seed=71, router="xWr")
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    t0 = time.time()
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws,
+                            tuning=binding.make_tuning(1, 0, 1, debug_flags=4))
+    code, detail = L.ctx.moe_last_device_status()          # synchronises
+    assert time.time() - t0 < 10.0, "the drill must end by itself"
+    assert code == 6, "MOE_ERR_TIMEOUT expected"
+    assert detail >> 16 == 3 and (detail & 0xFFFF) in (1, 2, 3, 4, 5, 6, 7, 8), "kernel 3 (one launch), some role"
+    assert L.ctx.moe_last_device_status() == (0, 0), "reading the status clears it"
+    # the same context computes correctly afterwards: scheduler and ready counters were re-armed
+    for tn in (None, binding.make_tuning(1, 0, 1, schedule=1, dep_lead_D=2)):
+        L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws, tuning=tn)
+        torch.cuda.synchronize()
+        assert_out_close(dev_bf16_to_f64(out), oracle_for(L)["out"], "after the drill")
+    L.check_device_status()
