@@ -91,6 +91,9 @@ typedef struct {
   size_t x_stage;    /* bf16  [T,H]  device staging for moe_fused_forward_host */
   size_t logits_stage; /* fp32 [T,E] device staging for moe_fused_forward_host */
   size_t out_stage;  /* bf16  [T,H]  device staging for moe_fused_forward_host */
+  size_t x_stage_b;  /* second staging slot of moe_fused_forward_host_pipelined: bf16 [T,H] */
+  size_t logits_stage_b; /* fp32 [T,E] */
+  size_t out_stage_b;    /* bf16 [T,H] */
   size_t total;      /* = moe_workspace_bytes */
 } moe_workspace_layout;
 
@@ -204,6 +207,22 @@ moe_status moe_fused_forward_host(moe_ctx* ctx, const void* x_host, const float*
                                   const void* w_gate, const void* w_up, const void* w_down,
                                   void* out_host, void* workspace, size_t workspace_bytes,
                                   const moe_tuning* tuning, void* stream);
+
+/*
+ * The host-buffer call as a two-deep pipeline, for callers that run step after step (serving): consecutive calls
+ * alternate between two staging slots, the input copy of call i+1 runs on an internal copy stream while call i
+ * computes on `stream`, and the output copy of call i runs on a second internal stream while call i+1 computes.
+ * The intermediates are single-buffered, so the layers themselves still run one after another on `stream`.
+ * Same arguments as moe_fused_forward_host; x_host, logits_host and out_host should be pinned and must stay
+ * valid until the pipeline is flushed.  out_host of call i is complete only after a later
+ * moe_host_pipeline_flush(ctx, stream) followed by a synchronisation of `stream` (the flush makes `stream` wait
+ * for every copy issued so far).  Use one `stream` per context.
+ */
+moe_status moe_fused_forward_host_pipelined(moe_ctx* ctx, const void* x_host, const float* logits_host,
+                                            const void* w_gate, const void* w_up, const void* w_down,
+                                            void* out_host, void* workspace, size_t workspace_bytes,
+                                            const moe_tuning* tuning, void* stream);
+moe_status moe_host_pipeline_flush(moe_ctx* ctx, void* stream);
 
 /*
  * Synchronise `stream`, then read and clear the device status word.  *code is MOE_OK or MOE_ERR_TIMEOUT;

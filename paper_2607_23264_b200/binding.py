@@ -24,7 +24,7 @@ EXPORTS = (
     "moe_plan_routing", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_fused_forward",
     "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count", "moe_set_kernel_timing",
     "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace", "moe_probe_mma_cycles",
-    "moe_get_ffn_order",
+    "moe_get_ffn_order", "moe_fused_forward_host_pipelined", "moe_host_pipeline_flush",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -51,7 +51,8 @@ class moe_tuning(C.Structure):
 
 class moe_workspace_layout(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in ("topk_ids", "topk_w", "counts", "offsets", "perm", "inv_perm", "x_perm",
-                                          "h", "y_perm", "x_stage", "logits_stage", "out_stage", "total")]
+                                          "h", "y_perm", "x_stage", "logits_stage", "out_stage", "x_stage_b",
+                                          "logits_stage_b", "out_stage_b", "total")]
 
 
 _lib = None
@@ -83,6 +84,8 @@ def load_library() -> C.CDLL:
     lib.moe_combine.argtypes = [vp, vp, i32p, f32p, vp, vp]
     lib.moe_fused_forward.argtypes = [vp, vp, f32p, vp, vp, vp, vp, vp, C.c_size_t, C.POINTER(moe_tuning), vp]
     lib.moe_fused_forward_host.argtypes = [vp, vp, f32p, vp, vp, vp, vp, vp, C.c_size_t, C.POINTER(moe_tuning), vp]
+    lib.moe_fused_forward_host_pipelined.argtypes = lib.moe_fused_forward_host.argtypes
+    lib.moe_host_pipeline_flush.argtypes = [vp, vp]
     lib.moe_last_device_status.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_last_launch_count.argtypes = [vp]
     lib.moe_last_launch_count.restype = C.c_int32
@@ -227,6 +230,17 @@ class Context:
                                                 _ptr(w_up), _ptr(w_down), _ptr(out_host), _ptr(workspace),
                                                 workspace.numel() * workspace.element_size(), _tuning_ref(tuning),
                                                 _stream(stream)), "moe_fused_forward_host")
+
+    def moe_fused_forward_host_pipelined(self, x_host, logits_host, w_gate, w_up, w_down, out_host, workspace,
+                                         tuning=None, stream=None):
+        _check(self._lib.moe_fused_forward_host_pipelined(self._handle, _ptr(x_host), _ptr(logits_host), _ptr(w_gate),
+                                                          _ptr(w_up), _ptr(w_down), _ptr(out_host), _ptr(workspace),
+                                                          workspace.numel() * workspace.element_size(),
+                                                          _tuning_ref(tuning), _stream(stream)),
+               "moe_fused_forward_host_pipelined")
+
+    def moe_host_pipeline_flush(self, stream=None):
+        _check(self._lib.moe_host_pipeline_flush(self._handle, _stream(stream)), "moe_host_pipeline_flush")
 
     def moe_last_device_status(self, stream=None):
         code, detail = C.c_int32(0), C.c_int32(0)

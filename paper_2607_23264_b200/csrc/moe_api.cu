@@ -64,6 +64,9 @@ void fill_layout(const moe_shape& s, moe_workspace_layout* L) {
   L->x_stage = take(T * H * 2);
   L->logits_stage = take(T * E * 4);
   L->out_stage = take(T * H * 2);
+  L->x_stage_b = take(T * H * 2);
+  L->logits_stage_b = take(T * E * 4);
+  L->out_stage_b = take(T * H * 2);
   L->total = off;
 }
 
@@ -154,6 +157,13 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   ok = ok && cudaMemset(ctx->d_sched, 0, 4 * 4) == cudaSuccess;
   ok = ok && moe::prepare_expert_ffn(ctx) == cudaSuccess;
   for (int i = 0; ok && i <= kMoeKernels; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) == cudaSuccess;
+  for (int i = 0; ok && i < 2; ++i) {
+    ok = cudaEventCreateWithFlags(&ctx->ev_h2d[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&ctx->ev_compute[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&ctx->ev_d2h[i], cudaEventDisableTiming) == cudaSuccess;
+  }
   if (!ok) {
     moe_destroy(ctx);
     return MOE_ERR_CUDA;
@@ -173,6 +183,13 @@ void moe_destroy(moe_ctx* ctx) {
   if (ctx->d_order) cudaFree(ctx->d_order);
   for (int i = 0; i <= kMoeKernels; ++i)
     if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
+  for (int i = 0; i < 2; ++i) {
+    if (ctx->ev_h2d[i]) cudaEventDestroy(ctx->ev_h2d[i]);
+    if (ctx->ev_compute[i]) cudaEventDestroy(ctx->ev_compute[i]);
+    if (ctx->ev_d2h[i]) cudaEventDestroy(ctx->ev_d2h[i]);
+  }
+  if (ctx->s_h2d) cudaStreamDestroy(ctx->s_h2d);
+  if (ctx->s_d2h) cudaStreamDestroy(ctx->s_d2h);
   delete ctx;
 }
 
@@ -305,6 +322,60 @@ moe_status moe_fused_forward_host(moe_ctx* ctx, const void* x_host, const float*
   if (st != MOE_OK) return st;
   if (cudaMemcpyAsync(out_host, ws + L.out_stage, act_bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
     return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+moe_status moe_fused_forward_host_pipelined(moe_ctx* ctx, const void* x_host, const float* logits_host,
+                                            const void* w_gate, const void* w_up, const void* w_down,
+                                            void* out_host, void* workspace, size_t workspace_bytes,
+                                            const moe_tuning* tuning, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  const moe_shape& s = ctx->shape;
+  if (s.T == 0) { ctx->last_launches = 0; return MOE_OK; }
+  if (!x_host || !logits_host || !out_host || !workspace) return MOE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MOE_ERR_INVALID_ARG;
+  moe_workspace_layout L;
+  fill_layout(s, &L);
+  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE_TOO_SMALL;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const int slot = ctx->pipe_slot;
+  unsigned char* x_dev = ws + (slot ? L.x_stage_b : L.x_stage);
+  unsigned char* lg_dev = ws + (slot ? L.logits_stage_b : L.logits_stage);
+  unsigned char* out_dev = ws + (slot ? L.out_stage_b : L.out_stage);
+  const size_t act_bytes = static_cast<size_t>(s.T) * s.H * 2;
+  const size_t logit_bytes = static_cast<size_t>(s.T) * s.E * 4;
+  // input copy: once the layer that last read this slot (two calls ago) has finished
+  bool ok = cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_compute[slot], 0) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(x_dev, x_host, act_bytes, cudaMemcpyHostToDevice, ctx->s_h2d) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(lg_dev, logits_host, logit_bytes, cudaMemcpyHostToDevice, ctx->s_h2d) == cudaSuccess;
+  ok = ok && cudaEventRecord(ctx->ev_h2d[slot], ctx->s_h2d) == cudaSuccess;
+  // the layer: after its inputs have landed and the slot's previous output has left
+  ok = ok && cudaStreamWaitEvent(cs, ctx->ev_h2d[slot], 0) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(cs, ctx->ev_d2h[slot], 0) == cudaSuccess;
+  if (!ok) return MOE_ERR_CUDA;
+  st = moe_fused_forward(ctx, x_dev, reinterpret_cast<const float*>(lg_dev), w_gate, w_up, w_down, out_dev, workspace,
+                         workspace_bytes, tuning, stream);
+  if (st != MOE_OK) return st;
+  ok = cudaEventRecord(ctx->ev_compute[slot], cs) == cudaSuccess;
+  // output copy: overlaps the next call's layer
+  ok = ok && cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_compute[slot], 0) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(out_host, out_dev, act_bytes, cudaMemcpyDeviceToHost, ctx->s_d2h) == cudaSuccess;
+  ok = ok && cudaEventRecord(ctx->ev_d2h[slot], ctx->s_d2h) == cudaSuccess;
+  if (!ok) return MOE_ERR_CUDA;
+  ctx->pipe_slot = slot ^ 1;
+  return MOE_OK;
+}
+
+moe_status moe_host_pipeline_flush(moe_ctx* ctx, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  for (int i = 0; i < 2; ++i) {
+    if (cudaStreamWaitEvent(cs, ctx->ev_d2h[i], 0) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaStreamWaitEvent(cs, ctx->ev_h2d[i], 0) != cudaSuccess) return MOE_ERR_CUDA;
+  }
   return MOE_OK;
 }
 

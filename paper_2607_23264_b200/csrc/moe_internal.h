@@ -38,6 +38,10 @@ struct moe_ctx {
   unsigned long long* d_trace;   // [2][num_sms][kMoeTraceFields] wait counters of Linear-1 and Linear-2
   moe_encode_tiled_fn encode_tiled;
   int32_t last_launches;
+  // Two-deep pipeline of moe_fused_forward_host_pipelined: copy streams, per-slot events, next slot.
+  cudaStream_t s_h2d, s_d2h;
+  cudaEvent_t ev_h2d[2], ev_compute[2], ev_d2h[2];
+  int pipe_slot;
   // Optional per-kernel timing: event i is recorded after kernel i (event 0 before the first kernel).
   int timing;
   uint32_t ev_recorded;          // bit i set when ev[i] was recorded by the last call

@@ -46,7 +46,7 @@ def test_workspace_layout_is_aligned_and_ordered(lib):
     R = T * k
     sizes = dict(topk_ids=R * 4, topk_w=R * 4, counts=E * 4, offsets=(E + 1) * 4, perm=R * 4, inv_perm=R * 4,
                  x_perm=R * H * 2, h=R * F * 2, y_perm=R * H * 2, x_stage=T * H * 2, logits_stage=T * E * 4,
-                 out_stage=T * H * 2)
+                 out_stage=T * H * 2, x_stage_b=T * H * 2, logits_stage_b=T * E * 4, out_stage_b=T * H * 2)
     prev_end = 0
     for name, size in sizes.items():
         assert L[name] % 256 == 0

@@ -156,6 +156,32 @@ def test_fused_forward_host_matches_device_path():
     assert np.array_equal(out_host.numpy().view(np.uint16), dev_to_bits(out))
 
 
+def test_pipelined_host_calls_match_device_path():
+    """Five pipelined host-buffer steps on different batches: every out_host equals the device-resident result."""
+    cfg = SMALL[1]
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    rng = np.random.default_rng(9)
+    xs, lgs, outs, want = [], [], [], []
+    for i in range(5):
+        xb = np.roll(L.x_bits, 7 * i, axis=0).copy()
+        lg = gen.make_logits(cfg, xb)
+        out = L.nan_bf16(cfg.T, cfg.H)
+        L.ctx.moe_fused_forward(bits_to_dev(xb), torch.from_numpy(lg).to(DEV), L.w_gate, L.w_up, L.w_down, out, ws)
+        torch.cuda.synchronize()
+        want.append(dev_to_bits(out))
+        xs.append(torch.from_numpy(xb.view(np.int16)).pin_memory())
+        lgs.append(torch.from_numpy(lg).pin_memory())
+        outs.append(torch.zeros((cfg.T, cfg.H), dtype=torch.int16).pin_memory())
+    for i in range(5):
+        L.ctx.moe_fused_forward_host_pipelined(xs[i], lgs[i], L.w_gate, L.w_up, L.w_down, outs[i], ws)
+    L.ctx.moe_host_pipeline_flush()
+    torch.cuda.synchronize()
+    for i in range(5):
+        assert np.array_equal(outs[i].numpy().view(np.uint16), want[i]), f"step {i}"
+    L.check_device_status()
+
+
 def test_pacing_points_are_bitwise_identical():
     """Store pacing reorders stores in time only: all 20 sweep points give the same bits."""
     cfg = gen.MoEConfig("pace", T=900, H=512, F=768, E=4, k=2, seed=31, router="xWr")
