@@ -297,6 +297,27 @@ def main():
     ctx.moe_set_kernel_timing(False)
     kernel_ms = [float(np.mean([s[i] for s in per_step_kernel])) for i in range(len(binding.KERNEL_NAMES))]
 
+    # per-step statistics with one event pair per step (the paper reports medians of 20 trials, Sec. 5.1); small
+    # layers whose working set fits L2 are also timed cold, a 512 MB memset between steps evicting L2
+    def per_step(flush):
+        scrub = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if flush else None
+        times = []
+        for _ in range(args.steps):
+            if flush:
+                scrub.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            step()
+            b.record(stream)
+            b.synchronize()
+            times.append(a.elapsed_time(b))
+        return {"median_ms": statistics.median(times), "min_ms": min(times), "max_ms": max(times)}
+
+    step_stats = {"warm": per_step(False)}
+    weights_bytes = 6 * cfg.E * cfg.H * cfg.F
+    if weights_bytes < (256 << 20) or cfg.T <= 256:
+        step_stats["cold_l2_flushed"] = per_step(True)
+
     ffn_trace = None
     if args.trace:
         ttn = binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule, dep_lead_D=args.lead,
@@ -414,7 +435,7 @@ def main():
                 "api": "moe_fused_forward_host_pipelined + moe_host_pipeline_flush (two staging slots)",
                 "serial_ms_per_step": e2e_serial_ms / args.steps,
                 "serial_value": tokens / (e2e_serial_ms / args.steps * 1e-3)},
-        "gpu_launches": launches, "clocks": clocks, "tuning": [args.burst, args.mode, args.ik],
+        "per_step": step_stats, "gpu_launches": launches, "clocks": clocks, "tuning": [args.burst, args.mode, args.ik],
         "schedule": {"schedule": args.schedule, "lead_D": args.lead, "one_launch": one_launch},
     }
     if ffn_trace is not None:
