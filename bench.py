@@ -170,6 +170,8 @@ def main():
     ap.add_argument("--schedule", type=int, default=0, help="0 Expert-Wave order, 1 interleaved order (Algorithm 1)")
     ap.add_argument("--lead", type=int, default=0, help="schedule 1: row lead D (0 = the anti-starvation knee)")
     ap.add_argument("--one-launch", action="store_true", help="schedule 0 as one launch with ready counters")
+    ap.add_argument("--pairs", choices=["auto", "on", "off"], default="auto",
+                    help="CTA-pair (cta_group::2) kernel: auto = for layers with many rows per expert")
     ap.add_argument("--sweep", action="store_true", help="store-pacing sweep (20 points) instead of the bench line")
     ap.add_argument("--probe-mma", action="store_true",
                     help="print SM clocks per tcgen05.mma for several tile shapes (tensor-pipe calibration) and exit")
@@ -256,7 +258,7 @@ def main():
         run_sweep(args, cfg, ctx, binding, (x, d_logits, w_gate, w_up, w_down, out, ws), timed, rank)
         return
 
-    dbg = 2 if args.one_launch else 0
+    dbg = (2 if args.one_launch else 0) | {"auto": 0, "on": 8, "off": 16}[args.pairs]
     tuning = binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule, dep_lead_D=args.lead,
                                  debug_flags=dbg)
     step = lambda: ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tuning)

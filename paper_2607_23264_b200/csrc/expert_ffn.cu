@@ -26,6 +26,7 @@
 //      row-major Linear-1 and Linear-2 tile lists (row = one 128-row block) and emits the Linear-2 tile only
 //      while Linear-1 leads by D rows, else the next Linear-1 tile.  One launch; a Linear-2 tile waits (bounded)
 //      until all Linear-1 tiles of its row have published their h rows.
+// Layers whose experts hold many rows run the CTA-pair variant further down (256-row tiles, cta_group::2).
 #include <cuda_bf16.h>
 
 #include <climits>
@@ -173,9 +174,10 @@ __device__ __forceinline__ void report_timeout(const FfnParams& p, int role) {
 }
 
 // Hold the epilogue until the MMA warp has issued `ik` more K-blocks than at `start`, or cannot advance.
-__device__ __forceinline__ void pace_gap(SharedTail* st, uint32_t start, int ik) {
+__device__ __forceinline__ void pace_gap(volatile uint32_t* progress, volatile int* idle, volatile int* aborting,
+                                         uint32_t start, int ik) {
   for (int spin = 0; spin < (1 << 16); ++spin) {
-    if (st->mma_progress - start >= static_cast<uint32_t>(ik) || st->mma_idle || st->abort_flag) return;
+    if (*progress - start >= static_cast<uint32_t>(ik) || *idle || *aborting) return;
     __nanosleep(64);
   }
 }
@@ -202,14 +204,15 @@ __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target,
 // Drain one finished accumulator: rows of this thread's TMEM lane, kGated ? silu(g)*u of 128 columns
 // : 256 plain columns, written as bf16 with 16-byte stores masked to the expert's rows and to N.
 template <bool kGated>
-__device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams& p, SharedTail* st, uint32_t t_addr,
-                                                  int row, long long* w_gap) {
+__device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams& p, uint32_t t_addr, int row,
+                                                  long long* w_gap, volatile uint32_t* progress, volatile int* idle,
+                                                  volatile int* aborting) {
   const PhaseDesc& d = p.ph[kGated ? 0 : 1];
   const bool row_ok = row < t.row_end;
   __nv_bfloat16* out_row = d.out + static_cast<size_t>(row) * d.N + t.n0;
   constexpr int kChunks = kGated ? (128 / kChunkCols) : (BN_ACC / kChunkCols);
   int in_burst = 0;
-  uint32_t gap_start = st->mma_progress;
+  uint32_t gap_start = *progress;
 #pragma unroll 1
   for (int c = 0; c < kChunks; ++c) {
     uint32_t v[32];
@@ -254,9 +257,9 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
     }
     if (p.mode == 1 && ++in_burst >= p.burst && c + 1 < kChunks) {
       const long long t_gap = clock64();
-      pace_gap(st, gap_start, p.ik);
+      pace_gap(progress, idle, aborting, gap_start, p.ik);
       *w_gap += clock64() - t_gap;
-      gap_start = st->mma_progress;
+      gap_start = *progress;
       in_burst = 0;
     }
   }
@@ -509,8 +512,10 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       const long long t_store = clock64();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               static_cast<uint32_t>(acc * BN_ACC);
-      if (t.phase == 0) drain_accumulator<true>(t, p, st, t_addr, t.row0 + r_in_tile, &w_gap);
-      else drain_accumulator<false>(t, p, st, t_addr, t.row0 + r_in_tile, &w_gap);
+      if (t.phase == 0)
+        drain_accumulator<true>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle, abort_flag);
+      else
+        drain_accumulator<false>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle, abort_flag);
       ptx::tc_fence_before_sync();
       if (chained && t.phase == 0) {
         // publish this warp's 32 rows x 128 columns of h to the Linear-2 tiles of the block
@@ -556,6 +561,253 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       p.sched[1] = 0;
     }
     __threadfence();
+  }
+}
+
+
+// ------------------------------------------------------------------------------------------------------------
+// CTA-pair variant for layers whose experts hold many rows: a cluster of two CTAs computes a 256-row x 256-column
+// tile with tcgen05.mma.cta_group::2.  Each CTA loads its own 128 rows of A and one 128-row weight box (for
+// Linear-1 the leader holds the gate box, its peer the up box), so a stage is 32 KiB per CTA instead of 48 and
+// six stages fit; the leader's MMA thread issues for both, reading the peer's operands from the peer's shared
+// memory, and each CTA's epilogue drains its own 128 accumulator rows.  Static schedule: pair c takes tiles
+// c, c + pairs, ... in the order expert -> N block -> 256-row block (fastest); one GEMM per launch.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = kABytes + kBHalfBytes;   // 32 KiB per CTA
+
+struct PairTail {
+  uint64_t full[kPairStages];       // used in the leader: its own expect_tx arrival + the bytes of both CTAs
+  uint64_t empty[kPairStages];      // one per CTA, both arrived on by the leader's multicast commit
+  uint64_t tmem_full[2];            // one per CTA, multicast commit
+  uint64_t tmem_empty[2];           // used in the leader: 4 epilogue warps of each CTA
+  uint32_t tmem_base;
+  volatile int abort_flag;
+  volatile uint32_t mma_progress;
+  volatile int mma_idle;
+  int32_t pair_prefix[kMaxExperts + 1];   // exclusive prefix of 256-row blocks per expert
+};
+constexpr size_t kPairSmemBytes = 1024 + static_cast<size_t>(kPairStages) * kPairStageBytes + sizeof(PairTail);
+
+__device__ __forceinline__ Tile decode_pair_tile(int tile, int phase, uint32_t rank, const PairTail* st,
+                                                 const FfnParams& p) {
+  const PhaseDesc& d = p.ph[phase];
+  const int e = find_expert([&](int i) { return st->pair_prefix[i]; }, tile / d.n_blocks, p.E);
+  const int pb = st->pair_prefix[e + 1] - st->pair_prefix[e];
+  const int local = tile - d.n_blocks * st->pair_prefix[e];
+  const int n_blk = local / pb;
+  const int pair_row = local - n_blk * pb;
+  Tile t;
+  t.phase = phase;
+  t.row0 = p.offsets[e] + pair_row * 2 * BM + static_cast<int>(rank) * BM;   // this CTA's 128 rows
+  t.row_end = p.offsets[e + 1];
+  t.n0 = n_blk * d.out_cols_per_tile;
+  t.w_row0 = e * d.N + t.n0;
+  t.block = 0;
+  return t;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
+                       const __grid_constant__ CUtensorMap tm_b1, const FfnParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+  unsigned char* stage_base = smem_raw + pad;
+  const uint32_t stage_u32 = raw + pad;
+  PairTail* st = reinterpret_cast<PairTail*>(stage_base + static_cast<size_t>(kPairStages) * kPairStageBytes);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t rank = ptx::cluster_ctarank();            // 0 = leader (issues the MMAs), 1 = peer
+  const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+  const int phase = p.phase_lo;
+  const PhaseDesc& d = p.ph[phase];
+
+  if (tid == 0) {
+    for (int s = 0; s < kPairStages; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&st->full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&st->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(ptx::smem_u32(&st->tmem_full[a]), 1);
+      ptx::mbar_init(ptx::smem_u32(&st->tmem_empty[a]), 8);   // four epilogue warps in each CTA of the pair
+    }
+    st->abort_flag = 0;
+    st->mma_progress = 0;
+    st->mma_idle = 0;
+    st->pair_prefix[0] = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async_smem();
+  }
+  if (warp == 0) {
+    int32_t run = 0;
+    for (int base = 0; base < p.E; base += 32) {
+      const int e = base + lane;
+      int32_t v = 0;
+      if (e < p.E) v = (p.offsets[e + 1] - p.offsets[e] + 2 * BM - 1) / (2 * BM);
+      int32_t incl = v;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += o;
+      }
+      if (e < p.E) st->pair_prefix[e + 1] = run + incl;
+      run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tm_a);
+      ptx::prefetch_tensormap(&tm_b0);
+      ptx::prefetch_tensormap(&tm_b1);
+    }
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(&st->tmem_base), kTmemCols);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::cluster_sync();            // both CTAs' barriers exist before anything signals across the pair
+  ptx::tc_fence_after_sync();
+
+  const uint32_t tmem_base = st->tmem_base;
+  const int total_tiles = st->pair_prefix[p.E] * d.n_blocks;
+  volatile int* abort_flag = &st->abort_flag;
+  const CUtensorMap* mb = (rank == 0) ? &tm_b0 : &tm_b1;      // this CTA's half of the 256 weight rows
+  const int b_shift = (rank == 0) ? 0 : d.b1_row_shift;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      long long w_empty = 0;
+      const long long t_begin = clock64();
+      for (int tile = pair; ok && tile < total_tiles; tile += pairs) {
+        const Tile t = decode_pair_tile(tile, phase, rank, st, p);
+        for (int kb = 0; kb < d.k_blocks; ++kb) {
+          if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->empty[stage]), ph ^ 1u, abort_flag, &w_empty)) {
+            report_timeout(p, 1);
+            ok = false;
+            break;
+          }
+          const uint32_t full_local = ptx::smem_u32(&st->full[stage]);
+          const uint32_t full_leader = ptx::map_to_cta(full_local, 0);
+          const uint32_t sa = stage_u32 + stage * kPairStageBytes;
+          if (rank == 0) ptx::mbar_expect_tx(full_local, 2 * kPairStageBytes);   // the bytes of both CTAs
+          ptx::tma_load_2d_pair(sa, &tm_a, full_leader, kb * BK, t.row0);
+          ptx::tma_load_2d_pair(sa + kABytes, mb, full_leader, kb * BK, t.w_row0 + b_shift);
+          if (++stage == kPairStages) { stage = 0; ph ^= 1u; }
+        }
+      }
+      if (p.trace) {
+        p.trace[blockIdx.x * kMoeTraceFields + 0] = static_cast<unsigned long long>(clock64() - t_begin);
+        p.trace[blockIdx.x * kMoeTraceFields + 1] = static_cast<unsigned long long>(w_empty);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(2 * BM, BN_ACC);
+      int stage = 0;
+      uint32_t ph = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      uint32_t progress = 0;
+      bool ok = true;
+      long long w_full = 0, w_tmem = 0;
+      unsigned long long n_tiles = 0;
+      for (int tile = pair; ok && tile < total_tiles; tile += pairs) {
+        st->mma_idle = 1;
+        if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, &w_tmem)) {
+          report_timeout(p, 2);
+          break;
+        }
+        st->mma_idle = 0;
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN_ACC);
+        for (int kb = 0; kb < d.k_blocks; ++kb) {
+          if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), ph, abort_flag, &w_full)) {
+            report_timeout(p, 3);
+            ok = false;
+            break;
+          }
+          ptx::tc_fence_after_sync();
+          const uint32_t sa = stage_u32 + stage * kPairStageBytes;
+          const uint64_t a_desc = ptx::smem_desc_sw128(sa);
+          const uint64_t b_desc = ptx::smem_desc_sw128(sa + kABytes);
+#pragma unroll
+          for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
+            ptx::tc_mma_bf16_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * k4),
+                                  b_desc + static_cast<uint64_t>(2 * k4), idesc, (kb | k4) != 0 ? 1u : 0u);
+          }
+          ptx::tc_commit_pair(ptx::smem_u32(&st->empty[stage]), 3);    // frees the stage in both CTAs
+          st->mma_progress = ++progress;
+          if (++stage == kPairStages) { stage = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::tc_commit_pair(ptx::smem_u32(&st->tmem_full[acc]), 3);    // accumulator complete, both CTAs
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+        ++n_tiles;
+      }
+      st->mma_idle = 1;
+      if (p.trace) {
+        p.trace[blockIdx.x * kMoeTraceFields + 2] = static_cast<unsigned long long>(w_full);
+        p.trace[blockIdx.x * kMoeTraceFields + 3] = static_cast<unsigned long long>(w_tmem);
+        p.trace[blockIdx.x * kMoeTraceFields + 6] = n_tiles;
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
+    const int quarter = warp & 3;
+    const int r_in_tile = quarter * 32 + lane;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    long long w_acc = 0, busy = 0, w_gap = 0;
+    const uint32_t empty_leader0 = ptx::map_to_cta(ptx::smem_u32(&st->tmem_empty[0]), 0);
+    const uint32_t empty_leader1 = ptx::map_to_cta(ptx::smem_u32(&st->tmem_empty[1]), 0);
+    for (int tile = pair; tile < total_tiles; tile += pairs) {
+      const Tile t = decode_pair_tile(tile, phase, rank, st, p);
+      if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, &w_acc)) {
+        if (lane == 0) report_timeout(p, 4);
+        break;
+      }
+      ptx::tc_fence_after_sync();
+      const long long t_store = clock64();
+      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                              static_cast<uint32_t>(acc * BN_ACC);
+      // pacing needs the MMA warp's progress counter, which lives in the leader: the peer drains unpaced
+      FfnParams q = p;
+      if (rank != 0) q.mode = 0;
+      if (phase == 0)
+        drain_accumulator<true>(t, q, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle, abort_flag);
+      else
+        drain_accumulator<false>(t, q, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle, abort_flag);
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(acc ? empty_leader1 : empty_leader0);
+      busy += clock64() - t_store;
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (p.trace && warp == 2 && lane == 0) {
+      p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
+      p.trace[blockIdx.x * kMoeTraceFields + 5] = static_cast<unsigned long long>(busy);
+      p.trace[blockIdx.x * kMoeTraceFields + 7] = static_cast<unsigned long long>(w_gap);
+    }
+  }
+
+  __syncthreads();
+  if (st->abort_flag) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  ptx::cluster_sync();            // the peer's shared memory and barriers stay alive until both CTAs are done
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 
@@ -638,10 +890,50 @@ extern "C" moe_status moe_probe_mma_cycles(moe_ctx* ctx, int32_t M, int32_t N, i
 
 namespace moe {
 
-cudaError_t prepare_expert_ffn(moe_ctx*) {
-  return cudaFuncSetAttribute(expert_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              static_cast<int>(kSmemBytes));
+cudaError_t prepare_expert_ffn(moe_ctx* ctx) {
+  cudaError_t e = cudaFuncSetAttribute(expert_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(kSmemBytes));
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(expert_ffn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(kPairSmemBytes));
+  if (e != cudaSuccess) return e;
+  // how many CTA pairs can be resident at once (an SM left over in a GPC cannot join a pair)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * (ctx->num_sms / 2));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kPairSmemBytes;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int clusters = 0;
+  e = cudaOccupancyMaxActiveClusters(&clusters, expert_ffn_pair_kernel, &cfg);
+  if (e != cudaSuccess) return e;
+  ctx->max_pairs = clusters < ctx->num_sms / 2 ? clusters : ctx->num_sms / 2;
+  return cudaSuccess;
 }
+
+namespace {
+cudaError_t launch_pair(moe_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
+                        const FfnParams& p, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * ctx->max_pairs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kPairSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, expert_ffn_pair_kernel, a, b0, b1, p);
+}
+}  // namespace
 
 moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* offsets, const void* w_gate,
                              const void* w_up, const void* w_down, void* h_ws, void* y_perm,
@@ -677,12 +969,32 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
   p.withhold_ready = (tn.debug_flags & 4) != 0;
   p.wait_budget = p.withhold_ready ? 200000000LL : ptx::kWaitClockBudget;   // the drill gives up after ~0.1 s
   const bool trace = (tn.debug_flags & 1) != 0;
+  if (trace && cudaMemsetAsync(ctx->d_trace, 0, static_cast<size_t>(2) * ctx->num_sms * kMoeTraceFields * 8, stream) !=
+                   cudaSuccess)
+    return MOE_ERR_CUDA;   // roles that do not run in a variant (the peer's MMA warp) leave zeros, not stale counts
   // Launch-latency-bound layers (every tile fits in about one wave of CTAs) run both GEMMs in one launch.
   const long long max_blocks = static_cast<long long>(R / 128) + s.E;
   const bool tiny = max_blocks * (p.ph[0].n_blocks + p.ph[1].n_blocks) <= 2LL * grid;
   const bool one_launch = tn.schedule == 1 || (tn.debug_flags & 6) != 0 || tiny;
 
-  if (one_launch) {
+  // CTA pairs (256-row tiles) pay off when experts hold many rows; single-block experts would waste the peer.
+  const bool dense = R / static_cast<uint64_t>(s.E) >= 1024;
+  const bool pairs = !one_launch && ctx->max_pairs > 0 && ((tn.debug_flags & 8) != 0 || (dense && (tn.debug_flags & 16) == 0));
+  if (pairs) {
+    p.trace = trace ? ctx->d_trace : nullptr;
+    p.phase_lo = 0;
+    p.phase_hi = 1;
+    p.kernel_id = 4;
+    if (launch_pair(ctx, tm_x, tm_wg, tm_wu, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+    moe_mark(ctx, 5, stream);
+    p.trace = trace ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
+    p.phase_lo = 1;
+    p.phase_hi = 2;
+    p.kernel_id = 5;
+    if (launch_pair(ctx, tm_h, tm_wd, tm_wd, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+    moe_mark(ctx, 6, stream);
+    ctx->last_launches += 2;
+  } else if (one_launch) {
     p.phase_lo = 0;
     p.phase_hi = 2;
     p.sched = ctx->d_sched;

@@ -26,7 +26,7 @@ moe_status check_tuning(const moe_tuning* t) {
   if (t->interleave_mode != 0 && t->interleave_mode != 1) return MOE_ERR_INVALID_ARG;
   if (!(t->interleave_k == 1 || t->interleave_k == 2 || t->interleave_k == 4)) return MOE_ERR_INVALID_ARG;
   if (t->schedule != 0 && t->schedule != 1) return MOE_ERR_UNSUPPORTED;
-  if (t->dep_lead_D < 0 || (t->schedule == 0 && t->dep_lead_D != 0) || (t->debug_flags & ~7) != 0)
+  if (t->dep_lead_D < 0 || (t->schedule == 0 && t->dep_lead_D != 0) || (t->debug_flags & ~31) != 0)
     return MOE_ERR_INVALID_ARG;
   return MOE_OK;
 }

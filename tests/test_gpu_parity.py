@@ -236,6 +236,35 @@ def test_schedules_are_bitwise_identical(cfg):
     L.check_device_status()
 
 
+@pytest.mark.parametrize("cfg", [SMALL[1], SMALL[3], SMALL[5], SMALL[7],
+                                 gen.MoEConfig("pairs", T=3000, H=512, F=640, E=3, k=2, seed=81, router="xWr")],
+                         ids=lambda c: c.name)
+def test_cta_pair_kernel_matches_single_cta_kernel(cfg):
+    """The cta_group::2 variant (256-row tiles over a cluster of two CTAs), forced on, gives the same bits as the
+    single-CTA kernel, ragged and empty experts and odd block counts included."""
+    L = Layer(cfg)
+    lay = L.ctx.workspace_layout()
+    ws = torch.empty(lay["total"], dtype=torch.uint8, device=DEV)
+    base = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, base, ws,
+                            tuning=binding.make_tuning(1, 0, 1, debug_flags=16))       # single-CTA kernel
+    torch.cuda.synchronize()
+    assert_out_close(dev_bf16_to_f64(base), oracle_for(L)["out"], f"out[{cfg.name}]")
+    R = cfg.R
+    h_base = ws[lay["h"]:lay["h"] + R * cfg.F * 2].clone()
+    y_base = ws[lay["y_perm"]:lay["y_perm"] + R * cfg.H * 2].clone()
+    for tn in (binding.make_tuning(1, 0, 1, debug_flags=8), binding.make_tuning(2, 1, 1, debug_flags=8 | 1)):
+        ws[lay["h"]:lay["h"] + R * cfg.F * 2].fill_(0xFF)
+        ws[lay["y_perm"]:lay["y_perm"] + R * cfg.H * 2].fill_(0xFF)
+        out = L.nan_bf16(cfg.T, cfg.H)
+        L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws, tuning=tn)
+        torch.cuda.synchronize()
+        L.check_device_status()
+        assert torch.equal(ws[lay["h"]:lay["h"] + R * cfg.F * 2], h_base), "h"
+        assert torch.equal(ws[lay["y_perm"]:lay["y_perm"] + R * cfg.H * 2], y_base), "y_perm"
+        assert torch.equal(out.view(torch.int16), base.view(torch.int16))
+
+
 def test_zero_tokens_is_a_no_op():
     ctx = binding.Context(0, 128, 128, 4, 2)
     counts = torch.full((4,), -1, dtype=torch.int32, device=DEV)
@@ -288,7 +317,7 @@ def test_ffn_trace_and_kernel_times():
     L.ctx.moe_set_kernel_timing(True)
     out2 = L.nan_bf16(cfg.T, cfg.H)
     L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out2, ws,
-                            tuning=binding.make_tuning(1, 1, 2, debug_flags=1))
+                            tuning=binding.make_tuning(1, 1, 2, debug_flags=1 | 16))     # single-CTA kernel, traced
     ms = L.ctx.moe_get_kernel_times()
     L.ctx.moe_set_kernel_timing(False)
     assert len(ms) == 7 and all(0 < v < 100 for v in ms)
@@ -300,6 +329,14 @@ def test_ffn_trace_and_kernel_times():
     assert tr[0, :, 6].sum() == mblocks * ((cfg.F + 127) // 128)
     assert tr[1, :, 6].sum() == mblocks * ((cfg.H + 255) // 256)
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16)), "tracing must not change values"
+    # the CTA-pair kernel works on 256-row blocks; only the leader of a pair counts tiles
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out2, ws,
+                            tuning=binding.make_tuning(1, 0, 1, debug_flags=1 | 8))
+    tr = L.ctx.moe_get_ffn_trace()
+    pblocks = int(((counts + 255) // 256).sum())
+    assert tr[0, :, 6].sum() == pblocks * ((cfg.F + 127) // 128)
+    assert tr[1, :, 6].sum() == pblocks * ((cfg.H + 255) // 256)
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
     L.check_device_status()
 
 
