@@ -31,10 +31,10 @@ from paper_2607_23264_b200 import inputs as gen  # noqa: E402
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one expert_gemm_kernel<true> (Linear-1) launch on the
-# C2 workload: the ncu capture of the two-expert case P1 (504.1 MB read + 109.2 MB written, see
+# C2 workload: the ncu capture of the two-expert case P1 (511.7 MB read + 109.9 MB written, see
 # profiles/expert_gemm_P1_ncu_full.md) scaled by 4, since DRAM traffic is per expert and C2 has four times
 # P1's experts at the same rows per expert.  C3: one-pass DRAM counters on the full layer (same file).
-LINEAR1_DRAM_TRAFFIC_BYTES = {"C2": 4 * (504_129_280 + 109_233_664), "C3": 11_263_676_672 + 136_142_592}
+LINEAR1_DRAM_TRAFFIC_BYTES = {"C2": 4 * (511_678_208 + 109_886_720), "C3": 11_263_676_672 + 136_142_592}
 
 
 def load_peaks():
@@ -399,8 +399,9 @@ def main():
         l1_bytes, l2_bytes = l1_bytes + l2_bytes, 0
     l1_gbs = l1_bytes / (kernel_ms[4] * 1e-3) / 1e9
     l2_gbs = 0.0 if one_launch else l2_bytes / (kernel_ms[5] * 1e-3) / 1e9
+    pair_kernel = not one_launch and (args.pairs == "on" or (args.pairs == "auto" and cfg.R // cfg.E >= 1024))
     gemm_name = ("expert_ffn_kernel (Linear-1 + SiLU*mul + Linear-2, one launch)" if one_launch
-                 else "expert_ffn_kernel, Linear-1 + SiLU*mul launch")
+                 else ("expert_ffn_pair_kernel" if pair_kernel else "expert_ffn_kernel") + ", Linear-1 + SiLU*mul launch")
     # the roofline that binds Linear-1: tensor time at the measured GEMM peak vs HBM time at the measured copy rate
     t_tensor = l1_flops / (peak_tf * 1e12)
     t_hbm = l1_bytes / (peak_hbm * 1e9)
