@@ -175,6 +175,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="store-pacing sweep (20 points) instead of the bench line")
     ap.add_argument("--probe-mma", action="store_true",
                     help="print SM clocks per tcgen05.mma for several tile shapes (tensor-pipe calibration) and exit")
+    ap.add_argument("--fp8", action="store_true",
+                    help="time the FP8 (E4M3, W8A8) variant of the layer instead (weights quantised on the GPU first)")
     ap.add_argument("--xstage-probe", action="store_true",
                     help="run the burst/gap store microbenchmark on local HBM, print the rows and the calibration, exit")
     ap.add_argument("--trace", action="store_true",
@@ -256,6 +258,9 @@ def main():
 
     if args.sweep:
         run_sweep(args, cfg, ctx, binding, (x, d_logits, w_gate, w_up, w_down, out, ws), timed, rank)
+        return
+    if args.fp8:
+        run_fp8(args, cfg, ctx, binding, (x, d_logits, w_gate, w_up, w_down, out), timed, rank, world, dev)
         return
 
     dbg = (2 if args.one_launch else 0) | {"auto": 0, "on": 8, "off": 16}[args.pairs]
@@ -455,6 +460,55 @@ def main():
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
+    """The FP8 (E4M3, W8A8) variant: same layer, same algorithmic flops, experts in E4M3 with row scales."""
+    import torch
+    x, d_logits, w_gate, w_up, w_down, out = bufs
+    wq = []
+    for w in (w_gate, w_up, w_down):
+        E, r, c = w.shape
+        codes = torch.empty((E * r, c), dtype=torch.uint8, device=dev)
+        scales = torch.empty((E * r,), dtype=torch.float32, device=dev)
+        ctx.moe_quantize_rows(w.view(E * r, c), E * r, c, codes, scales)
+        wq += [codes, scales]
+    torch.cuda.synchronize()
+    del w_gate, w_up, w_down
+    ws = torch.empty(ctx.workspace_layout_fp8()["total"], dtype=torch.uint8, device=dev)
+    tn = binding.make_tuning(args.burst, args.mode, args.ik, debug_flags={"auto": 0, "on": 8, "off": 16}[args.pairs])
+    step = lambda: ctx.moe_fused_forward_fp8(x, d_logits, *wq, out, ws, tuning=tn)
+    ms = timed(step, args.steps, args.warmup) / args.steps
+    ctx.moe_set_kernel_timing(True)
+    per = []
+    for _ in range(args.steps):
+        step()
+        per.append(ctx.moe_get_kernel_times())
+    ctx.moe_set_kernel_timing(False)
+    km = [float(np.mean([p[i] for p in per])) for i in range(len(binding.KERNEL_NAMES))]
+    code, detail = ctx.moe_last_device_status()
+    if code != 0:
+        raise RuntimeError(f"device status {code} detail {detail:#x}")
+    if rank != 0:
+        return
+    peaks, kind = load_peaks()
+    peak = 2.0 * float(peaks["bf16_tflops"])      # E4M3 runs at twice the bf16 rate on this part (4.5 vs 2.25 PFLOP/s nominal)
+    R = cfg.R
+    l1_tf = 4 * R * cfg.H * cfg.F / (km[4] * 1e-3) / 1e12
+    tflops = cfg.flops * world / (ms * 1e-3) / 1e12
+    line = {
+        "metric": "fused MoE fwd tokens/s", "variant": "fp8 (E4M3 W8A8, per-row scales)", "value": cfg.T * world / (ms * 1e-3),
+        "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3", "data": "synthetic",
+        "config": workload_config(cfg, world), "tflops": tflops, "frac_fp8_peak": tflops / world / peak,
+        "kernels_ms": {"routing": km[0] + km[1] + km[2], "quantize_x+dispatch": km[3], "linear1": km[4],
+                       "quantize_h+linear2": km[5], "combine": km[6]},
+        "roofline": {"kernel": "expert FFN Linear-1 launch, E4M3 operands", "bound": "tensor", "achieved": l1_tf,
+                     "peak": peak, "unit": "TFLOP/s", "frac": l1_tf / peak, "traffic": None,
+                     "peak_source": f"2 x {kind} bf16_tflops (burst): nominal fp8 / bf16 ratio"},
+        "gpu_launches": ctx.moe_last_launch_count() * args.steps,
+    }
+    print(json.dumps(line), flush=True)
 
 
 def run_xstage_probe(dev):

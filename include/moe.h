@@ -210,6 +210,66 @@ moe_status moe_fused_forward_host(moe_ctx* ctx, const void* x_host, const float*
                                   void* out_host, void* workspace, size_t workspace_bytes,
                                   const moe_tuning* tuning, void* stream);
 
+/* ------------------------------------------------------------------------------------------------------------
+ * FP8 (W8A8) variant of the expert FFN.  The paper's kernels run W8A8 / W4A8 (Sec. 5.3) without saying how values
+ * are scaled; the scheme here needs no scaling inside the MMA loop: E4M3 storage (round to nearest even, saturating
+ * at 448), one fp32 scale per row of every quantised matrix (per token row for x and h, per output channel for the
+ * weights), scale = amax(|row|) / 448 (1 for an all-zero row), code = convert(fp32(v) / scale); a GEMM multiplies
+ * codes with fp32 accumulation and its epilogue applies row scale x column scale.  h is produced in bf16, then
+ * quantised row by row for Linear-2; y_perm and out stay bf16.  Routing, combine and all plan arrays are those of
+ * the bf16 layer.  H and F must be multiples of 128.
+ * ------------------------------------------------------------------------------------------------------------ */
+
+/* in_bf16 [rows, cols] bf16 (cols a multiple of 8) -> codes [rows, cols] E4M3 bytes, scales [rows] fp32. */
+moe_status moe_quantize_rows(moe_ctx* ctx, const void* in_bf16, int64_t rows, int32_t cols, void* codes,
+                             float* scales, void* stream);
+
+/* xq_perm[inv_perm[t*k+j], :] = xq[t, :] (E4M3 bytes, [T,H] -> [R,H]) and sx_perm[inv_perm[t*k+j]] = sx[t]. */
+moe_status moe_dispatch_fp8(moe_ctx* ctx, const void* xq, const float* sx, const int32_t* inv_perm, void* xq_perm,
+                            float* sx_perm, void* stream);
+
+typedef struct {
+  const void* xq_perm;      /* E4M3 [R,H] expert-contiguous rows */
+  const float* sx_perm;     /* fp32 [R]   their scales */
+  const int32_t* offsets;   /* int32 [E+1] */
+  const void* wq_gate;      /* E4M3 [E,F,H] */
+  const float* s_gate;      /* fp32 [E,F] */
+  const void* wq_up;        /* E4M3 [E,F,H] */
+  const float* s_up;        /* fp32 [E,F] */
+  const void* wq_down;      /* E4M3 [E,H,F] */
+  const float* s_down;      /* fp32 [E,H] */
+  void* h_ws;               /* out: bf16 [R,F]  silu(g)*u */
+  void* hq_ws;              /* out: E4M3 [R,F]  its quantised copy (Linear-2 input) */
+  float* sh_ws;             /* out: fp32 [R]    row scales of hq */
+  void* y_perm;             /* out: bf16 [R,H] */
+} moe_fp8_ffn_args;
+
+/* Linear-1 (E4M3 x E4M3 -> fp32, scales, SiLU*mul) -> h bf16 -> row quantisation -> Linear-2 -> y_perm bf16.
+ * Three launches; Expert-Wave order only (tuning->schedule must be 0). */
+moe_status moe_expert_ffn_fp8(moe_ctx* ctx, const moe_fp8_ffn_args* args, const moe_tuning* tuning, void* stream);
+
+/* Byte offsets of the workspace slices of moe_fused_forward_fp8 (256-byte aligned). */
+typedef struct {
+  size_t topk_ids, topk_w, counts, offsets, perm, inv_perm;   /* as in moe_workspace_layout */
+  size_t xq;         /* E4M3 [T,H] */
+  size_t sx;         /* fp32 [T]   */
+  size_t xq_perm;    /* E4M3 [R,H] */
+  size_t sx_perm;    /* fp32 [R]   */
+  size_t h;          /* bf16 [R,F] */
+  size_t hq;         /* E4M3 [R,F] */
+  size_t sh;         /* fp32 [R]   */
+  size_t y_perm;     /* bf16 [R,H] */
+  size_t total;
+} moe_workspace_layout_fp8;
+moe_status moe_get_workspace_layout_fp8(const moe_shape* shape, moe_workspace_layout_fp8* out_layout);
+
+/* The whole layer with FP8 experts on one stream: plan_routing, quantize x, dispatch_fp8, expert_ffn_fp8, combine.
+ * x [T,H] bf16 and logits as in moe_fused_forward; weights pre-quantised (moe_quantize_rows over their rows). */
+moe_status moe_fused_forward_fp8(moe_ctx* ctx, const void* x, const float* logits, const void* wq_gate,
+                                 const float* s_gate, const void* wq_up, const float* s_up, const void* wq_down,
+                                 const float* s_down, void* out, void* workspace, size_t workspace_bytes,
+                                 const moe_tuning* tuning, void* stream);
+
 /*
  * The host-buffer call as a two-deep pipeline, for callers that run step after step (serving): consecutive calls
  * alternate between two staging slots, the input copy of call i+1 runs on an internal copy stream while call i

@@ -24,7 +24,8 @@ EXPORTS = (
     "moe_plan_routing", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_fused_forward",
     "moe_fused_forward_host", "moe_last_device_status", "moe_last_launch_count", "moe_set_kernel_timing",
     "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace", "moe_probe_mma_cycles",
-    "moe_get_ffn_order", "moe_fused_forward_host_pipelined", "moe_host_pipeline_flush",
+    "moe_get_ffn_order", "moe_fused_forward_host_pipelined", "moe_host_pipeline_flush", "moe_quantize_rows",
+    "moe_dispatch_fp8", "moe_expert_ffn_fp8", "moe_get_workspace_layout_fp8", "moe_fused_forward_fp8",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -53,6 +54,16 @@ class moe_workspace_layout(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in ("topk_ids", "topk_w", "counts", "offsets", "perm", "inv_perm", "x_perm",
                                           "h", "y_perm", "x_stage", "logits_stage", "out_stage", "x_stage_b",
                                           "logits_stage_b", "out_stage_b", "total")]
+
+
+class moe_fp8_ffn_args(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("xq_perm", "sx_perm", "offsets", "wq_gate", "s_gate", "wq_up", "s_up",
+                                          "wq_down", "s_down", "h_ws", "hq_ws", "sh_ws", "y_perm")]
+
+
+class moe_workspace_layout_fp8(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("topk_ids", "topk_w", "counts", "offsets", "perm", "inv_perm", "xq", "sx",
+                                          "xq_perm", "sx_perm", "h", "hq", "sh", "y_perm", "total")]
 
 
 _lib = None
@@ -86,6 +97,12 @@ def load_library() -> C.CDLL:
     lib.moe_fused_forward_host.argtypes = [vp, vp, f32p, vp, vp, vp, vp, vp, C.c_size_t, C.POINTER(moe_tuning), vp]
     lib.moe_fused_forward_host_pipelined.argtypes = lib.moe_fused_forward_host.argtypes
     lib.moe_host_pipeline_flush.argtypes = [vp, vp]
+    lib.moe_quantize_rows.argtypes = [vp, vp, C.c_int64, C.c_int32, vp, f32p, vp]
+    lib.moe_dispatch_fp8.argtypes = [vp, vp, f32p, i32p, vp, f32p, vp]
+    lib.moe_expert_ffn_fp8.argtypes = [vp, C.POINTER(moe_fp8_ffn_args), C.POINTER(moe_tuning), vp]
+    lib.moe_get_workspace_layout_fp8.argtypes = [C.POINTER(moe_shape), C.POINTER(moe_workspace_layout_fp8)]
+    lib.moe_fused_forward_fp8.argtypes = [vp, vp, f32p, vp, f32p, vp, f32p, vp, f32p, vp, vp, C.c_size_t,
+                                          C.POINTER(moe_tuning), vp]
     lib.moe_last_device_status.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_last_launch_count.argtypes = [vp]
     lib.moe_last_launch_count.restype = C.c_int32
@@ -241,6 +258,35 @@ class Context:
 
     def moe_host_pipeline_flush(self, stream=None):
         _check(self._lib.moe_host_pipeline_flush(self._handle, _stream(stream)), "moe_host_pipeline_flush")
+
+    # ---- FP8 (E4M3, W8A8) variant
+    def workspace_layout_fp8(self) -> dict:
+        L = moe_workspace_layout_fp8()
+        shape = moe_shape(self.T, self.H, self.F, self.E, self.k, 1, 0)
+        _check(self._lib.moe_get_workspace_layout_fp8(C.byref(shape), C.byref(L)), "moe_get_workspace_layout_fp8")
+        return {n: getattr(L, n) for n, _ in moe_workspace_layout_fp8._fields_}
+
+    def moe_quantize_rows(self, in_bf16, rows, cols, codes, scales, stream=None):
+        _check(self._lib.moe_quantize_rows(self._handle, _ptr(in_bf16), rows, cols, _ptr(codes), _ptr(scales),
+                                           _stream(stream)), "moe_quantize_rows")
+
+    def moe_dispatch_fp8(self, xq, sx, inv_perm, xq_perm, sx_perm, stream=None):
+        _check(self._lib.moe_dispatch_fp8(self._handle, _ptr(xq), _ptr(sx), _ptr(inv_perm), _ptr(xq_perm),
+                                          _ptr(sx_perm), _stream(stream)), "moe_dispatch_fp8")
+
+    def moe_expert_ffn_fp8(self, xq_perm, sx_perm, offsets, wq_gate, s_gate, wq_up, s_up, wq_down, s_down, h_ws, hq_ws,
+                           sh_ws, y_perm, tuning=None, stream=None):
+        tensors = (xq_perm, sx_perm, offsets, wq_gate, s_gate, wq_up, s_up, wq_down, s_down, h_ws, hq_ws, sh_ws, y_perm)
+        args = moe_fp8_ffn_args(*[None if t is None else t.data_ptr() for t in tensors])
+        _check(self._lib.moe_expert_ffn_fp8(self._handle, C.byref(args), _tuning_ref(tuning), _stream(stream)),
+               "moe_expert_ffn_fp8")
+
+    def moe_fused_forward_fp8(self, x, logits, wq_gate, s_gate, wq_up, s_up, wq_down, s_down, out, workspace,
+                              tuning=None, stream=None):
+        _check(self._lib.moe_fused_forward_fp8(self._handle, _ptr(x), _ptr(logits), _ptr(wq_gate), _ptr(s_gate),
+                                               _ptr(wq_up), _ptr(s_up), _ptr(wq_down), _ptr(s_down), _ptr(out),
+                                               _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                               _tuning_ref(tuning), _stream(stream)), "moe_fused_forward_fp8")
 
     def moe_last_device_status(self, stream=None):
         code, detail = C.c_int32(0), C.c_int32(0)

@@ -78,6 +78,11 @@ struct PhaseDesc {          // one of the two GEMMs
   int out_cols_per_tile;    // 128 (Linear-1) or 256 (Linear-2)
   int b1_row_shift;         // row offset of the second weight box: 0 (up matrix) or 128 (same matrix)
   __nv_bfloat16* out;       // [R, N]
+  // FP8 (E4M3) operands: fp32 scales applied in the epilogue, out = acc * row_scale[row] * col_scale[weight row];
+  // all nullptr for bf16 operands.  col_scale0 belongs to the first weight box, col_scale1 to the second.
+  const float* row_scale;   // [R]
+  const float* col_scale0;  // [E * N]
+  const float* col_scale1;  // [E * N]
 };
 
 struct FfnParams {
@@ -94,6 +99,8 @@ struct FfnParams {
   int phase_lo, phase_hi;   // GEMMs in this launch: [0,1) Linear-1, [1,2) Linear-2, [0,2) both
   int schedule;             // 0 merged order drawn dynamically, 1 Algorithm 1
   int lead_D;               // Algorithm 1: minimum row lead of Linear-1 over Linear-2 (>= 1)
+  int fp8;                  // operands are E4M3 bytes (128 per swizzle row) instead of bf16 (64 per row)
+  int k_elems;              // K elements per pipeline stage: 64 (bf16) or 128 (E4M3)
   int withhold_ready;       // host-requested failure drill: Linear-1 never publishes its rows (one-launch runs)
   long long wait_budget;    // clocks a cross-CTA wait may last before it gives up
   int kernel_id;
@@ -222,13 +229,35 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
       ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
       ptx::tmem_ld_32x32(t_addr + 128 + c * kChunkCols, u);
       ptx::tmem_ld_wait();
+      if (d.row_scale != nullptr) {
+        const float rs = row_ok ? d.row_scale[row] : 0.f;
+        const int w0 = t.w_row0 + c * kChunkCols;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) o[i] = silu_mul(__uint_as_float(v[i]), __uint_as_float(u[i]));
+        for (int i = 0; i < 32; ++i) {
+          const bool in = t.n0 + c * kChunkCols + i < d.N;
+          const float sg = in ? d.col_scale0[w0 + i] : 0.f, su = in ? d.col_scale1[w0 + i] : 0.f;
+          o[i] = silu_mul(__uint_as_float(v[i]) * (rs * sg), __uint_as_float(u[i]) * (rs * su));
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = silu_mul(__uint_as_float(v[i]), __uint_as_float(u[i]));
+      }
     } else {
       ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
       ptx::tmem_ld_wait();
+      if (d.row_scale != nullptr) {
+        const float rs = row_ok ? d.row_scale[row] : 0.f;
+        // columns 0..127 of the tile come from the first weight box, 128..255 from the second (same matrix)
+        const int w0 = t.w_row0 + c * kChunkCols;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
+        for (int i = 0; i < 32; ++i) {
+          const bool in = t.n0 + c * kChunkCols + i < d.N;
+          o[i] = __uint_as_float(v[i]) * (rs * (in ? d.col_scale0[w0 + i] : 0.f));
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
+      }
     }
     const int col0 = t.n0 + c * kChunkCols;
     if (row_ok) {
@@ -407,9 +436,9 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           const uint32_t full = ptx::smem_u32(&st->full[stage]);
           const uint32_t sa = stage_u32 + stage * kStageBytes;
           ptx::mbar_expect_tx(full, kStageBytes);
-          ptx::tma_load_2d(sa, ma, full, kb * BK, t.row0);
-          ptx::tma_load_2d(sa + kABytes, mb0, full, kb * BK, t.w_row0);
-          ptx::tma_load_2d(sa + kABytes + kBHalfBytes, mb1, full, kb * BK, t.w_row0 + d.b1_row_shift);
+          ptx::tma_load_2d(sa, ma, full, kb * p.k_elems, t.row0);
+          ptx::tma_load_2d(sa + kABytes, mb0, full, kb * p.k_elems, t.w_row0);
+          ptx::tma_load_2d(sa + kABytes + kBHalfBytes, mb1, full, kb * p.k_elems, t.w_row0 + d.b1_row_shift);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -421,7 +450,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN_ACC);
+      const uint32_t idesc = p.fp8 ? ptx::idesc_e4m3_f32(BM, BN_ACC) : ptx::idesc_bf16_f32(BM, BN_ACC);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -463,8 +492,10 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #pragma unroll
           for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
             // +32 bytes along K inside the swizzle row = +2 in the descriptor's 16-byte address units
-            ptx::tc_mma_bf16(d_tmem, a_desc + static_cast<uint64_t>(2 * k4), b_desc + static_cast<uint64_t>(2 * k4),
-                             idesc, (kb | k4) != 0 ? 1u : 0u);
+            // (16 bf16 or 32 E4M3 elements per instruction: 32 bytes either way)
+            const uint64_t adv = static_cast<uint64_t>(2 * k4);
+            if (p.fp8) ptx::tc_mma_e4m3(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
+            else ptx::tc_mma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
           }
           ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // stage is free once these MMAs have read it
           st->mma_progress = ++progress;
@@ -695,8 +726,8 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
           const uint32_t full_leader = ptx::map_to_cta(full_local, 0);
           const uint32_t sa = stage_u32 + stage * kPairStageBytes;
           if (rank == 0) ptx::mbar_expect_tx(full_local, 2 * kPairStageBytes);   // the bytes of both CTAs
-          ptx::tma_load_2d_pair(sa, &tm_a, full_leader, kb * BK, t.row0);
-          ptx::tma_load_2d_pair(sa + kABytes, mb, full_leader, kb * BK, t.w_row0 + b_shift);
+          ptx::tma_load_2d_pair(sa, &tm_a, full_leader, kb * p.k_elems, t.row0);
+          ptx::tma_load_2d_pair(sa + kABytes, mb, full_leader, kb * p.k_elems, t.w_row0 + b_shift);
           if (++stage == kPairStages) { stage = 0; ph ^= 1u; }
         }
       }
@@ -708,7 +739,7 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(2 * BM, BN_ACC);
+      const uint32_t idesc = p.fp8 ? ptx::idesc_e4m3_f32(2 * BM, BN_ACC) : ptx::idesc_bf16_f32(2 * BM, BN_ACC);
       int stage = 0;
       uint32_t ph = 0;
       int acc = 0;
@@ -738,8 +769,9 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
           const uint64_t b_desc = ptx::smem_desc_sw128(sa + kABytes);
 #pragma unroll
           for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
-            ptx::tc_mma_bf16_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * k4),
-                                  b_desc + static_cast<uint64_t>(2 * k4), idesc, (kb | k4) != 0 ? 1u : 0u);
+            const uint64_t adv = static_cast<uint64_t>(2 * k4);
+            if (p.fp8) ptx::tc_mma_e4m3_pair(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
+            else ptx::tc_mma_bf16_pair(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
           }
           ptx::tc_commit_pair(ptx::smem_u32(&st->empty[stage]), 3);    // frees the stage in both CTAs
           st->mma_progress = ++progress;
@@ -856,14 +888,17 @@ __global__ void __launch_bounds__(128, 1) mma_cycle_probe(int M, int N, int iter
   }
 }
 
-CUresult encode_2d(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols) {
+// Tensor map over a row-major [rows, cols] matrix of bf16 (elem_bytes 2) or E4M3 bytes (elem_bytes 1): boxes of
+// 128 rows x 128 bytes, 128-byte swizzle.
+CUresult encode_2d(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, int elem_bytes) {
   const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), 128u};
+  const cuuint64_t strides[1] = {cols * static_cast<uint64_t>(elem_bytes)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes), 128u};
   const cuuint32_t elem[2] = {1u, 1u};
-  return ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
-                           elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return ctx->encode_tiled(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+                           const_cast<void*>(base), dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
 }  // namespace
@@ -935,66 +970,75 @@ cudaError_t launch_pair(moe_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b
 }
 }  // namespace
 
-moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* offsets, const void* w_gate,
-                             const void* w_up, const void* w_down, void* h_ws, void* y_perm,
-                             float* h_fp32_debug, const moe_tuning* tuning, cudaStream_t stream) {
+// Everything one expert-FFN call needs on the host side; fp8 selects E4M3 operands with epilogue scales.
+struct FfnCall {
+  const void* a1;          // Linear-1 input rows [R,H]
+  const void* w_gate;
+  const void* w_up;
+  const void* w_down;
+  void* h_bf16;            // Linear-1 output [R,F] bf16
+  const void* a2;          // Linear-2 input rows [R,F]: h_bf16 itself, or its E4M3 copy
+  void* y_perm;            // [R,H] bf16
+  float* h_dbg;
+  int fp8;
+  const float *s_a1, *s_gate, *s_up, *s_a2, *s_down;   // fp8 scales
+};
+
+static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets, const moe_tuning* tuning,
+                          cudaStream_t stream, bool second_phase_only, bool first_phase_only) {
   const moe_shape& s = ctx->shape;
   const uint64_t R = static_cast<uint64_t>(s.T) * s.k;
   if (R == 0) return MOE_OK;
   moe_tuning tn = {1, 0, 1, 0, 0, 0};
   if (tuning) tn = *tuning;
+  const int eb = c.fp8 ? 1 : 2;
+  const int k_elems = 128 / eb;
 
   CUtensorMap tm_x, tm_wg, tm_wu, tm_h, tm_wd;
-  if (encode_2d(ctx, &tm_x, x_perm, R, s.H) != CUDA_SUCCESS) return MOE_ERR_CUDA;
-  if (encode_2d(ctx, &tm_wg, w_gate, static_cast<uint64_t>(s.E) * s.F, s.H) != CUDA_SUCCESS) return MOE_ERR_CUDA;
-  if (encode_2d(ctx, &tm_wu, w_up, static_cast<uint64_t>(s.E) * s.F, s.H) != CUDA_SUCCESS) return MOE_ERR_CUDA;
-  if (encode_2d(ctx, &tm_h, h_ws, R, s.F) != CUDA_SUCCESS) return MOE_ERR_CUDA;
-  if (encode_2d(ctx, &tm_wd, w_down, static_cast<uint64_t>(s.E) * s.H, s.F) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_2d(ctx, &tm_x, c.a1, R, s.H, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_2d(ctx, &tm_wg, c.w_gate, static_cast<uint64_t>(s.E) * s.F, s.H, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_2d(ctx, &tm_wu, c.w_up, static_cast<uint64_t>(s.E) * s.F, s.H, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_2d(ctx, &tm_h, c.a2, R, s.F, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_2d(ctx, &tm_wd, c.w_down, static_cast<uint64_t>(s.E) * s.H, s.F, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
 
   FfnParams p{};
   p.offsets = offsets;
   p.E = s.E;
-  p.ph[0] = PhaseDesc{s.F, s.H, (s.F + 127) / 128, (s.H + BK - 1) / BK, 128, 0, static_cast<__nv_bfloat16*>(h_ws)};
-  p.ph[1] = PhaseDesc{s.H, s.F, (s.H + 255) / 256, (s.F + BK - 1) / BK, 256, 128, static_cast<__nv_bfloat16*>(y_perm)};
-  p.h_dbg = h_fp32_debug;
+  p.ph[0] = PhaseDesc{s.F, s.H, (s.F + 127) / 128, (s.H + k_elems - 1) / k_elems, 128, 0,
+                      static_cast<__nv_bfloat16*>(c.h_bf16), c.s_a1, c.s_gate, c.s_up};
+  p.ph[1] = PhaseDesc{s.H, s.F, (s.H + 255) / 256, (s.F + k_elems - 1) / k_elems, 256, 128,
+                      static_cast<__nv_bfloat16*>(c.y_perm), c.s_a2, c.s_down, c.s_down};
+  p.h_dbg = c.h_dbg;
   p.burst = tn.store_burst_tiles;
   p.mode = tn.interleave_mode;
   p.ik = tn.interleave_k;
   p.status = ctx->d_status;
   p.ready = ctx->d_ready;
   p.schedule = tn.schedule;
+  p.fp8 = c.fp8;
+  p.k_elems = k_elems;
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
   // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
   p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);
   p.withhold_ready = (tn.debug_flags & 4) != 0;
   p.wait_budget = p.withhold_ready ? 200000000LL : ptx::kWaitClockBudget;   // the drill gives up after ~0.1 s
   const bool trace = (tn.debug_flags & 1) != 0;
-  if (trace && cudaMemsetAsync(ctx->d_trace, 0, static_cast<size_t>(2) * ctx->num_sms * kMoeTraceFields * 8, stream) !=
-                   cudaSuccess)
+  if (trace && !second_phase_only &&
+      cudaMemsetAsync(ctx->d_trace, 0, static_cast<size_t>(2) * ctx->num_sms * kMoeTraceFields * 8, stream) !=
+          cudaSuccess)
     return MOE_ERR_CUDA;   // roles that do not run in a variant (the peer's MMA warp) leave zeros, not stale counts
+  const bool split = second_phase_only || first_phase_only;   // the caller runs something between the two GEMMs
   // Launch-latency-bound layers (every tile fits in about one wave of CTAs) run both GEMMs in one launch.
   const long long max_blocks = static_cast<long long>(R / 128) + s.E;
   const bool tiny = max_blocks * (p.ph[0].n_blocks + p.ph[1].n_blocks) <= 2LL * grid;
-  const bool one_launch = tn.schedule == 1 || (tn.debug_flags & 6) != 0 || tiny;
-
+  const bool one_launch = !split && (tn.schedule == 1 || (tn.debug_flags & 6) != 0 || tiny);
   // CTA pairs (256-row tiles) pay off when experts hold many rows; single-block experts would waste the peer.
   const bool dense = R / static_cast<uint64_t>(s.E) >= 1024;
-  const bool pairs = !one_launch && ctx->max_pairs > 0 && ((tn.debug_flags & 8) != 0 || (dense && (tn.debug_flags & 16) == 0));
-  if (pairs) {
-    p.trace = trace ? ctx->d_trace : nullptr;
-    p.phase_lo = 0;
-    p.phase_hi = 1;
-    p.kernel_id = 4;
-    if (launch_pair(ctx, tm_x, tm_wg, tm_wu, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
-    moe_mark(ctx, 5, stream);
-    p.trace = trace ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
-    p.phase_lo = 1;
-    p.phase_hi = 2;
-    p.kernel_id = 5;
-    if (launch_pair(ctx, tm_h, tm_wd, tm_wd, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
-    moe_mark(ctx, 6, stream);
-    ctx->last_launches += 2;
-  } else if (one_launch) {
+  const bool pairs = !one_launch && ctx->max_pairs > 0 &&
+                     ((tn.debug_flags & 8) != 0 || (dense && (tn.debug_flags & 16) == 0));
+  unsigned long long* trace2 = trace ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
+
+  if (one_launch) {
     p.phase_lo = 0;
     p.phase_hi = 2;
     p.sched = ctx->d_sched;
@@ -1005,24 +1049,77 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
     moe_mark(ctx, 5, stream);
     moe_mark(ctx, 6, stream);
     ctx->last_launches += 1;
-  } else {
+    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  }
+  if (!second_phase_only) {
     p.phase_lo = 0;
     p.phase_hi = 1;
     p.sched = ctx->d_sched;
     p.trace = trace ? ctx->d_trace : nullptr;
-    p.kernel_id = 1;
-    expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+    p.kernel_id = pairs ? 4 : 1;
+    if (pairs) {
+      if (launch_pair(ctx, tm_x, tm_wg, tm_wu, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+    } else {
+      expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+    }
     moe_mark(ctx, 5, stream);
+    ctx->last_launches += 1;
+  }
+  if (!first_phase_only) {
     p.phase_lo = 1;
     p.phase_hi = 2;
     p.sched = ctx->d_sched + 2;
-    p.trace = trace ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
-    p.kernel_id = 2;
-    expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+    p.trace = trace2;
+    p.kernel_id = pairs ? 5 : 2;
+    if (pairs) {
+      if (launch_pair(ctx, tm_h, tm_wd, tm_wd, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+    } else {
+      expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+    }
     moe_mark(ctx, 6, stream);
-    ctx->last_launches += 2;
+    ctx->last_launches += 1;
   }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* offsets, const void* w_gate,
+                             const void* w_up, const void* w_down, void* h_ws, void* y_perm,
+                             float* h_fp32_debug, const moe_tuning* tuning, cudaStream_t stream) {
+  FfnCall c{};
+  c.a1 = x_perm;
+  c.w_gate = w_gate;
+  c.w_up = w_up;
+  c.w_down = w_down;
+  c.h_bf16 = h_ws;
+  c.a2 = h_ws;
+  c.y_perm = y_perm;
+  c.h_dbg = h_fp32_debug;
+  return run_ffn(ctx, c, offsets, tuning, stream, false, false);
+}
+
+moe_status launch_expert_ffn_fp8(moe_ctx* ctx, const moe_fp8_ffn_args* a, const moe_tuning* tuning,
+                                 cudaStream_t stream) {
+  const moe_shape& s = ctx->shape;
+  FfnCall c{};
+  c.a1 = a->xq_perm;
+  c.w_gate = a->wq_gate;
+  c.w_up = a->wq_up;
+  c.w_down = a->wq_down;
+  c.h_bf16 = a->h_ws;
+  c.a2 = a->hq_ws;
+  c.y_perm = a->y_perm;
+  c.fp8 = 1;
+  c.s_a1 = a->sx_perm;
+  c.s_gate = a->s_gate;
+  c.s_up = a->s_up;
+  c.s_a2 = a->sh_ws;
+  c.s_down = a->s_down;
+  moe_status st = run_ffn(ctx, c, a->offsets, tuning, stream, false, true);          // Linear-1 -> h (bf16)
+  if (st != MOE_OK) return st;
+  if (launch_quantize_rows(ctx, a->h_ws, static_cast<long long>(s.T) * s.k, s.F, a->hq_ws, a->sh_ws, stream) !=
+      cudaSuccess)
+    return MOE_ERR_CUDA;                                                              // h -> E4M3 + row scales
+  return run_ffn(ctx, c, a->offsets, tuning, stream, true, false);                    // Linear-2
 }
 
 }  // namespace moe

@@ -297,6 +297,148 @@ moe_status moe_fused_forward(moe_ctx* ctx, const void* x, const float* logits, c
   return MOE_OK;
 }
 
+// ------------------------------------------------------------------------------------------------ FP8 variant
+namespace {
+void fill_layout_fp8(const moe_shape& s, moe_workspace_layout_fp8* L) {
+  const size_t T = s.T, H = s.H, F = s.F, E = s.E, k = s.k, R = T * k;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t at = off; off += up256(bytes); return at; };
+  L->topk_ids = take(R * 4);
+  L->topk_w = take(R * 4);
+  L->counts = take(E * 4);
+  L->offsets = take((E + 1) * 4);
+  L->perm = take(R * 4);
+  L->inv_perm = take(R * 4);
+  L->xq = take(T * H);
+  L->sx = take(T * 4);
+  L->xq_perm = take(R * H);
+  L->sx_perm = take(R * 4);
+  L->h = take(R * F * 2);
+  L->hq = take(R * F);
+  L->sh = take(R * 4);
+  L->y_perm = take(R * H * 2);
+  L->total = off;
+}
+moe_status check_fp8_shape(const moe_ctx* ctx) {
+  return (ctx->shape.H % 128 == 0 && ctx->shape.F % 128 == 0) ? MOE_OK : MOE_ERR_UNSUPPORTED_SHAPE;
+}
+}  // namespace
+
+moe_status moe_get_workspace_layout_fp8(const moe_shape* shape, moe_workspace_layout_fp8* out_layout) {
+  if (!out_layout) return MOE_ERR_INVALID_ARG;
+  std::memset(out_layout, 0, sizeof(*out_layout));
+  moe_status st = check_shape(shape);
+  if (st != MOE_OK) return st;
+  if (shape->H % 128 != 0 || shape->F % 128 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
+  fill_layout_fp8(*shape, out_layout);
+  return MOE_OK;
+}
+
+moe_status moe_quantize_rows(moe_ctx* ctx, const void* in_bf16, int64_t rows, int32_t cols, void* codes,
+                             float* scales, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  ctx->last_launches = 0;
+  if (rows < 0 || cols <= 0 || cols % 8 != 0) return MOE_ERR_INVALID_ARG;
+  if (rows == 0) return MOE_OK;
+  if (!in_bf16 || !codes || !scales || !aligned16(in_bf16) || (reinterpret_cast<uintptr_t>(codes) & 7u) != 0)
+    return MOE_ERR_INVALID_ARG;
+  return moe::launch_quantize_rows(ctx, in_bf16, rows, cols, codes, scales, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_dispatch_fp8(moe_ctx* ctx, const void* xq, const float* sx, const int32_t* inv_perm, void* xq_perm,
+                            float* sx_perm, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  st = check_fp8_shape(ctx);
+  if (st != MOE_OK) return st;
+  begin_call(ctx, 3, stream);
+  if (ctx->shape.T == 0) return MOE_OK;
+  if (!xq || !sx || !inv_perm || !xq_perm || !sx_perm) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(xq) || !aligned16(inv_perm) || !aligned16(xq_perm)) return MOE_ERR_INVALID_ARG;
+  return moe::launch_dispatch_fp8(ctx, xq, sx, inv_perm, xq_perm, sx_perm, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_expert_ffn_fp8(moe_ctx* ctx, const moe_fp8_ffn_args* a, const moe_tuning* tuning, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  st = check_fp8_shape(ctx);
+  if (st != MOE_OK) return st;
+  begin_call(ctx, 4, stream);
+  st = check_tuning(tuning);
+  if (st != MOE_OK) return st;
+  if (tuning && (tuning->schedule != 0 || (tuning->debug_flags & 6) != 0)) return MOE_ERR_UNSUPPORTED;
+  if (ctx->shape.T == 0) return MOE_OK;
+  if (!a) return MOE_ERR_INVALID_ARG;
+  const void* ptrs[] = {a->xq_perm, a->sx_perm, a->offsets, a->wq_gate, a->s_gate, a->wq_up, a->s_up,
+                        a->wq_down, a->s_down, a->h_ws, a->hq_ws, a->sh_ws, a->y_perm};
+  for (const void* q : ptrs)
+    if (!q || (reinterpret_cast<uintptr_t>(q) & 15u) != 0) return MOE_ERR_INVALID_ARG;
+  return moe::launch_expert_ffn_fp8(ctx, a, tuning, static_cast<cudaStream_t>(stream));
+}
+
+moe_status moe_fused_forward_fp8(moe_ctx* ctx, const void* x, const float* logits, const void* wq_gate,
+                                 const float* s_gate, const void* wq_up, const float* s_up, const void* wq_down,
+                                 const float* s_down, void* out, void* workspace, size_t workspace_bytes,
+                                 const moe_tuning* tuning, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  st = check_fp8_shape(ctx);
+  if (st != MOE_OK) return st;
+  st = check_tuning(tuning);
+  if (st != MOE_OK) return st;
+  if (tuning && (tuning->schedule != 0 || (tuning->debug_flags & 6) != 0)) return MOE_ERR_UNSUPPORTED;
+  const moe_shape& s = ctx->shape;
+  if (s.T == 0) { ctx->last_launches = 0; return MOE_OK; }
+  const void* ptrs[] = {x, logits, wq_gate, s_gate, wq_up, s_up, wq_down, s_down, out};
+  for (const void* q : ptrs)
+    if (!q || (reinterpret_cast<uintptr_t>(q) & 15u) != 0) return MOE_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MOE_ERR_INVALID_ARG;
+  moe_workspace_layout_fp8 L;
+  fill_layout_fp8(s, &L);
+  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE_TOO_SMALL;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  int32_t* topk_ids = reinterpret_cast<int32_t*>(ws + L.topk_ids);
+  float* topk_w = reinterpret_cast<float*>(ws + L.topk_w);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+  int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
+  int32_t* perm = reinterpret_cast<int32_t*>(ws + L.perm);
+  int32_t* inv_perm = reinterpret_cast<int32_t*>(ws + L.inv_perm);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  begin_call(ctx, 0, stream);
+  if (moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (moe::launch_quantize_rows(ctx, x, s.T, s.H, ws + L.xq, reinterpret_cast<float*>(ws + L.sx), cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (moe::launch_dispatch_fp8(ctx, ws + L.xq, reinterpret_cast<const float*>(ws + L.sx), inv_perm, ws + L.xq_perm,
+                               reinterpret_cast<float*>(ws + L.sx_perm), cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  moe_fp8_ffn_args a;
+  a.xq_perm = ws + L.xq_perm;
+  a.sx_perm = reinterpret_cast<const float*>(ws + L.sx_perm);
+  a.offsets = offsets;
+  a.wq_gate = wq_gate;
+  a.s_gate = s_gate;
+  a.wq_up = wq_up;
+  a.s_up = s_up;
+  a.wq_down = wq_down;
+  a.s_down = s_down;
+  a.h_ws = ws + L.h;
+  a.hq_ws = ws + L.hq;
+  a.sh_ws = reinterpret_cast<float*>(ws + L.sh);
+  a.y_perm = ws + L.y_perm;
+  st = moe::launch_expert_ffn_fp8(ctx, &a, tuning, cs);
+  if (st != MOE_OK) return st;
+  if (moe::launch_combine(ctx, ws + L.y_perm, inv_perm, topk_w, out, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
 moe_status moe_fused_forward_host(moe_ctx* ctx, const void* x_host, const float* logits_host,
                                   const void* w_gate, const void* w_up, const void* w_down,
                                   void* out_host, void* workspace, size_t workspace_bytes,

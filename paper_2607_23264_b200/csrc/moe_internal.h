@@ -72,6 +72,17 @@ moe_status launch_expert_ffn(moe_ctx* ctx, const void* x_perm, const int32_t* of
                              const void* w_up, const void* w_down, void* h_ws, void* y_perm,
                              float* h_fp32_debug, const moe_tuning* tuning, cudaStream_t stream);
 
+moe_status launch_expert_ffn_fp8(moe_ctx* ctx, const moe_fp8_ffn_args* args, const moe_tuning* tuning,
+                                 cudaStream_t stream);
+
+// bf16 [rows, cols] -> E4M3 codes [rows, cols] + one fp32 scale per row (amax / 448).
+cudaError_t launch_quantize_rows(moe_ctx* ctx, const void* in_bf16, long long rows, int cols, void* codes,
+                                 float* scales, cudaStream_t stream);
+
+// Row mover for E4M3 rows with their scales: xq_perm[inv_perm[t*k+j]] = xq[t], sx_perm[..] = sx[t].
+cudaError_t launch_dispatch_fp8(moe_ctx* ctx, const void* xq, const float* sx, const int32_t* inv_perm,
+                                void* xq_perm, float* sx_perm, cudaStream_t stream);
+
 cudaError_t prepare_expert_ffn(moe_ctx* ctx);  // one-time kernel attributes (dynamic shared memory size)
 
 }  // namespace moe
