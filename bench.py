@@ -325,6 +325,18 @@ def main():
     if weights_bytes < (256 << 20) or cfg.T <= 256:
         step_stats["cold_l2_flushed"] = per_step(True)
 
+    # SM clock while the first grouped-GEMM kernel runs, from the kernel's own clock64 span against its CUDA-event
+    # time (nvidia-smi, sampled every 100 ms, often misses a timed region this short)
+    ctx.moe_set_kernel_timing(True)
+    ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws,
+                          tuning=binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule,
+                                                     dep_lead_D=args.lead, debug_flags=dbg | 1))
+    span = float(ctx.moe_get_ffn_trace()[0, :, 0].max())
+    ms4 = ctx.moe_get_kernel_times()[4]
+    ctx.moe_set_kernel_timing(False)
+    if clocks is not None and ms4 > 0:
+        clocks["sm_mhz_kernel"] = span / (ms4 * 1e-3) / 1e6
+
     ffn_trace = None
     if args.trace:
         ttn = binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule, dep_lead_D=args.lead,

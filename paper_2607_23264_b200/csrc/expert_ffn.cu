@@ -210,7 +210,7 @@ __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target,
 
 // Drain one finished accumulator: rows of this thread's TMEM lane, kGated ? silu(g)*u of 128 columns
 // : 256 plain columns, written as bf16 with 16-byte stores masked to the expert's rows and to N.
-template <bool kGated>
+template <bool kGated, bool kFp8>
 __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams& p, uint32_t t_addr, int row,
                                                   long long* w_gap, volatile uint32_t* progress, volatile int* idle,
                                                   volatile int* aborting) {
@@ -229,7 +229,7 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
       ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
       ptx::tmem_ld_32x32(t_addr + 128 + c * kChunkCols, u);
       ptx::tmem_ld_wait();
-      if (d.row_scale != nullptr) {
+      if constexpr (kFp8) {
         const float rs = row_ok ? d.row_scale[row] : 0.f;
         const int w0 = t.w_row0 + c * kChunkCols;
 #pragma unroll
@@ -245,7 +245,7 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
     } else {
       ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
       ptx::tmem_ld_wait();
-      if (d.row_scale != nullptr) {
+      if constexpr (kFp8) {
         const float rs = row_ok ? d.row_scale[row] : 0.f;
         // columns 0..127 of the tile come from the first weight box, 128..255 from the second (same matrix)
         const int w0 = t.w_row0 + c * kChunkCols;
@@ -294,6 +294,7 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
   }
 }
 
+template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wg,
                   const __grid_constant__ CUtensorMap tm_wu, const __grid_constant__ CUtensorMap tm_h,
@@ -450,7 +451,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = p.fp8 ? ptx::idesc_e4m3_f32(BM, BN_ACC) : ptx::idesc_bf16_f32(BM, BN_ACC);
+      constexpr uint32_t idesc = kFp8 ? ptx::idesc_e4m3_f32(BM, BN_ACC) : ptx::idesc_bf16_f32(BM, BN_ACC);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -494,7 +495,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             // +32 bytes along K inside the swizzle row = +2 in the descriptor's 16-byte address units
             // (16 bf16 or 32 E4M3 elements per instruction: 32 bytes either way)
             const uint64_t adv = static_cast<uint64_t>(2 * k4);
-            if (p.fp8) ptx::tc_mma_e4m3(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
+            if constexpr (kFp8) ptx::tc_mma_e4m3(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
             else ptx::tc_mma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
           }
           ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // stage is free once these MMAs have read it
@@ -544,9 +545,11 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               static_cast<uint32_t>(acc * BN_ACC);
       if (t.phase == 0)
-        drain_accumulator<true>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle, abort_flag);
+        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
+                                      abort_flag);
       else
-        drain_accumulator<false>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle, abort_flag);
+        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
+                                       abort_flag);
       ptx::tc_fence_before_sync();
       if (chained && t.phase == 0) {
         // publish this warp's 32 rows x 128 columns of h to the Linear-2 tiles of the block
@@ -638,6 +641,7 @@ __device__ __forceinline__ Tile decode_pair_tile(int tile, int phase, uint32_t r
   return t;
 }
 
+template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                        const __grid_constant__ CUtensorMap tm_b1, const FfnParams p) {
@@ -739,7 +743,7 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
-      const uint32_t idesc = p.fp8 ? ptx::idesc_e4m3_f32(2 * BM, BN_ACC) : ptx::idesc_bf16_f32(2 * BM, BN_ACC);
+      constexpr uint32_t idesc = kFp8 ? ptx::idesc_e4m3_f32(2 * BM, BN_ACC) : ptx::idesc_bf16_f32(2 * BM, BN_ACC);
       int stage = 0;
       uint32_t ph = 0;
       int acc = 0;
@@ -770,7 +774,7 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
 #pragma unroll
           for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
             const uint64_t adv = static_cast<uint64_t>(2 * k4);
-            if (p.fp8) ptx::tc_mma_e4m3_pair(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
+            if constexpr (kFp8) ptx::tc_mma_e4m3_pair(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
             else ptx::tc_mma_bf16_pair(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
           }
           ptx::tc_commit_pair(ptx::smem_u32(&st->empty[stage]), 3);    // frees the stage in both CTAs
@@ -814,9 +818,11 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       FfnParams q = p;
       if (rank != 0) q.mode = 0;
       if (phase == 0)
-        drain_accumulator<true>(t, q, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle, abort_flag);
+        drain_accumulator<true, kFp8>(t, q, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
+                                      abort_flag);
       else
-        drain_accumulator<false>(t, q, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle, abort_flag);
+        drain_accumulator<false, kFp8>(t, q, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
+                                       abort_flag);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(acc ? empty_leader1 : empty_leader0);
@@ -926,12 +932,12 @@ extern "C" moe_status moe_probe_mma_cycles(moe_ctx* ctx, int32_t M, int32_t N, i
 namespace moe {
 
 cudaError_t prepare_expert_ffn(moe_ctx* ctx) {
-  cudaError_t e = cudaFuncSetAttribute(expert_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kSmemBytes));
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(expert_ffn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(kPairSmemBytes));
-  if (e != cudaSuccess) return e;
+  cudaError_t e = cudaSuccess;
+  const int smem1 = static_cast<int>(kSmemBytes), smem2 = static_cast<int>(kPairSmemBytes);
+  if ((e = cudaFuncSetAttribute(expert_ffn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(expert_ffn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(expert_ffn_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(expert_ffn_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2)) != cudaSuccess) return e;
   // how many CTA pairs can be resident at once (an SM left over in a GPC cannot join a pair)
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (ctx->num_sms / 2));
@@ -945,7 +951,7 @@ cudaError_t prepare_expert_ffn(moe_ctx* ctx) {
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
   int clusters = 0;
-  e = cudaOccupancyMaxActiveClusters(&clusters, expert_ffn_pair_kernel, &cfg);
+  e = cudaOccupancyMaxActiveClusters(&clusters, expert_ffn_pair_kernel<false>, &cfg);
   if (e != cudaSuccess) return e;
   ctx->max_pairs = clusters < ctx->num_sms / 2 ? clusters : ctx->num_sms / 2;
   return cudaSuccess;
@@ -966,9 +972,16 @@ cudaError_t launch_pair(moe_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, expert_ffn_pair_kernel, a, b0, b1, p);
+  return p.fp8 ? cudaLaunchKernelEx(&cfg, expert_ffn_pair_kernel<true>, a, b0, b1, p)
+               : cudaLaunchKernelEx(&cfg, expert_ffn_pair_kernel<false>, a, b0, b1, p);
 }
 }  // namespace
+
+static void launch_single(int grid, const CUtensorMap& x, const CUtensorMap& wg, const CUtensorMap& wu,
+                          const CUtensorMap& h, const CUtensorMap& wd, const FfnParams& p, cudaStream_t stream) {
+  if (p.fp8) expert_ffn_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(x, wg, wu, h, wd, p);
+  else expert_ffn_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(x, wg, wu, h, wd, p);
+}
 
 // Everything one expert-FFN call needs on the host side; fp8 selects E4M3 operands with epilogue scales.
 struct FfnCall {
@@ -1045,7 +1058,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.trace = trace ? ctx->d_trace : nullptr;
     p.order_log = trace ? ctx->d_order : nullptr;
     p.kernel_id = 3;
-    expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+    launch_single(grid, tm_x, tm_wg, tm_wu, tm_h, tm_wd, p, stream);
     moe_mark(ctx, 5, stream);
     moe_mark(ctx, 6, stream);
     ctx->last_launches += 1;
@@ -1060,7 +1073,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     if (pairs) {
       if (launch_pair(ctx, tm_x, tm_wg, tm_wu, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
-      expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+      launch_single(grid, tm_x, tm_wg, tm_wu, tm_h, tm_wd, p, stream);
     }
     moe_mark(ctx, 5, stream);
     ctx->last_launches += 1;
@@ -1074,7 +1087,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     if (pairs) {
       if (launch_pair(ctx, tm_h, tm_wd, tm_wd, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
-      expert_ffn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, tm_h, tm_wd, p);
+      launch_single(grid, tm_x, tm_wg, tm_wu, tm_h, tm_wd, p, stream);
     }
     moe_mark(ctx, 6, stream);
     ctx->last_launches += 1;

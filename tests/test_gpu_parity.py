@@ -363,3 +363,29 @@ def test_expired_wait_is_reported_not_hung():
         torch.cuda.synchronize()
         assert_out_close(dev_bf16_to_f64(out), oracle_for(L)["out"], "after the drill")
     L.check_device_status()
+
+
+def test_random_small_layers_property():
+    """Property tier: random small layers (ragged loads, empty experts, k up to 4, E up to 11) through every
+    schedule and kernel variant; indices bit-exact, output within tolerance, variants bitwise equal."""
+    rng = np.random.default_rng(2026)
+    for trial in range(16):
+        cfg = gen.random_small_config(rng)
+        L = Layer(cfg)
+        ref = oracle_for(L)
+        lay = L.ctx.workspace_layout()
+        ws = torch.empty(lay["total"], dtype=torch.uint8, device=DEV)
+        outs = []
+        for tn in (None, binding.make_tuning(1, 0, 1, debug_flags=8), binding.make_tuning(1, 0, 1, debug_flags=16),
+                   binding.make_tuning(1, 0, 1, schedule=1, dep_lead_D=1 + trial % 3)):
+            out = L.nan_bf16(cfg.T, cfg.H)
+            L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws, tuning=tn)
+            torch.cuda.synchronize()
+            outs.append(out)
+        what = f"trial {trial}: {cfg}"
+        perm = ws[lay["perm"]:lay["perm"] + 4 * cfg.R].view(torch.int32).cpu().numpy()
+        assert np.array_equal(perm, ref["perm"]), what
+        assert_out_close(dev_bf16_to_f64(outs[0]), ref["out"], what)
+        for o in outs[1:]:
+            assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16)), what
+        L.check_device_status()
