@@ -1,7 +1,7 @@
 // Routing plan: top-k + softmax weights, per-expert histogram, exclusive scan, stable permutation.
 //
 // The token range is cut into chunks of `tokens_per_chunk` tokens (at most 256 slots).  Three launches:
-//   1. route_topk_hist : one CTA per chunk; a warp per token selects the k largest logits by k rounds of
+//   1. route_topk_hist : one CTA per chunk; a warp per token selects the k largest logits by k passes of
 //                        warp arg-max (shuffle reduction, ties to the lower index) and computes the
 //                        softmax weights; the CTA then histograms its slots per expert.
 //   2. route_scan      : one CTA; exclusive prefix of the chunk histograms over chunks (per expert) and
@@ -38,7 +38,7 @@ route_topk_hist(const float* __restrict__ logits, int T, int E, int k, int token
     const float* row = logits + static_cast<size_t>(t) * E;
     for (int e = lane; e < E; e += 32) my[e] = row[e];
     __syncwarp();
-    float sel_logit = 0.f;   // lane j keeps the logit picked in round j
+    float sel_logit = 0.f;   // lane j keeps the logit picked in pass j
     int sel_id = 0;
     for (int j = 0; j < k; ++j) {
       float best = -INFINITY;
@@ -57,7 +57,7 @@ route_topk_hist(const float* __restrict__ logits, int T, int E, int k, int token
       if (lane == 0) my[best_e] = -INFINITY;    // taken
       __syncwarp();
     }
-    // softmax over the k selected logits; round 0 picked the maximum
+    // softmax over the k selected logits; pass 0 picked the maximum
     const float m = __shfl_sync(kFull, sel_logit, 0);
     float p = (lane < k) ? expf(sel_logit - m) : 0.f;
     float sum = p;
