@@ -112,6 +112,15 @@ const char* moe_status_string(moe_status s);
 moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device);
 void moe_destroy(moe_ctx* ctx);
 
+/*
+ * Serving batches vary in size: a context created for T tokens also runs any smaller batch.  This sets the
+ * number of tokens the following calls process (0 <= tokens <= the T given to moe_create); every tensor
+ * argument then has `tokens` rows ([tokens,H], [tokens*k], ...), and the workspace slices are those of
+ * moe_get_workspace_layout for a shape with T = tokens (a workspace sized for the creation shape always suffices).
+ * No device work, no allocation.  Errors: INVALID_ARG.
+ */
+moe_status moe_set_active_tokens(moe_ctx* ctx, int32_t tokens);
+
 /* Size and slicing of the caller-provided workspace of moe_fused_forward.  Returns 0 / fills zeros for a
  * shape moe_create would reject. */
 size_t moe_workspace_bytes(const moe_shape* shape);

@@ -26,6 +26,7 @@ EXPORTS = (
     "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace", "moe_probe_mma_cycles",
     "moe_get_ffn_order", "moe_fused_forward_host_pipelined", "moe_host_pipeline_flush", "moe_quantize_rows",
     "moe_dispatch_fp8", "moe_expert_ffn_fp8", "moe_get_workspace_layout_fp8", "moe_fused_forward_fp8",
+    "moe_set_active_tokens",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -103,6 +104,7 @@ def load_library() -> C.CDLL:
     lib.moe_get_workspace_layout_fp8.argtypes = [C.POINTER(moe_shape), C.POINTER(moe_workspace_layout_fp8)]
     lib.moe_fused_forward_fp8.argtypes = [vp, vp, f32p, vp, f32p, vp, f32p, vp, f32p, vp, vp, C.c_size_t,
                                           C.POINTER(moe_tuning), vp]
+    lib.moe_set_active_tokens.argtypes = [vp, C.c_int32]
     lib.moe_last_device_status.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_last_launch_count.argtypes = [vp]
     lib.moe_last_launch_count.restype = C.c_int32
@@ -209,6 +211,11 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def moe_set_active_tokens(self, tokens: int):
+        """Process `tokens` <= the creation T in the following calls (tensor arguments shrink accordingly)."""
+        _check(self._lib.moe_set_active_tokens(self._handle, tokens), "moe_set_active_tokens")
+        self.T = tokens
 
     def workspace_bytes(self) -> int:
         return moe_workspace_bytes(self.T, self.H, self.F, self.E, self.k)

@@ -46,6 +46,15 @@ inline void begin_call(moe_ctx* ctx, int first_mark, void* stream) {
   moe_mark(ctx, first_mark, static_cast<cudaStream_t>(stream));
 }
 
+// A routing chunk holds at most 256 slots (k <= 32, so at least 8 tokens).  Small batches use smaller chunks,
+// down to one token per warp, so that the top-k work spreads over about two CTAs per SM.
+void set_chunking(moe_ctx* ctx, int tokens) {
+  ctx->tokens_per_chunk = kRouteThreads / ctx->shape.k;
+  const int spread = (tokens + 2 * ctx->num_sms - 1) / (2 * ctx->num_sms);
+  if (spread < ctx->tokens_per_chunk) ctx->tokens_per_chunk = spread < 8 ? 8 : spread;
+  ctx->num_chunks = tokens ? (tokens + ctx->tokens_per_chunk - 1) / ctx->tokens_per_chunk : 0;
+}
+
 inline size_t up256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
 void fill_layout(const moe_shape& s, moe_workspace_layout* L) {
@@ -123,13 +132,10 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
     delete ctx;
     return MOE_ERR_CUDA;
   }
-  // A routing chunk holds at most 256 slots (k <= 32, so at least 8 tokens).  Small batches use smaller chunks,
-  // down to one token per warp, so that the top-k work spreads over about two CTAs per SM.
-  ctx->tokens_per_chunk = kRouteThreads / shape->k;
-  const int spread = (shape->T + 2 * ctx->num_sms - 1) / (2 * ctx->num_sms);
-  if (spread < ctx->tokens_per_chunk) ctx->tokens_per_chunk = spread < 8 ? 8 : spread;
-  ctx->num_chunks = shape->T ? (shape->T + ctx->tokens_per_chunk - 1) / ctx->tokens_per_chunk : 0;
-  const size_t hist_elems = static_cast<size_t>(ctx->num_chunks ? ctx->num_chunks : 1) * shape->E;
+  ctx->max_tokens = shape->T;
+  set_chunking(ctx, shape->T);
+  // scratch for the finest chunking any batch up to T can use (8 tokens per chunk)
+  const size_t hist_elems = static_cast<size_t>(shape->T / 8 + 1) * shape->E;
 
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -169,6 +175,13 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
     return MOE_ERR_CUDA;
   }
   *out_ctx = ctx;
+  return MOE_OK;
+}
+
+moe_status moe_set_active_tokens(moe_ctx* ctx, int32_t tokens) {
+  if (!ctx || tokens < 0 || tokens > ctx->max_tokens) return MOE_ERR_INVALID_ARG;
+  ctx->shape.T = tokens;
+  set_chunking(ctx, tokens);
   return MOE_OK;
 }
 

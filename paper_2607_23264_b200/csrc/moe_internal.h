@@ -28,6 +28,7 @@ struct moe_ctx {
   int device;
   int num_sms;
   int max_pairs;         // CTA pairs (clusters of two) of the pair kernel that can be resident at once
+  int max_tokens;        // T given at creation: the size of the routing scratch; shape.T is the active batch
   int tokens_per_chunk;  // routing: tokens handled by one CTA, so that a chunk has at most 256 slots
   int num_chunks;
   int32_t* d_chunk_hist;  // [num_chunks, E] slots of each chunk per expert

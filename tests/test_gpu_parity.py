@@ -389,3 +389,52 @@ def test_random_small_layers_property():
         for o in outs[1:]:
             assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16)), what
         L.check_device_status()
+
+
+def test_smaller_batches_on_one_context():
+    """A context created for T tokens serves any smaller batch (moe_set_active_tokens), with a workspace sized once."""
+    cfg = gen.MoEConfig("varT", T=900, H=256, F=384, E=6, k=2, seed=101, router="xWr")
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)      # sized for the creation shape
+    for tokens in (900, 1, 137, 512, 0, 900):
+        L.ctx.moe_set_active_tokens(tokens)
+        assert L.ctx.workspace_bytes() <= ws.numel()
+        out = L.nan_bf16(max(tokens, 1), cfg.H)
+        L.ctx.moe_fused_forward(L.x[:tokens].contiguous() if tokens else L.x, L.d_logits[:tokens].contiguous() if tokens
+                                else L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
+        torch.cuda.synchronize()
+        if tokens:
+            ref = orc.forward(L.x_bits[:tokens], L.logits[:tokens], cfg.k, L.weights)
+            assert_out_close(dev_bf16_to_f64(out[:tokens]), ref["out"], f"{tokens} tokens")
+    with pytest.raises(binding.MoeError):
+        L.ctx.moe_set_active_tokens(901)
+    L.check_device_status()
+
+
+def test_fused_forward_replays_from_a_cuda_graph():
+    """The layer makes no host synchronisation and no allocation, so a stream capture records it and the graph
+    replays it on new input values in the same buffers."""
+    cfg = SMALL[5]
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    x_buf, lg_buf = L.x.clone(), L.d_logits.clone()
+    L.ctx.moe_fused_forward(x_buf, lg_buf, L.w_gate, L.w_up, L.w_down, out, ws)      # warm-up outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        L.ctx.moe_fused_forward(x_buf, lg_buf, L.w_gate, L.w_up, L.w_down, out, ws, stream=side)
+        graph.capture_end()
+    torch.cuda.synchronize()
+    xb = np.roll(L.x_bits, 5, axis=0).copy()
+    lg = gen.make_logits(cfg, xb)
+    x_buf.copy_(bits_to_dev(xb))
+    lg_buf.copy_(torch.from_numpy(lg).to(DEV))
+    out.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    ref = orc.forward(xb, lg, cfg.k, L.weights)
+    assert_out_close(dev_bf16_to_f64(out), ref["out"], "graph replay")
+    L.check_device_status()
