@@ -337,6 +337,29 @@ def main():
     if clocks is not None and ms4 > 0:
         clocks["sm_mhz_kernel"] = span / (ms4 * 1e-3) / 1e6
 
+    # the same step replayed from a CUDA graph (launch overhead off the critical path; matters for small layers)
+    try:
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            g.capture_begin()
+            ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tuning, stream=side)
+            g.capture_end()
+        torch.cuda.synchronize()
+        for _ in range(3):
+            g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.steps):
+            g.replay()
+        b.record(stream)
+        b.synchronize()
+        step_stats["graph_replay_ms_per_step"] = a.elapsed_time(b) / args.steps
+    except Exception as exc:      # a capture failure must not lose the bench line
+        step_stats["graph_replay_ms_per_step"] = None
+        step_stats["graph_error"] = str(exc)[:200]
+
     ffn_trace = None
     if args.trace:
         ttn = binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule, dep_lead_D=args.lead,
