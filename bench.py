@@ -222,7 +222,8 @@ def main():
     w_gate = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
     w_up = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
     w_down = torch.empty((cfg.E, cfg.H, cfg.F), dtype=torch.bfloat16, device=dev)
-    keep_host = rank == 0 and not (args.no_cpu_baseline or args.sweep or args.profile) and cfg.E <= 16
+    want_cpu = rank == 0 and not (args.no_cpu_baseline or args.sweep or args.profile or args.fp8)
+    keep_host = want_cpu and cfg.E <= 16
     host_w = {}
 
     def sink(e, g, u, d):
@@ -488,8 +489,31 @@ def main():
         rate, dt = oracle_sample_rate(cfg, x_bits, logits, lambda e: host_w[e], args.cpu_baseline_tokens)
         line["cpu_baseline"] = {
             "value": rate, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
-            "sample": f"{args.cpu_baseline_tokens} seeded-random tokens of {cfg.name} (row-sampled fp64 oracle, "
-                      f"{dt:.1f} s)"}
+            "sample": f"{min(args.cpu_baseline_tokens, cfg.T)} seeded-random tokens of {cfg.name} (row-sampled fp64 "
+                      f"oracle, {dt:.1f} s)"}
+    elif want_cpu:
+        # many experts: sample tokens until they touch about 64 experts, regenerate those experts' weights on the
+        # host first (input generation, not timed), then time the oracle on the sample
+        from oracle import moe_oracle as orc
+        ids, _ = orc.topk_route(logits, cfg.k)
+        rng = np.random.default_rng(1234)
+        toks, experts = [], set()
+        for t in rng.permutation(cfg.T):
+            toks.append(int(t))
+            experts.update(ids[t].tolist())
+            if len(experts) >= 64 or len(toks) >= args.cpu_baseline_tokens:
+                break
+        stream_w = gen.WeightStream(cfg, sorted(experts))
+        held = {e: stream_w(e) for e in sorted(experts)}
+        stream_w.close()
+        toks = np.sort(np.array(toks))
+        t0 = time.perf_counter()
+        orc.forward_tokens(toks, x_bits, logits, cfg.k, lambda e: held[e])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {
+            "value": len(toks) / dt, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"{len(toks)} seeded-random tokens of {cfg.name} touching {len(experts)} experts "
+                      f"(row-sampled fp64 oracle, {dt:.1f} s)"}
     else:
         line["cpu_baseline"] = None
     print(json.dumps(line), flush=True)
