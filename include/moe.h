@@ -34,7 +34,8 @@ typedef enum {
   MOE_ERR_INVALID_ARG = 1,         /* null pointer, misaligned pointer, wrong device, bad tuning value */
   MOE_ERR_UNSUPPORTED_SHAPE = 2,   /* H or F not a multiple of 64, k or E out of range, T < 0 */
   MOE_ERR_WORKSPACE_TOO_SMALL = 3,
-  MOE_ERR_BAD_ROUTING = 4,         /* reserved: routing input violates the contract */
+  MOE_ERR_BAD_ROUTING = 4,         /* device status only: an expert id given to moe_plan_routing_from_topk is
+                                      outside [0, E) */
   MOE_ERR_CUDA = 5,                /* a CUDA runtime or driver call failed */
   MOE_ERR_TIMEOUT = 6,             /* device status only: a bounded on-device wait expired */
   MOE_ERR_UNSUPPORTED = 7,         /* ep_size != 1, unknown schedule */
@@ -139,6 +140,18 @@ moe_status moe_get_workspace_layout(const moe_shape* shape, moe_workspace_layout
 moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids, float* topk_w,
                             int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
                             void* stream);
+
+/*
+ * The same plan for routers the library does not know (sigmoid scores, bias-corrected or group-limited top-k, ...):
+ * the caller supplies the expert ids it chose, topk_ids [T,k] int32, and keeps its own combine weights for
+ * moe_combine.  Counts, offsets and the stable permutation are built exactly as in moe_plan_routing.  Every id
+ * must lie in [0, E); an id outside is reported through the status word (MOE_ERR_BAD_ROUTING, detail = the flat
+ * slot t*k+j) and treated as expert 0 so that no write goes out of bounds; the plan is then meaningless.
+ * topk_ids_checked [T,k] int32 receives the ids actually used (it may be the same buffer as topk_ids).
+ */
+moe_status moe_plan_routing_from_topk(moe_ctx* ctx, const int32_t* topk_ids, int32_t* topk_ids_checked,
+                                      int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
+                                      void* stream);
 
 /*
  * The routing plan for callers that must not allocate.  (The paper has no counterpart: this entry point

@@ -26,7 +26,7 @@ EXPORTS = (
     "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace", "moe_probe_mma_cycles",
     "moe_get_ffn_order", "moe_fused_forward_host_pipelined", "moe_host_pipeline_flush", "moe_quantize_rows",
     "moe_dispatch_fp8", "moe_expert_ffn_fp8", "moe_get_workspace_layout_fp8", "moe_fused_forward_fp8",
-    "moe_set_active_tokens",
+    "moe_set_active_tokens", "moe_plan_routing_from_topk",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -105,6 +105,7 @@ def load_library() -> C.CDLL:
     lib.moe_fused_forward_fp8.argtypes = [vp, vp, f32p, vp, f32p, vp, f32p, vp, f32p, vp, vp, C.c_size_t,
                                           C.POINTER(moe_tuning), vp]
     lib.moe_set_active_tokens.argtypes = [vp, C.c_int32]
+    lib.moe_plan_routing_from_topk.argtypes = [vp, i32p, i32p, i32p, i32p, i32p, i32p, vp]
     lib.moe_last_device_status.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_last_launch_count.argtypes = [vp]
     lib.moe_last_launch_count.restype = C.c_int32
@@ -227,6 +228,11 @@ class Context:
         _check(self._lib.moe_plan_routing(self._handle, _ptr(logits), _ptr(topk_ids), _ptr(topk_w), _ptr(counts),
                                           _ptr(offsets), _ptr(perm), _ptr(inv_perm), _stream(stream)),
                "moe_plan_routing")
+
+    def moe_plan_routing_from_topk(self, topk_ids, topk_ids_checked, counts, offsets, perm, inv_perm, stream=None):
+        _check(self._lib.moe_plan_routing_from_topk(self._handle, _ptr(topk_ids), _ptr(topk_ids_checked), _ptr(counts),
+                                                    _ptr(offsets), _ptr(perm), _ptr(inv_perm), _stream(stream)),
+               "moe_plan_routing_from_topk")
 
     def moe_dispatch(self, x, inv_perm, x_perm, stream=None):
         _check(self._lib.moe_dispatch(self._handle, _ptr(x), _ptr(inv_perm), _ptr(x_perm), _stream(stream)),

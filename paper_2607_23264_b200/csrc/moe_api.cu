@@ -229,6 +229,29 @@ moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids
              : MOE_ERR_CUDA;
 }
 
+moe_status moe_plan_routing_from_topk(moe_ctx* ctx, const int32_t* topk_ids, int32_t* topk_ids_checked,
+                                      int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
+                                      void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  begin_call(ctx, 0, stream);
+  const moe_shape& s = ctx->shape;
+  if (!counts || !offsets) return MOE_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (s.T == 0) {
+    if (cudaMemsetAsync(counts, 0, static_cast<size_t>(s.E) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaMemsetAsync(offsets, 0, static_cast<size_t>(s.E + 1) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+  }
+  if (!topk_ids || !topk_ids_checked || !perm || !inv_perm) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(topk_ids) || !aligned16(topk_ids_checked) || !aligned16(counts) || !aligned16(offsets) ||
+      !aligned16(perm) || !aligned16(inv_perm))
+    return MOE_ERR_INVALID_ARG;
+  return moe::launch_plan_from_topk(ctx, topk_ids, topk_ids_checked, counts, offsets, perm, inv_perm, cs) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
 moe_status moe_dispatch(moe_ctx* ctx, const void* x, const int32_t* inv_perm, void* x_perm, void* stream) {
   moe_status st = check_ctx(ctx);
   if (st != MOE_OK) return st;

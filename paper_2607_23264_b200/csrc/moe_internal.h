@@ -62,6 +62,10 @@ cudaError_t launch_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk
                                 int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
                                 cudaStream_t stream);
 
+// Plan from expert ids chosen by the caller; ids_checked receives the ids with out-of-range ones replaced by 0.
+cudaError_t launch_plan_from_topk(moe_ctx* ctx, const int32_t* topk_ids, int32_t* ids_checked, int32_t* counts,
+                                  int32_t* offsets, int32_t* perm, int32_t* inv_perm, cudaStream_t stream);
+
 cudaError_t launch_dispatch(moe_ctx* ctx, const void* x, const int32_t* inv_perm, void* x_perm,
                             cudaStream_t stream);
 

@@ -78,6 +78,35 @@ route_topk_hist(const float* __restrict__ logits, int T, int E, int k, int token
   for (int e = tid; e < E; e += kRouteThreads) chunk_hist[static_cast<size_t>(chunk) * E + e] = s_hist[e];
 }
 
+// Histogram of externally supplied expert ids (same chunking as route_topk_hist).  An id outside [0, E) violates
+// the contract: it is reported through the status word and counted as expert 0 so that nothing is written out of
+// bounds; the plan is then meaningless.
+__global__ void __launch_bounds__(kRouteThreads)
+route_hist_ids(const int32_t* __restrict__ topk_ids, int T, int E, int k, int tokens_per_chunk,
+               int32_t* __restrict__ ids_checked, int32_t* __restrict__ chunk_hist, int32_t* __restrict__ status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  int32_t* s_hist = reinterpret_cast<int32_t*>(smem_raw);   // [E]
+  const int tid = threadIdx.x, chunk = blockIdx.x;
+  const int t_begin = chunk * tokens_per_chunk;
+  const int t_end = min(T, t_begin + tokens_per_chunk);
+  const int n_slots = (t_end - t_begin) * k;
+  for (int e = tid; e < E; e += kRouteThreads) s_hist[e] = 0;
+  __syncthreads();
+  if (tid < n_slots) {
+    const size_t s = static_cast<size_t>(t_begin) * k + tid;
+    int e = topk_ids[s];
+    if (e < 0 || e >= E) {
+      atomicCAS(&status[0], 0, MOE_ERR_BAD_ROUTING);
+      atomicCAS(&status[1], 0, static_cast<int>(s));
+      e = 0;
+    }
+    ids_checked[s] = e;
+    atomicAdd(&s_hist[e], 1);
+  }
+  __syncthreads();
+  for (int e = tid; e < E; e += kRouteThreads) chunk_hist[static_cast<size_t>(chunk) * E + e] = s_hist[e];
+}
+
 // One CTA of 1024 threads, E <= 1024: thread e walks the chunks of expert e, then a block scan over e.
 __global__ void __launch_bounds__(1024)
 route_scan(const int32_t* __restrict__ chunk_hist, int32_t* __restrict__ chunk_base, int num_chunks, int E,
@@ -180,6 +209,19 @@ cudaError_t launch_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk
   route_scatter<<<ctx->num_chunks, kRouteThreads, smem3, stream>>>(topk_ids, offsets, ctx->d_chunk_base, s.T, s.E,
                                                                    s.k, ctx->tokens_per_chunk, perm, inv_perm);
   moe_mark(ctx, 3, stream);
+  ctx->last_launches += 3;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_plan_from_topk(moe_ctx* ctx, const int32_t* topk_ids, int32_t* ids_checked, int32_t* counts,
+                                  int32_t* offsets, int32_t* perm, int32_t* inv_perm, cudaStream_t stream) {
+  const moe_shape& s = ctx->shape;
+  const int warps = kRouteThreads / 32;
+  route_hist_ids<<<ctx->num_chunks, kRouteThreads, static_cast<size_t>(s.E) * 4, stream>>>(
+      topk_ids, s.T, s.E, s.k, ctx->tokens_per_chunk, ids_checked, ctx->d_chunk_hist, ctx->d_status);
+  route_scan<<<1, 1024, 0, stream>>>(ctx->d_chunk_hist, ctx->d_chunk_base, ctx->num_chunks, s.E, counts, offsets);
+  route_scatter<<<ctx->num_chunks, kRouteThreads, static_cast<size_t>(warps) * s.E * 4, stream>>>(
+      ids_checked, offsets, ctx->d_chunk_base, s.T, s.E, s.k, ctx->tokens_per_chunk, perm, inv_perm);
   ctx->last_launches += 3;
   return cudaGetLastError();
 }

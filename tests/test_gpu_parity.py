@@ -438,3 +438,50 @@ def test_fused_forward_replays_from_a_cuda_graph():
     ref = orc.forward(xb, lg, cfg.k, L.weights)
     assert_out_close(dev_bf16_to_f64(out), ref["out"], "graph replay")
     L.check_device_status()
+
+
+def test_plan_from_external_topk_and_bad_ids():
+    """Expert ids chosen by the caller (any router): the plan equals the oracle's plan for those ids; an id out of
+    range is reported in the status word and cannot write out of bounds."""
+    rng = np.random.default_rng(17)
+    T, E, k = 777, 33, 5
+    ids = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)      # not sorted by any score
+    ctx = binding.Context(T, 64, 64, E, k)
+    i32 = dict(dtype=torch.int32, device=DEV)
+    d_ids = torch.from_numpy(ids).to(DEV)
+    checked = torch.full((T, k), -1, **i32)
+    counts, offsets = torch.full((E,), -1, **i32), torch.full((E + 1,), -1, **i32)
+    perm, inv = torch.full((T * k + 1,), -7, **i32), torch.full((T * k + 1,), -7, **i32)
+    ctx.moe_plan_routing_from_topk(d_ids, checked, counts, offsets, perm, inv)
+    torch.cuda.synchronize()
+    c, o, p, ip = orc.plan_permutation(ids, E)
+    assert np.array_equal(checked.cpu().numpy(), ids)
+    assert np.array_equal(counts.cpu().numpy(), c) and np.array_equal(offsets.cpu().numpy(), o)
+    assert np.array_equal(perm[:-1].cpu().numpy(), p) and np.array_equal(inv[:-1].cpu().numpy(), ip)
+    assert perm[-1].item() == -7 and inv[-1].item() == -7, "canaries"
+    assert ctx.moe_last_device_status() == (0, 0)
+    bad = ids.copy()
+    bad[5, 2] = E + 3
+    ctx.moe_plan_routing_from_topk(torch.from_numpy(bad).to(DEV), checked, counts, offsets, perm, inv)
+    code, detail = ctx.moe_last_device_status()
+    assert code == 4 and detail == 5 * k + 2, "MOE_ERR_BAD_ROUTING with the offending slot"
+    assert checked[5, 2].item() == 0 and int(offsets[-1]) == T * k and perm[-1].item() == -7
+
+
+def test_wide_router_and_large_batch_plans():
+    """The limits of the routing plan: E = 1024 with k = 32 through the whole layer, and a 65536-token batch."""
+    cfg = gen.MoEConfig("wide", T=40, H=64, F=64, E=1024, k=32, seed=111, router="iid")
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
+    torch.cuda.synchronize()
+    L.check_device_status()
+    assert_out_close(dev_bf16_to_f64(out), oracle_for(L)["out"], "E=1024, k=32")
+    big = gen.MoEConfig("bigT", T=65536, H=64, F=64, E=256, k=8, seed=112, router="iid")
+    logits = gen.make_logits(big, None)
+    Lb = Layer(big, upload_weights=False, logits=logits, x_bits=np.zeros((1, 64), np.uint16))
+    Lb.plan()
+    ids, w = orc.topk_route(logits, big.k)
+    c, o, p, ip = orc.plan_permutation(ids, big.E)
+    assert_plan_matches(Lb, dict(topk_ids=ids, topk_w=w, counts=c, offsets=o, perm=p, inv_perm=ip))
