@@ -222,7 +222,7 @@ def main():
     w_gate = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
     w_up = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
     w_down = torch.empty((cfg.E, cfg.H, cfg.F), dtype=torch.bfloat16, device=dev)
-    want_cpu = rank == 0 and not (args.no_cpu_baseline or args.sweep or args.profile or args.fp8)
+    want_cpu = rank == 0 and world == 1 and not (args.no_cpu_baseline or args.sweep or args.profile or args.fp8)
     keep_host = want_cpu and cfg.E <= 16
     host_w = {}
 

@@ -300,7 +300,8 @@ moe_status moe_fused_forward_fp8(moe_ctx* ctx, const void* x, const float* logit
  * Same arguments as moe_fused_forward_host; x_host, logits_host and out_host should be pinned and must stay
  * valid until the pipeline is flushed.  out_host of call i is complete only after a later
  * moe_host_pipeline_flush(ctx, stream) followed by a synchronisation of `stream` (the flush makes `stream` wait
- * for every copy issued so far).  Use one `stream` per context.
+ * for every copy issued so far).  Use one `stream` per context, and flush before mixing in calls of
+ * moe_fused_forward_host, which shares the first staging slot.
  */
 moe_status moe_fused_forward_host_pipelined(moe_ctx* ctx, const void* x_host, const float* logits_host,
                                             const void* w_gate, const void* w_up, const void* w_down,
