@@ -100,9 +100,14 @@ def test_fused_forward_fp8_parity(cfg):
             dq, sd = f8.quantize_rows(orc.bf16_to_f64(L.weights(e)[2]))
             y_ref_own[lo:hi] = f8.scaled_gemm(hq[lo:hi], sh[lo:hi], dq, sd)
     assert rel_fro(y, y_ref_own) <= TOL_FRO
-    # end to end against the oracle (its own h quantisation): a flipped code moves one element by one E4M3 step
+    # the output against the oracle's combine of those rows: the bf16 path's elementwise bound
+    out_np = dev_bf16_to_f64(out)
+    assert_out_close(out_np, orc.combine(y_ref_own, ref["inv_perm"], ref["topk_w"]), f"fp8 out[{cfg.name}]")
+    # end to end against the fully independent oracle (its own h, its own codes): where the GPU's bf16 h and the
+    # oracle's differ in the last bit, an E4M3 code can flip and move that element of h by one step (up to 7 % of
+    # the row maximum), so single outputs may leave the elementwise bound; the norms must still agree
     assert rel_fro(y, ref["y_perm"]) <= 2e-2
-    assert_out_close(dev_bf16_to_f64(out), ref["out"], f"fp8 out[{cfg.name}]")
+    assert rel_fro(out_np, ref["out"]) <= 2e-2
     # and the FP8 layer stays within E4M3 noise of the bf16 layer
     full = orc.forward(L.x_bits, L.logits, cfg.k, L.weights)
     assert rel_fro(dev_bf16_to_f64(out), full["out"]) < 0.08
