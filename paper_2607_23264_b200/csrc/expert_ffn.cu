@@ -26,6 +26,10 @@
 //      row-major Linear-1 and Linear-2 tile lists (row = one 128-row block) and emits the Linear-2 tile only
 //      while Linear-1 leads by D rows, else the next Linear-1 tile.  One launch; a Linear-2 tile waits (bounded)
 //      until all Linear-1 tiles of its row have published their h rows.
+// An expert with at most 64 rows is computed with the operands swapped: each 128-row weight box is the MMA's M
+// side and the expert's rows, padded to a multiple of 16, its N side.  A tcgen05.mma costs 128 clocks at N = 256 but
+// 46 at N <= 32, so the two instructions per K step (one per weight box) take 92 clocks instead of 128; the
+// shared-memory stage is the same three boxes, only the MMA issue and the epilogue (lane = output column) differ.
 // Layers whose experts hold many rows run the CTA-pair variant further down (256-row tiles, cta_group::2).
 #include <cuda_bf16.h>
 
@@ -50,6 +54,7 @@ constexpr int kTmemCols = 512;
 constexpr int kChunkCols = 32;     // accumulator columns per tcgen05.ld = columns of one store tile
 constexpr int kRing = 4;           // tile codes the producer may publish ahead of the consumers
 constexpr int kHotBlocks = 2;      // experts with at least this many 128-row blocks count as tensor-bound
+constexpr int kSwapRows = 64;      // experts with at most this many rows run with swapped operands
 constexpr int kPhaseShift = 30;    // tile code = phase << 30 | index in the phase's tile list; -1 = no more tiles
 
 struct SharedTail {
@@ -60,6 +65,7 @@ struct SharedTail {
   uint64_t ring_full[kRing];
   uint64_t ring_empty[kRing];
   int32_t ring_tile[kRing];
+  int32_t ring_npad[kRing];         // 0, or the padded row count of a tile computed with swapped operands
   uint32_t tmem_base;
   volatile int abort_flag;
   volatile uint32_t mma_progress;   // K-blocks issued so far by the MMA warp (pacing clock)
@@ -113,6 +119,7 @@ struct Tile {
   int n0;        // first output column
   int w_row0;    // first row of the weight box in the [E*N, K] weight matrix
   int block;     // global index of the 128-row block (ready counter)
+  int n_pad;     // 0 for a 128-row tile; else operands are swapped and this is the row count padded to 16
 };
 
 // Largest e with prefix(e) <= q, prefix non-decreasing with prefix(0) = 0 and q < prefix(E).
@@ -136,6 +143,8 @@ __device__ __forceinline__ Tile make_tile(int phase, int e, int m_blk, int n_blk
   t.n0 = n_blk * d.out_cols_per_tile;
   t.w_row0 = e * d.N + t.n0;
   t.block = st->hot_prefix[e] + st->cold_prefix[e] + m_blk;
+  const int rows = t.row_end - p.offsets[e];                      // the whole expert
+  t.n_pad = rows <= kSwapRows ? ((rows + 15) & ~15) : 0;          // few rows: swapped operands (m_blk is 0 then)
   return t;
 }
 
@@ -294,6 +303,55 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
   }
 }
 
+// Drain an accumulator computed with swapped operands: this thread's TMEM lane is output column n0 + f (and
+// n0 + 128 + f for Linear-2's second weight box); accumulator column j is row row0 + j.  Few rows, so plain 2-byte
+// stores (a warp writes 64 contiguous bytes per row).  Not paced: these tiles are a few rows long.
+template <bool kGated, bool kFp8>
+__device__ __forceinline__ void drain_swapped(const Tile& t, const FfnParams& p, uint32_t t_addr, int f) {
+  const PhaseDesc& d = p.ph[kGated ? 0 : 1];
+  const int col_a = t.n0 + f;
+  const int col_b = col_a + 128;
+  float sa = 1.f, sb = 1.f;                       // column scales of this lane's weight rows (E4M3 operands)
+  if constexpr (kFp8) {
+    if (kGated) {
+      if (col_a < d.N) { sa = d.col_scale0[t.w_row0 + f]; sb = d.col_scale1[t.w_row0 + f]; }
+    } else {
+      if (col_a < d.N) sa = d.col_scale0[t.w_row0 + f];
+      if (col_b < d.N) sb = d.col_scale0[t.w_row0 + 128 + f];
+    }
+  }
+#pragma unroll 1
+  for (int j0 = 0; j0 < t.n_pad; j0 += 16) {
+    uint32_t va[16], vb[16];
+    ptx::tmem_ld_32x16(t_addr + j0, va);
+    ptx::tmem_ld_32x16(t_addr + 128 + j0, vb);
+    ptx::tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int r = t.row0 + j0 + i;
+      if (r < t.row_end) {
+        float a = __uint_as_float(va[i]), b = __uint_as_float(vb[i]);
+        if constexpr (kFp8) {
+          const float rs = d.row_scale[r];
+          a *= rs * sa;
+          b *= rs * sb;
+        }
+        const size_t base = static_cast<size_t>(r) * d.N;
+        if constexpr (kGated) {
+          if (col_a < d.N) {
+            const float hv = silu_mul(a, b);
+            d.out[base + col_a] = __float2bfloat16_rn(hv);
+            if (p.h_dbg != nullptr) p.h_dbg[base + col_a] = hv;
+          }
+        } else {
+          if (col_a < d.N) d.out[base + col_a] = __float2bfloat16_rn(a);
+          if (col_b < d.N) d.out[base + col_b] = __float2bfloat16_rn(b);
+        }
+      }
+    }
+  }
+}
+
 template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wg,
@@ -411,11 +469,13 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           else if (pos < tiles1 + tiles2) code = (1 << kPhaseShift) | (pos - tiles1);
         }
         if (p.order_log && n_drawn < kMoeOrderLogCap) p.order_log[blockIdx.x * kMoeOrderLogCap + n_drawn++] = code;
+        Tile t{};
+        if (code >= 0) t = decode_tile(code, st, p);
         st->ring_tile[slot] = code;
+        st->ring_npad[slot] = t.n_pad;
         ptx::mbar_arrive(ptx::smem_u32(&st->ring_full[slot]));
         if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
         if (code < 0) break;
-        const Tile t = decode_tile(code, st, p);
         const PhaseDesc& d = p.ph[t.phase];
         const CUtensorMap* ma = t.phase == 0 ? &tm_x : &tm_h;
         const CUtensorMap* mb0 = t.phase == 0 ? &tm_wg : &tm_wd;
@@ -469,10 +529,12 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           break;
         }
         const int code = st->ring_tile[slot];
+        const int n_pad = st->ring_npad[slot];
         ptx::mbar_arrive(ptx::smem_u32(&st->ring_empty[slot]));
         if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
         if (code < 0) break;
         const int k_blocks = p.ph[code >> kPhaseShift].k_blocks;
+        const uint32_t idesc_swap = kFp8 ? ptx::idesc_e4m3_f32(BM, n_pad) : ptx::idesc_bf16_f32(BM, n_pad);
         if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, &w_tmem)) {
           report_timeout(p, 2);
           break;
@@ -490,13 +552,31 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           const uint32_t sa = stage_u32 + stage * kStageBytes;
           const uint64_t a_desc = ptx::smem_desc_sw128(sa);
           const uint64_t b_desc = ptx::smem_desc_sw128(sa + kABytes);
+          if (n_pad == 0) {
 #pragma unroll
-          for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
-            // +32 bytes along K inside the swizzle row = +2 in the descriptor's 16-byte address units
-            // (16 bf16 or 32 E4M3 elements per instruction: 32 bytes either way)
-            const uint64_t adv = static_cast<uint64_t>(2 * k4);
-            if constexpr (kFp8) ptx::tc_mma_e4m3(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
-            else ptx::tc_mma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
+            for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
+              // +32 bytes along K inside the swizzle row = +2 in the descriptor's 16-byte address units
+              // (16 bf16 or 32 E4M3 elements per instruction: 32 bytes either way)
+              const uint64_t adv = static_cast<uint64_t>(2 * k4);
+              if constexpr (kFp8) ptx::tc_mma_e4m3(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
+              else ptx::tc_mma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
+            }
+          } else {
+            // swapped operands: each 128-row weight box is the M side, the expert's rows (first box) the N side;
+            // the first weight box accumulates into columns 0.., the second into columns 128..
+            const uint64_t w1_desc = ptx::smem_desc_sw128(sa + kABytes + kBHalfBytes);
+#pragma unroll
+            for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
+              const uint64_t adv = static_cast<uint64_t>(2 * k4);
+              const uint32_t accum = (kb | k4) != 0 ? 1u : 0u;
+              if constexpr (kFp8) {
+                ptx::tc_mma_e4m3(d_tmem, b_desc + adv, a_desc + adv, idesc_swap, accum);
+                ptx::tc_mma_e4m3(d_tmem + 128u, w1_desc + adv, a_desc + adv, idesc_swap, accum);
+              } else {
+                ptx::tc_mma_bf16(d_tmem, b_desc + adv, a_desc + adv, idesc_swap, accum);
+                ptx::tc_mma_bf16(d_tmem + 128u, w1_desc + adv, a_desc + adv, idesc_swap, accum);
+              }
+            }
           }
           ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // stage is free once these MMAs have read it
           st->mma_progress = ++progress;
@@ -544,12 +624,16 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       const long long t_store = clock64();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               static_cast<uint32_t>(acc * BN_ACC);
-      if (t.phase == 0)
+      if (t.n_pad != 0) {
+        if (t.phase == 0) drain_swapped<true, kFp8>(t, p, t_addr, r_in_tile);
+        else drain_swapped<false, kFp8>(t, p, t_addr, r_in_tile);
+      } else if (t.phase == 0) {
         drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
                                       abort_flag);
-      else
+      } else {
         drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
                                        abort_flag);
+      }
       ptx::tc_fence_before_sync();
       if (chained && t.phase == 0) {
         // publish this warp's 32 rows x 128 columns of h to the Linear-2 tiles of the block
@@ -638,6 +722,7 @@ __device__ __forceinline__ Tile decode_pair_tile(int tile, int phase, uint32_t r
   t.n0 = n_blk * d.out_cols_per_tile;
   t.w_row0 = e * d.N + t.n0;
   t.block = 0;
+  t.n_pad = 0;
   return t;
 }
 
