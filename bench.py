@@ -177,6 +177,8 @@ def main():
                     help="print SM clocks per tcgen05.mma for several tile shapes (tensor-pipe calibration) and exit")
     ap.add_argument("--fp8", action="store_true",
                     help="time the FP8 (E4M3, W8A8) variant of the layer instead (weights quantised on the GPU first)")
+    ap.add_argument("--router", action="store_true",
+                    help="time the router front end (logits + top-k in one kernel, then the plan) on --config's shape")
     ap.add_argument("--xstage-probe", action="store_true",
                     help="run the burst/gap store microbenchmark on local HBM, print the rows and the calibration, exit")
     ap.add_argument("--trace", action="store_true",
@@ -211,6 +213,9 @@ def main():
         return
     if args.xstage_probe:
         run_xstage_probe(dev)
+        return
+    if args.router:
+        run_router(args, cfg, binding, local_rank, dev)
         return
     replicas.init_process_group(world, "nccl", torch.device(dev))
 
@@ -568,6 +573,79 @@ def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         "gpu_launches": ctx.moe_last_launch_count() * args.steps,
     }
     print(json.dumps(line), flush=True)
+
+
+def run_router(args, cfg, binding, local_rank, dev):
+    """Router front end alone: x and the prepared router weights resident on the device."""
+    import torch
+    x_bits = gen.make_x(cfg)
+    w_router = gen.make_router(cfg)
+    bias = gen.zipf_log_bias(cfg.E).astype(np.float32) if cfg.router == "xWr_zipf" else None
+    ctx = binding.Context(cfg.T, cfg.H, cfg.F, cfg.E, cfg.k, device=local_rank)
+    x = torch.from_numpy(np.ascontiguousarray(x_bits).view(np.int16)).to(dev).view(torch.bfloat16)
+    d_w = torch.from_numpy(w_router).to(dev)
+    d_bias = torch.from_numpy(bias).to(dev) if bias is not None else None
+    w_split = torch.zeros(ctx.router_weight_bytes() // 2, dtype=torch.bfloat16, device=dev)
+    scratch = torch.empty(ctx.router_scratch_bytes() // 4, device=dev)
+    ctx.moe_router_prepare(d_w, w_split)
+    R = cfg.T * cfg.k
+    i32 = dict(dtype=torch.int32, device=dev)
+    ids, w = torch.empty((cfg.T, cfg.k), **i32), torch.empty((cfg.T, cfg.k), device=dev)
+    counts, offsets = torch.empty(cfg.E, **i32), torch.empty(cfg.E + 1, **i32)
+    perm, inv_perm = torch.empty(R, **i32), torch.empty(R, **i32)
+    logits = torch.empty((cfg.T, cfg.E), device=dev)
+    # several copies of x, more than L2 in total, used in turn: every timed call reads its activations from HBM while
+    # the calls queue back to back (no host gap inside the timed region)
+    n_rot = max(2, -(-(256 << 20) // max(1, x.numel() * 2)))
+    n_rot = min(n_rot, 64)
+    xs = [x] + [x.clone() for _ in range(n_rot - 1)]
+    l2_note = (f"{n_rot} copies of x used in turn ({n_rot * x.numel() * 2 >> 20} MiB)" if n_rot * x.numel() * 2 >= (256 << 20)
+               else f"{n_rot} copies of x used in turn; they fit in L2 (warm)")
+    ctx.moe_route_tokens(x, w_split, d_bias, scratch, logits, ids, w, counts, offsets, perm, inv_perm)
+    routed = lambda i, st=None: ctx.moe_route_tokens(xs[i % n_rot], w_split, d_bias, scratch, None, ids, w, counts,
+                                                     offsets, perm, inv_perm, stream=st)
+    plain = lambda i, st=None: ctx.moe_plan_routing(logits, ids, w, counts, offsets, perm, inv_perm, stream=st)
+    rows = {}
+    stream = torch.cuda.current_stream()
+    for name, fn in (("route_tokens", routed), ("plan_routing_from_logits", plain)):
+        for i in range(args.warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        # one CUDA graph holding n_rot calls (each on its own copy of x): replaying it keeps the host's launch cost
+        # out of the timed region, which for calls this short would otherwise be most of it
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            g.capture_begin()
+            for i in range(n_rot):
+                fn(i, side)
+            g.capture_end()
+        torch.cuda.synchronize()
+        for _ in range(args.warmup):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            g.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        rows[name] = {"call_us": e0.elapsed_time(e1) * 1e3 / (args.steps * n_rot)}
+    code, detail = ctx.moe_last_device_status()
+    epad = ctx.router_weight_bytes() // (2 * cfg.H * 2)
+    alg_bytes = 2 * cfg.T * cfg.H + 2 * 2 * epad * cfg.H + 8 * R
+    # the calls share the plan's scan and scatter; what the front end adds is the difference
+    us = rows["route_tokens"]["call_us"]
+    peaks, peaks_src = load_peaks()
+    print(json.dumps({
+        "router": True, "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k,
+                                   "l2": l2_note},
+        "steps": args.steps, "warmup": args.warmup, "dtype": "bf16 x (2 bf16 terms of fp32 W_r), fp32 accumulate",
+        "timings": rows, "device_status": code,
+        "route_tokens_call": {"us": us, "algorithmic_bytes": alg_bytes, "GBps": alg_bytes / us * 1e-3,
+                          "frac_hbm": alg_bytes / us * 1e-3 / peaks["hbm_gbs"], "peaks": peaks_src,
+                          "tflops_bf16_issued": 2.0 * 2 * cfg.T * cfg.H * epad / us * 1e-6},
+    }), flush=True)
 
 
 def run_xstage_probe(dev):

@@ -180,6 +180,37 @@ moe_status moe_plan_routing_static(const moe_shape* shape, const float* logits, 
                                    int32_t* inv_perm, void* stream);
 
 /*
+ * Router front end: the step before the Dispatch bookkeeping of Sec. 4.3, for callers that hold the router matrix
+ * instead of logits.  The paper does not change the router (Sec. 7) and gives no kernel for it; the operation is
+ *     logits[t,e] = sum_c x[t,c] * w_router[c,e] (+ bias[e]),
+ * followed by the plan of moe_plan_routing on those logits.
+ *
+ * moe_router_prepare splits w_router [H,E] fp32 (device) once into two bf16 terms (the bf16 rounding of the value
+ * and the bf16 rounding of the remainder: 16 significant bits, relative error below 2^-17), stored as [2][Epad][H]
+ * with H contiguous and the expert rows padded to Epad (a multiple of 16, of 128 above 128 experts; padding rows are
+ * zero); w_split (device, caller-owned) holds moe_router_weight_bytes bytes.  With bf16 x every partial product is
+ * exact in fp32; what separates the logits from an fp64 product is the tensor path's fp32 accumulation (about 2^-24
+ * of the running sum per instruction) and the bits the split drops: |delta| <= 1e-4 * (1 + |logit|) for H <= 8192
+ * on N(0,1) data (about 6e-5 at H = 7168).
+ *
+ * moe_route_tokens computes the logits on the bf16 tensor path and selects the top k per token in the same kernel,
+ * on the fp32 logits it computed, with the rules of moe_plan_routing (ties to the lower expert index, softmax over
+ * the k selected logits); counts, offsets, perm and inv_perm follow as in moe_plan_routing_from_topk.  The result
+ * is bit-identical to moe_plan_routing applied to the returned logits, and run-to-run deterministic.
+ *   x [T,H] bf16, w_split from moe_router_prepare, bias [E] fp32 or NULL,
+ *   scratch: device, at least moe_router_scratch_bytes bytes (partial sums of the K split; contents undefined after),
+ *   logits_out: NULL, or fp32 [T,E] that receives the logits the selection used,
+ *   -> topk_ids, topk_w, counts, offsets, perm, inv_perm as moe_plan_routing.
+ * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL (scratch), CUDA; TIMEOUT through the status word (detail 101-103).
+ */
+size_t moe_router_weight_bytes(const moe_shape* shape);
+size_t moe_router_scratch_bytes(const moe_shape* shape);
+moe_status moe_router_prepare(moe_ctx* ctx, const float* w_router, void* w_split, void* stream);
+moe_status moe_route_tokens(moe_ctx* ctx, const void* x, const void* w_split, const float* bias, void* scratch,
+                            size_t scratch_bytes, float* logits_out, int32_t* topk_ids, float* topk_w,
+                            int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* stream);
+
+/*
  * Dispatch (Sec. 2.2 / Sec. 4.3 "Dispatch input"): x_perm[inv_perm[t*k+j], :] = x[t, :] for every slot,
  * i.e. x_perm[row, :] = x[perm[row] div k, :].  Each token row is read once and written k times with
  * 16-byte accesses.   x [T,H] bf16, inv_perm [R] int32 -> x_perm [R,H] bf16 (bit-exact copies).
@@ -222,7 +253,17 @@ moe_status moe_fused_forward(moe_ctx* ctx, const void* x, const float* logits, c
                              size_t workspace_bytes, const moe_tuning* tuning, void* stream);
 
 /*
- * Same, with the per-step tensors in HOST memory (pinned memory makes the copies asynchronous):
+ * The whole layer starting from the router matrix: moe_route_tokens (logits not kept), dispatch, expert_ffn,
+ * combine on one stream.  w_split from moe_router_prepare; bias [E] fp32 or NULL; router_scratch as the scratch of
+ * moe_route_tokens (at least moe_router_scratch_bytes bytes); everything else as moe_fused_forward.
+ */
+moe_status moe_fused_forward_routed(moe_ctx* ctx, const void* x, const void* w_split, const float* bias,
+                                    const void* w_gate, const void* w_up, const void* w_down, void* out,
+                                    void* workspace, size_t workspace_bytes, void* router_scratch,
+                                    size_t router_scratch_bytes, const moe_tuning* tuning, void* stream);
+
+/*
+ * moe_fused_forward with the per-step tensors in HOST memory (pinned memory makes the copies asynchronous):
  * x_host [T,H] bf16 and logits_host [T,E] fp32 are copied to the workspace's staging slices, the layer
  * runs, and out [T,H] bf16 is copied back to out_host, all on `stream`.  Expert weights stay on the
  * device.  The caller synchronises the stream before reading out_host.

@@ -26,7 +26,8 @@ EXPORTS = (
     "moe_get_kernel_times", "moe_plan_routing_static", "moe_get_ffn_trace", "moe_probe_mma_cycles",
     "moe_get_ffn_order", "moe_fused_forward_host_pipelined", "moe_host_pipeline_flush", "moe_quantize_rows",
     "moe_dispatch_fp8", "moe_expert_ffn_fp8", "moe_get_workspace_layout_fp8", "moe_fused_forward_fp8",
-    "moe_set_active_tokens", "moe_plan_routing_from_topk",
+    "moe_set_active_tokens", "moe_plan_routing_from_topk", "moe_router_weight_bytes", "moe_router_scratch_bytes",
+    "moe_router_prepare", "moe_route_tokens", "moe_fused_forward_routed",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -106,6 +107,14 @@ def load_library() -> C.CDLL:
                                           C.POINTER(moe_tuning), vp]
     lib.moe_set_active_tokens.argtypes = [vp, C.c_int32]
     lib.moe_plan_routing_from_topk.argtypes = [vp, i32p, i32p, i32p, i32p, i32p, i32p, vp]
+    lib.moe_router_weight_bytes.argtypes = [C.POINTER(moe_shape)]
+    lib.moe_router_weight_bytes.restype = C.c_size_t
+    lib.moe_router_scratch_bytes.argtypes = [C.POINTER(moe_shape)]
+    lib.moe_router_scratch_bytes.restype = C.c_size_t
+    lib.moe_router_prepare.argtypes = [vp, f32p, vp, vp]
+    lib.moe_route_tokens.argtypes = [vp, vp, vp, f32p, vp, C.c_size_t, f32p, i32p, f32p, i32p, i32p, i32p, i32p, vp]
+    lib.moe_fused_forward_routed.argtypes = [vp, vp, vp, f32p, vp, vp, vp, vp, vp, C.c_size_t, vp, C.c_size_t,
+                                             C.POINTER(moe_tuning), vp]
     lib.moe_last_device_status.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_last_launch_count.argtypes = [vp]
     lib.moe_last_launch_count.restype = C.c_int32
@@ -115,7 +124,8 @@ def load_library() -> C.CDLL:
     lib.moe_get_ffn_order.argtypes = [vp, C.POINTER(C.c_int32), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_get_ffn_trace.argtypes = [vp, C.POINTER(C.c_uint64), C.c_int32, C.POINTER(C.c_int32), vp]
     for name in EXPORTS:
-        if name not in ("moe_status_string", "moe_destroy", "moe_workspace_bytes", "moe_last_launch_count"):
+        if name not in ("moe_status_string", "moe_destroy", "moe_workspace_bytes", "moe_last_launch_count",
+                        "moe_router_weight_bytes", "moe_router_scratch_bytes"):
             getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -233,6 +243,36 @@ class Context:
         _check(self._lib.moe_plan_routing_from_topk(self._handle, _ptr(topk_ids), _ptr(topk_ids_checked), _ptr(counts),
                                                     _ptr(offsets), _ptr(perm), _ptr(inv_perm), _stream(stream)),
                "moe_plan_routing_from_topk")
+
+    def _shape(self):
+        return moe_shape(self.T, self.H, self.F, self.E, self.k, self.ep_size, self.ep_rank)
+
+    def router_weight_bytes(self) -> int:
+        """Bytes of the prepared router weights (three bf16 terms of W_r, expert rows padded)."""
+        return int(self._lib.moe_router_weight_bytes(C.byref(self._shape())))
+
+    def router_scratch_bytes(self) -> int:
+        """Bytes of the scratch moe_route_tokens needs for the K-split partial logits."""
+        return int(self._lib.moe_router_scratch_bytes(C.byref(self._shape())))
+
+    def moe_router_prepare(self, w_router, w_split, stream=None):
+        _check(self._lib.moe_router_prepare(self._handle, _ptr(w_router), _ptr(w_split), _stream(stream)),
+               "moe_router_prepare")
+
+    def moe_route_tokens(self, x, w_split, bias, scratch, logits_out, topk_ids, topk_w, counts, offsets, perm,
+                         inv_perm, stream=None):
+        _check(self._lib.moe_route_tokens(self._handle, _ptr(x), _ptr(w_split), _ptr(bias), _ptr(scratch),
+                                          scratch.numel() * scratch.element_size(), _ptr(logits_out), _ptr(topk_ids),
+                                          _ptr(topk_w), _ptr(counts), _ptr(offsets), _ptr(perm), _ptr(inv_perm),
+                                          _stream(stream)), "moe_route_tokens")
+
+    def moe_fused_forward_routed(self, x, w_split, bias, w_gate, w_up, w_down, out, workspace, router_scratch,
+                                 tuning=None, stream=None):
+        _check(self._lib.moe_fused_forward_routed(self._handle, _ptr(x), _ptr(w_split), _ptr(bias), _ptr(w_gate),
+                                                  _ptr(w_up), _ptr(w_down), _ptr(out), _ptr(workspace),
+                                                  workspace.numel() * workspace.element_size(), _ptr(router_scratch),
+                                                  router_scratch.numel() * router_scratch.element_size(),
+                                                  _tuning_ref(tuning), _stream(stream)), "moe_fused_forward_routed")
 
     def moe_dispatch(self, x, inv_perm, x_perm, stream=None):
         _check(self._lib.moe_dispatch(self._handle, _ptr(x), _ptr(inv_perm), _ptr(x_perm), _stream(stream)),

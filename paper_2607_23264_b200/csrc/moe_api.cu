@@ -161,7 +161,11 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   ok = ok && cudaMemset(ctx->d_ready, 0, ready_bytes) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_sched, 4 * 4) == cudaSuccess;
   ok = ok && cudaMemset(ctx->d_sched, 0, 4 * 4) == cudaSuccess;
+  const size_t done_bytes = static_cast<size_t>(shape->T / 128 + 2) * 4;
+  ok = ok && cudaMalloc(&ctx->d_router_done, done_bytes) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->d_router_done, 0, done_bytes) == cudaSuccess;
   ok = ok && moe::prepare_expert_ffn(ctx) == cudaSuccess;
+  ok = ok && moe::prepare_router(ctx) == cudaSuccess;
   for (int i = 0; ok && i <= kMoeKernels; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) == cudaSuccess;
@@ -194,6 +198,7 @@ void moe_destroy(moe_ctx* ctx) {
   if (ctx->d_trace) cudaFree(ctx->d_trace);
   if (ctx->d_ready) cudaFree(ctx->d_ready);
   if (ctx->d_order) cudaFree(ctx->d_order);
+  if (ctx->d_router_done) cudaFree(ctx->d_router_done);
   for (int i = 0; i <= kMoeKernels; ++i)
     if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
   for (int i = 0; i < 2; ++i) {
@@ -325,6 +330,98 @@ moe_status moe_fused_forward(moe_ctx* ctx, const void* x, const float* logits, c
 
   begin_call(ctx, 0, stream);
   if (moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (moe::launch_dispatch(ctx, x, inv_perm, x_perm, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  st = moe::launch_expert_ffn(ctx, x_perm, offsets, w_gate, w_up, w_down, h, y_perm, nullptr, tuning, cs);
+  if (st != MOE_OK) return st;
+  if (moe::launch_combine(ctx, y_perm, inv_perm, topk_w, out, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ router front end
+
+size_t moe_router_weight_bytes(const moe_shape* shape) {
+  return check_shape(shape) == MOE_OK ? moe::router_weight_bytes(*shape) : 0;
+}
+
+size_t moe_router_scratch_bytes(const moe_shape* shape) {
+  return check_shape(shape) == MOE_OK ? moe::router_scratch_bytes(*shape) : 0;
+}
+
+moe_status moe_router_prepare(moe_ctx* ctx, const float* w_router, void* w_split, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  ctx->last_launches = 0;
+  if (!w_router || !w_split || !aligned16(w_router) || !aligned16(w_split)) return MOE_ERR_INVALID_ARG;
+  return moe::launch_router_prepare(ctx, w_router, w_split, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_route_tokens(moe_ctx* ctx, const void* x, const void* w_split, const float* bias, void* scratch,
+                            size_t scratch_bytes, float* logits_out, int32_t* topk_ids, float* topk_w,
+                            int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  begin_call(ctx, 0, stream);
+  const moe_shape& s = ctx->shape;
+  if (!counts || !offsets) return MOE_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (s.T == 0) {
+    if (cudaMemsetAsync(counts, 0, static_cast<size_t>(s.E) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaMemsetAsync(offsets, 0, static_cast<size_t>(s.E + 1) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+  }
+  if (!x || !w_split || !scratch || !topk_ids || !topk_w || !perm || !inv_perm) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(w_split) || !aligned16(bias) || !aligned16(scratch) || !aligned16(logits_out) ||
+      !aligned16(topk_ids) || !aligned16(topk_w) || !aligned16(counts) || !aligned16(offsets) || !aligned16(perm) ||
+      !aligned16(inv_perm))
+    return MOE_ERR_INVALID_ARG;
+  if (scratch_bytes < moe::router_scratch_bytes(s)) return MOE_ERR_WORKSPACE_TOO_SMALL;
+  st = moe::launch_router(ctx, x, w_split, bias, scratch, logits_out, topk_ids, topk_w, cs);
+  if (st != MOE_OK) return st;
+  return moe::launch_plan_from_topk(ctx, topk_ids, topk_ids, counts, offsets, perm, inv_perm, cs) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_fused_forward_routed(moe_ctx* ctx, const void* x, const void* w_split, const float* bias,
+                                    const void* w_gate, const void* w_up, const void* w_down, void* out,
+                                    void* workspace, size_t workspace_bytes, void* router_scratch,
+                                    size_t router_scratch_bytes, const moe_tuning* tuning, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  st = check_tuning(tuning);
+  if (st != MOE_OK) return st;
+  const moe_shape& s = ctx->shape;
+  if (s.T == 0) { ctx->last_launches = 0; return MOE_OK; }
+  if (!x || !w_split || !w_gate || !w_up || !w_down || !out || !workspace || !router_scratch)
+    return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(w_split) || !aligned16(bias) || !aligned16(w_gate) || !aligned16(w_up) ||
+      !aligned16(w_down) || !aligned16(out) || !aligned16(router_scratch) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+    return MOE_ERR_INVALID_ARG;
+  moe_workspace_layout L;
+  fill_layout(s, &L);
+  if (workspace_bytes < L.total || router_scratch_bytes < moe::router_scratch_bytes(s))
+    return MOE_ERR_WORKSPACE_TOO_SMALL;
+
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  int32_t* topk_ids = reinterpret_cast<int32_t*>(ws + L.topk_ids);
+  float* topk_w = reinterpret_cast<float*>(ws + L.topk_w);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+  int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
+  int32_t* perm = reinterpret_cast<int32_t*>(ws + L.perm);
+  int32_t* inv_perm = reinterpret_cast<int32_t*>(ws + L.inv_perm);
+  void* x_perm = ws + L.x_perm;
+  void* h = ws + L.h;
+  void* y_perm = ws + L.y_perm;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+  begin_call(ctx, 0, stream);
+  st = moe::launch_router(ctx, x, w_split, bias, router_scratch, nullptr, topk_ids, topk_w, cs);
+  if (st != MOE_OK) return st;
+  if (moe::launch_plan_from_topk(ctx, topk_ids, topk_ids, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
     return MOE_ERR_CUDA;
   if (moe::launch_dispatch(ctx, x, inv_perm, x_perm, cs) != cudaSuccess) return MOE_ERR_CUDA;
   st = moe::launch_expert_ffn(ctx, x_perm, offsets, w_gate, w_up, w_down, h, y_perm, nullptr, tuning, cs);

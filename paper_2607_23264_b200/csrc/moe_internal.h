@@ -36,6 +36,7 @@ struct moe_ctx {
   int32_t* d_status;      // [2] device status word: code, detail
   int32_t* d_sched;       // [4] tile scheduler of the two grouped GEMMs: {next tile, CTAs done} each; zero when idle
   int32_t* d_ready;       // [T*k/128 + E + 1] per 128-row block: Linear-1 warps that published its h rows; zero when idle
+  int32_t* d_router_done; // [1 + T/128 + 1] router front end: work ticket, then partial tiles written per row tile
   int32_t* d_order;       // [num_sms][kMoeOrderLogCap] tile codes drawn by each CTA in the last traced one-launch run
   unsigned long long* d_trace;   // [2][num_sms][kMoeTraceFields] wait counters of Linear-1 and Linear-2
   moe_encode_tiled_fn encode_tiled;
@@ -87,6 +88,16 @@ cudaError_t launch_quantize_rows(moe_ctx* ctx, const void* in_bf16, long long ro
 // Row mover for E4M3 rows with their scales: xq_perm[inv_perm[t*k+j]] = xq[t], sx_perm[..] = sx[t].
 cudaError_t launch_dispatch_fp8(moe_ctx* ctx, const void* xq, const float* sx, const int32_t* inv_perm,
                                 void* xq_perm, float* sx_perm, cudaStream_t stream);
+
+// Router front end.  Sizes of the prepared weights (three bf16 terms of W_r, expert rows padded) and of the scratch
+// for the K-split partial logits; the split of W_r; logits + top-k in one kernel (ids and weights only: the plan's
+// histogram, scan and scatter follow through launch_plan_from_topk).
+size_t router_weight_bytes(const moe_shape& s);
+size_t router_scratch_bytes(const moe_shape& s);
+cudaError_t launch_router_prepare(moe_ctx* ctx, const float* w_router, void* w_split, cudaStream_t stream);
+moe_status launch_router(moe_ctx* ctx, const void* x, const void* w_split, const float* bias, void* scratch,
+                         float* logits_out, int32_t* topk_ids, float* topk_w, cudaStream_t stream);
+cudaError_t prepare_router(moe_ctx* ctx);      // one-time kernel attributes
 
 cudaError_t prepare_expert_ffn(moe_ctx* ctx);  // one-time kernel attributes (dynamic shared memory size)
 

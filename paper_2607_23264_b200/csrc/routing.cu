@@ -2,8 +2,8 @@
 //
 // The token range is cut into chunks of `tokens_per_chunk` tokens (at most 256 slots).  Three launches:
 //   1. route_topk_hist : one CTA per chunk; a warp per token selects the k largest logits by k passes of
-//                        warp arg-max (shuffle reduction, ties to the lower index) and computes the
-//                        softmax weights; the CTA then histograms its slots per expert.
+//                        warp arg-max (integer warp reductions on order-preserving keys, ties to the lower
+//                        index) and computes the softmax weights; the CTA then histograms its slots per expert.
 //   2. route_scan      : one CTA; exclusive prefix of the chunk histograms over chunks (per expert) and
 //                        the exclusive scan of the totals over experts (offsets).
 //   3. route_scatter   : one CTA per chunk, one thread per slot; the stable rank of a slot among the
@@ -12,6 +12,7 @@
 // Everything is integer work on identical fp32 inputs, so ids, counts, offsets and both permutations are
 // reproducible bit for bit.
 #include "moe_internal.h"
+#include "route_select.cuh"
 
 namespace {
 
@@ -22,8 +23,7 @@ route_topk_hist(const float* __restrict__ logits, int T, int E, int k, int token
                 int32_t* __restrict__ topk_ids, float* __restrict__ topk_w, int32_t* __restrict__ chunk_hist) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int warps = kRouteThreads / 32;
-  float* s_logit = reinterpret_cast<float*>(smem_raw);                    // [warps][E]
-  int32_t* s_hist = reinterpret_cast<int32_t*>(s_logit + warps * E);      // [E]
+  int32_t* s_hist = reinterpret_cast<int32_t*>(smem_raw);                 // [E]
   int32_t* s_ids = s_hist + E;                                            // [256]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -33,43 +33,16 @@ route_topk_hist(const float* __restrict__ logits, int T, int E, int k, int token
 
   for (int e = tid; e < E; e += kRouteThreads) s_hist[e] = 0;
 
-  float* my = s_logit + warp * E;
   for (int t = t_begin + warp; t < t_end; t += warps) {
-    const float* row = logits + static_cast<size_t>(t) * E;
-    for (int e = lane; e < E; e += 32) my[e] = row[e];
-    __syncwarp();
-    float sel_logit = 0.f;   // lane j keeps the logit picked in pass j
-    int sel_id = 0;
-    for (int j = 0; j < k; ++j) {
-      float best = -INFINITY;
-      int best_e = 0x7FFFFFFF;
-      for (int e = lane; e < E; e += 32) {      // ascending e with strict '>' keeps the lowest index
-        const float v = my[e];
-        if (v > best) { best = v; best_e = e; }
-      }
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        const float ov = __shfl_xor_sync(kFull, best, off);
-        const int oe = __shfl_xor_sync(kFull, best_e, off);
-        if (ov > best || (ov == best && oe < best_e)) { best = ov; best_e = oe; }
-      }
-      if (lane == j) { sel_logit = best; sel_id = best_e; }
-      if (lane == 0) my[best_e] = -INFINITY;    // taken
-      __syncwarp();
-    }
-    // softmax over the k selected logits; pass 0 picked the maximum
-    const float m = __shfl_sync(kFull, sel_logit, 0);
-    float p = (lane < k) ? expf(sel_logit - m) : 0.f;
-    float sum = p;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
+    int sel_id;
+    float sel_w;
+    moe::warp_select_topk(logits + static_cast<size_t>(t) * E, E, k, lane, &sel_id, &sel_w);
     if (lane < k) {
       const size_t s = static_cast<size_t>(t) * k + lane;
       topk_ids[s] = sel_id;
-      topk_w[s] = p / sum;
+      topk_w[s] = sel_w;
       s_ids[(t - t_begin) * k + lane] = sel_id;
     }
-    __syncwarp();
   }
   __syncthreads();
   const int n_slots = (t_end - t_begin) * k;
@@ -199,7 +172,7 @@ cudaError_t launch_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk
                                 cudaStream_t stream) {
   const moe_shape& s = ctx->shape;
   const int warps = kRouteThreads / 32;
-  const size_t smem1 = (static_cast<size_t>(warps) * s.E + s.E + 256) * 4;
+  const size_t smem1 = (static_cast<size_t>(s.E) + 256) * 4;
   const size_t smem3 = static_cast<size_t>(warps) * s.E * 4;
   route_topk_hist<<<ctx->num_chunks, kRouteThreads, smem1, stream>>>(logits, s.T, s.E, s.k, ctx->tokens_per_chunk,
                                                                      topk_ids, topk_w, ctx->d_chunk_hist);
@@ -219,9 +192,12 @@ cudaError_t launch_plan_from_topk(moe_ctx* ctx, const int32_t* topk_ids, int32_t
   const int warps = kRouteThreads / 32;
   route_hist_ids<<<ctx->num_chunks, kRouteThreads, static_cast<size_t>(s.E) * 4, stream>>>(
       topk_ids, s.T, s.E, s.k, ctx->tokens_per_chunk, ids_checked, ctx->d_chunk_hist, ctx->d_status);
+  moe_mark(ctx, 1, stream);
   route_scan<<<1, 1024, 0, stream>>>(ctx->d_chunk_hist, ctx->d_chunk_base, ctx->num_chunks, s.E, counts, offsets);
+  moe_mark(ctx, 2, stream);
   route_scatter<<<ctx->num_chunks, kRouteThreads, static_cast<size_t>(warps) * s.E * 4, stream>>>(
       ids_checked, offsets, ctx->d_chunk_base, s.T, s.E, s.k, ctx->tokens_per_chunk, perm, inv_perm);
+  moe_mark(ctx, 3, stream);
   ctx->last_launches += 3;
   return cudaGetLastError();
 }
@@ -283,7 +259,7 @@ extern "C" moe_status moe_plan_routing_static(const moe_shape* shape, const floa
   int32_t* chunk_base = scratch + kStaticScratchInts;   // [num_chunks, E], every entry rewritten by kernel 2
 
   const int warps = kRouteThreads / 32;
-  const size_t smem1 = (static_cast<size_t>(warps) * E + E + 256) * 4;
+  const size_t smem1 = (static_cast<size_t>(E) + 256) * 4;
   const size_t smem3 = static_cast<size_t>(warps) * E * 4;
   const int nc = static_cast<int>(num_chunks);
   route_topk_hist<<<nc, kRouteThreads, smem1, cs>>>(logits, T, E, k, tokens_per_chunk, topk_ids, topk_w, chunk_hist);
