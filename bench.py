@@ -177,6 +177,8 @@ def main():
                     help="print SM clocks per tcgen05.mma for several tile shapes (tensor-pipe calibration) and exit")
     ap.add_argument("--fp8", action="store_true",
                     help="time the FP8 (E4M3, W8A8) variant of the layer instead (weights quantised on the GPU first)")
+    ap.add_argument("--mxfp8", action="store_true",
+                    help="the block-scaled FP8 variant of the experts (E4M3 elements, E8M0 scale per 32 elements along K)")
     ap.add_argument("--router", action="store_true",
                     help="time the router front end (logits + top-k in one kernel, then the plan) on --config's shape")
     ap.add_argument("--xstage-probe", action="store_true",
@@ -227,7 +229,7 @@ def main():
     w_gate = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
     w_up = torch.empty((cfg.E, cfg.F, cfg.H), dtype=torch.bfloat16, device=dev)
     w_down = torch.empty((cfg.E, cfg.H, cfg.F), dtype=torch.bfloat16, device=dev)
-    want_cpu = rank == 0 and world == 1 and not (args.no_cpu_baseline or args.sweep or args.profile or args.fp8)
+    want_cpu = rank == 0 and world == 1 and not (args.no_cpu_baseline or args.sweep or args.profile or args.fp8 or args.mxfp8)
     keep_host = want_cpu and cfg.E <= 16
     host_w = {}
 
@@ -267,6 +269,9 @@ def main():
         return
     if args.fp8:
         run_fp8(args, cfg, ctx, binding, (x, d_logits, w_gate, w_up, w_down, out), timed, rank, world, dev)
+        return
+    if args.mxfp8:
+        run_mxfp8(args, cfg, ctx, binding, (x, d_logits, w_gate, w_up, w_down, out), timed, rank, world, dev)
         return
 
     dbg = (2 if args.one_launch else 0) | {"auto": 0, "on": 8, "off": 16}[args.pairs]
@@ -569,6 +574,55 @@ def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
                        "quantize_h+linear2": km[5], "combine": km[6]},
         "roofline": {"kernel": "expert FFN Linear-1 launch, E4M3 operands", "bound": "tensor", "achieved": l1_tf,
                      "peak": peak, "unit": "TFLOP/s", "frac": l1_tf / peak, "traffic": None,
+                     "peak_source": f"2 x {kind} bf16_tflops (burst): nominal fp8 / bf16 ratio"},
+        "gpu_launches": ctx.moe_last_launch_count() * args.steps,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
+    """The block-scaled FP8 variant (MXFP8: E4M3 elements, E8M0 scale per 32 elements along K, applied inside the MMA)."""
+    import torch
+    x, d_logits, w_gate, w_up, w_down, out = bufs
+    wq = []
+    for w in (w_gate, w_up, w_down):
+        E, r, c = w.shape
+        codes = torch.empty((E * r, c), dtype=torch.uint8, device=dev)
+        words = torch.empty((c // 128, E * r), dtype=torch.int32, device=dev)
+        ctx.moe_quantize_rows_mx(w.view(E * r, c), E * r, c, codes, words)
+        wq += [codes, words]
+    torch.cuda.synchronize()
+    del w_gate, w_up, w_down
+    ws = torch.empty(ctx.workspace_layout_mx()["total"], dtype=torch.uint8, device=dev)
+    step = lambda: ctx.moe_fused_forward_mx(x, d_logits, *wq, out, ws)
+    ms = timed(step, args.steps, args.warmup) / args.steps
+    ctx.moe_set_kernel_timing(True)
+    per = []
+    for _ in range(args.steps):
+        step()
+        per.append(ctx.moe_get_kernel_times())
+    ctx.moe_set_kernel_timing(False)
+    km = [float(np.mean([p[i] for p in per])) for i in range(len(binding.KERNEL_NAMES))]
+    code, detail = ctx.moe_last_device_status()
+    if code != 0:
+        raise RuntimeError(f"device status {code} detail {detail:#x}")
+    if rank != 0:
+        return
+    peaks, kind = load_peaks()
+    peak = 2.0 * float(peaks["bf16_tflops"])      # E4M3 runs at twice the bf16 rate on this part (4.5 vs 2.25 PFLOP/s nominal)
+    R = cfg.R
+    l1_tf = 4 * R * cfg.H * cfg.F / (km[4] * 1e-3) / 1e12
+    tflops = cfg.flops * world / (ms * 1e-3) / 1e12
+    line = {
+        "metric": "fused MoE fwd tokens/s", "variant": "mxfp8 (E4M3 elements, E8M0 scale per 32 along K)",
+        "value": cfg.T * world / (ms * 1e-3),
+        "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "mxfp8_e4m3", "data": "synthetic",
+        "config": workload_config(cfg, world), "tflops": tflops, "frac_fp8_peak": tflops / world / peak,
+        "kernels_ms": {"routing": km[0] + km[1] + km[2], "quantize_x+dispatch": km[3], "linear1+quantize_h": km[4],
+                       "linear2": km[5], "combine": km[6]},
+        "roofline": {"kernel": "expert FFN Linear-1 launch, block-scaled E4M3 operands", "bound": "tensor",
+                     "achieved": l1_tf, "peak": peak, "unit": "TFLOP/s", "frac": l1_tf / peak, "traffic": None,
                      "peak_source": f"2 x {kind} bf16_tflops (burst): nominal fp8 / bf16 ratio"},
         "gpu_launches": ctx.moe_last_launch_count() * args.steps,
     }

@@ -333,6 +333,68 @@ moe_status moe_fused_forward_fp8(moe_ctx* ctx, const void* x, const float* logit
                                  const float* s_down, void* out, void* workspace, size_t workspace_bytes,
                                  const moe_tuning* tuning, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Block-scaled FP8 experts (MXFP8).  The paper's kernels are W8A8 / W4A8 (Sec. 5.3) and do not say how values are
+ * scaled; this is the block-scaled reading in the form the sm_100a tensor pipe applies inside the MMA: E4M3
+ * elements, 32 consecutive elements along K share a scale 2^e kept as the byte e + 127 (E8M0), e = the smallest
+ * integer with amax * 2^-e <= 448 (not below -127), code = convert(value * 2^-e) to nearest-even, never clipped.
+ * Scale bytes are stored four to a 32-bit word (the four blocks of a 128-element K stage, lowest block in the lowest
+ * byte), words as [K/128][rows].  H and F must be multiples of 128 (MOE_ERR_UNSUPPORTED_SHAPE otherwise).
+ * ------------------------------------------------------------------------------------------------ */
+
+/* in_bf16 [rows, cols] bf16 -> codes [rows, cols] E4M3 + sf_words [cols/128][rows] uint32.  cols % 128 == 0. */
+moe_status moe_quantize_rows_mx(moe_ctx* ctx, const void* in_bf16, int64_t rows, int32_t cols, void* codes,
+                                uint32_t* sf_words, void* stream);
+
+/* Dispatch of quantised token rows: xq_perm[inv_perm[t*k+j], :] = xq[t, :], sfx_perm[w][inv_perm[t*k+j]] = sfx[w][t].
+ *   xq [T,H] E4M3, sfx [H/128][T] -> xq_perm [R,H], sfx_perm [H/128][R]. */
+moe_status moe_dispatch_mx(moe_ctx* ctx, const void* xq, const uint32_t* sfx, const int32_t* inv_perm, void* xq_perm,
+                           uint32_t* sfx_perm, void* stream);
+
+typedef struct {
+  const void* xq_perm;      /* E4M3 [R,H] */
+  const uint32_t* sfx_perm; /* [H/128][R] */
+  const int32_t* offsets;   /* [E+1] */
+  const void* wq_gate;      /* E4M3 [E*F, H] */
+  const uint32_t* sf_gate;  /* [H/128][E*F] */
+  const void* wq_up;        /* E4M3 [E*F, H] */
+  const uint32_t* sf_up;    /* [H/128][E*F] */
+  const void* wq_down;      /* E4M3 [E*H, F] */
+  const uint32_t* sf_down;  /* [F/128][E*H] */
+  void* hq_ws;              /* out: E4M3 [R,F]: h = silu(gate) * up, quantised from its fp32 value (Linear-2 input) */
+  uint32_t* sfh_ws;         /* out: [F/128][R] */
+  void* y_perm;             /* out: bf16 [R,H] */
+  float* h_fp32_debug;      /* NULL, or fp32 [R,F] that receives h before its quantisation */
+} moe_mx_ffn_args;
+
+/* Linear-1 (block-scaled MMA, SiLU*mul, h quantised in the epilogue) and Linear-2 (-> y_perm bf16): two launches,
+ * 128 x 192 tiles, Expert-Wave order.  For expert e and its rows r, with deq() the dequantised operands:
+ *   h[r,f] = silu(sum_c deq(x)[r,c] deq(w_gate)[e,f,c]) * (sum_c deq(x)[r,c] deq(w_up)[e,f,c]),
+ *   y_perm[r,c] = sum_f deq(hq)[r,f] deq(w_down)[e,c,f]   (fp32 accumulation, bf16 out). */
+moe_status moe_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* args, void* stream);
+
+/* Byte offsets of the workspace slices of moe_fused_forward_mx (256-byte aligned). */
+typedef struct {
+  size_t topk_ids, topk_w, counts, offsets, perm, inv_perm;   /* as in moe_workspace_layout */
+  size_t xq;         /* E4M3 [T,H] */
+  size_t sfx;        /* uint32 [H/128][T] */
+  size_t xq_perm;    /* E4M3 [R,H] */
+  size_t sfx_perm;   /* uint32 [H/128][R] */
+  size_t hq;         /* E4M3 [R,F] */
+  size_t sfh;        /* uint32 [F/128][R] */
+  size_t y_perm;     /* bf16 [R,H] */
+  size_t total;
+} moe_workspace_layout_mx;
+moe_status moe_get_workspace_layout_mx(const moe_shape* shape, moe_workspace_layout_mx* out_layout);
+
+/* The whole layer with block-scaled FP8 experts on one stream: plan_routing, quantize x, dispatch_mx, expert_ffn_mx,
+ * combine.  x [T,H] bf16 and logits as in moe_fused_forward; weights pre-quantised (moe_quantize_rows_mx over the
+ * rows of each matrix: [E*F, H] for gate and up, [E*H, F] for down). */
+moe_status moe_fused_forward_mx(moe_ctx* ctx, const void* x, const float* logits, const void* wq_gate,
+                                const uint32_t* sf_gate, const void* wq_up, const uint32_t* sf_up, const void* wq_down,
+                                const uint32_t* sf_down, void* out, void* workspace, size_t workspace_bytes,
+                                void* stream);
+
 /*
  * The host-buffer call as a two-deep pipeline, for callers that run step after step (serving): consecutive calls
  * alternate between two staging slots, the input copy of call i+1 runs on an internal copy stream while call i

@@ -27,7 +27,8 @@ EXPORTS = (
     "moe_get_ffn_order", "moe_fused_forward_host_pipelined", "moe_host_pipeline_flush", "moe_quantize_rows",
     "moe_dispatch_fp8", "moe_expert_ffn_fp8", "moe_get_workspace_layout_fp8", "moe_fused_forward_fp8",
     "moe_set_active_tokens", "moe_plan_routing_from_topk", "moe_router_weight_bytes", "moe_router_scratch_bytes",
-    "moe_router_prepare", "moe_route_tokens", "moe_fused_forward_routed",
+    "moe_router_prepare", "moe_route_tokens", "moe_fused_forward_routed", "moe_quantize_rows_mx", "moe_dispatch_mx",
+    "moe_expert_ffn_mx", "moe_get_workspace_layout_mx", "moe_fused_forward_mx",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -66,6 +67,16 @@ class moe_fp8_ffn_args(C.Structure):
 class moe_workspace_layout_fp8(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in ("topk_ids", "topk_w", "counts", "offsets", "perm", "inv_perm", "xq", "sx",
                                           "xq_perm", "sx_perm", "h", "hq", "sh", "y_perm", "total")]
+
+
+class moe_mx_ffn_args(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("xq_perm", "sfx_perm", "offsets", "wq_gate", "sf_gate", "wq_up", "sf_up",
+                                          "wq_down", "sf_down", "hq_ws", "sfh_ws", "y_perm", "h_fp32_debug")]
+
+
+class moe_workspace_layout_mx(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("topk_ids", "topk_w", "counts", "offsets", "perm", "inv_perm", "xq", "sfx",
+                                          "xq_perm", "sfx_perm", "hq", "sfh", "y_perm", "total")]
 
 
 _lib = None
@@ -115,6 +126,11 @@ def load_library() -> C.CDLL:
     lib.moe_route_tokens.argtypes = [vp, vp, vp, f32p, vp, C.c_size_t, f32p, i32p, f32p, i32p, i32p, i32p, i32p, vp]
     lib.moe_fused_forward_routed.argtypes = [vp, vp, vp, f32p, vp, vp, vp, vp, vp, C.c_size_t, vp, C.c_size_t,
                                              C.POINTER(moe_tuning), vp]
+    lib.moe_quantize_rows_mx.argtypes = [vp, vp, C.c_int64, C.c_int32, vp, vp, vp]
+    lib.moe_dispatch_mx.argtypes = [vp, vp, vp, i32p, vp, vp, vp]
+    lib.moe_expert_ffn_mx.argtypes = [vp, C.POINTER(moe_mx_ffn_args), vp]
+    lib.moe_get_workspace_layout_mx.argtypes = [C.POINTER(moe_shape), C.POINTER(moe_workspace_layout_mx)]
+    lib.moe_fused_forward_mx.argtypes = [vp, vp, f32p, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
     lib.moe_last_device_status.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_last_launch_count.argtypes = [vp]
     lib.moe_last_launch_count.restype = C.c_int32
@@ -340,6 +356,33 @@ class Context:
                                                _ptr(wq_up), _ptr(s_up), _ptr(wq_down), _ptr(s_down), _ptr(out),
                                                _ptr(workspace), workspace.numel() * workspace.element_size(),
                                                _tuning_ref(tuning), _stream(stream)), "moe_fused_forward_fp8")
+
+    def workspace_layout_mx(self) -> dict:
+        L = moe_workspace_layout_mx()
+        _check(self._lib.moe_get_workspace_layout_mx(C.byref(self._shape()), C.byref(L)), "moe_get_workspace_layout_mx")
+        return {n: getattr(L, n) for n, _ in moe_workspace_layout_mx._fields_}
+
+    def moe_quantize_rows_mx(self, in_bf16, rows, cols, codes, sf_words, stream=None):
+        _check(self._lib.moe_quantize_rows_mx(self._handle, _ptr(in_bf16), rows, cols, _ptr(codes), _ptr(sf_words),
+                                              _stream(stream)), "moe_quantize_rows_mx")
+
+    def moe_dispatch_mx(self, xq, sfx, inv_perm, xq_perm, sfx_perm, stream=None):
+        _check(self._lib.moe_dispatch_mx(self._handle, _ptr(xq), _ptr(sfx), _ptr(inv_perm), _ptr(xq_perm),
+                                         _ptr(sfx_perm), _stream(stream)), "moe_dispatch_mx")
+
+    def moe_expert_ffn_mx(self, xq_perm, sfx_perm, offsets, wq_gate, sf_gate, wq_up, sf_up, wq_down, sf_down, hq_ws,
+                          sfh_ws, y_perm, h_fp32_debug=None, stream=None):
+        vals = [xq_perm, sfx_perm, offsets, wq_gate, sf_gate, wq_up, sf_up, wq_down, sf_down, hq_ws, sfh_ws, y_perm,
+                h_fp32_debug]
+        args = moe_mx_ffn_args(*[None if v is None else v.data_ptr() for v in vals])
+        _check(self._lib.moe_expert_ffn_mx(self._handle, C.byref(args), _stream(stream)), "moe_expert_ffn_mx")
+
+    def moe_fused_forward_mx(self, x, logits, wq_gate, sf_gate, wq_up, sf_up, wq_down, sf_down, out, workspace,
+                             stream=None):
+        _check(self._lib.moe_fused_forward_mx(self._handle, _ptr(x), _ptr(logits), _ptr(wq_gate), _ptr(sf_gate),
+                                              _ptr(wq_up), _ptr(sf_up), _ptr(wq_down), _ptr(sf_down), _ptr(out),
+                                              _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                              _stream(stream)), "moe_fused_forward_mx")
 
     def moe_last_device_status(self, stream=None):
         code, detail = C.c_int32(0), C.c_int32(0)

@@ -1,0 +1,426 @@
+// Expert feed-forward with block-scaled FP8 operands (MXFP8): E4M3 elements, one E8M0 scale per 32 elements along K,
+// applied by the tensor pipe inside the MMA (tcgen05.mma.kind::mxf8f6f4.block_scale, scales in tensor memory).
+//
+// One kernel, launched once for Linear-1 (gate | up, SwiGLU, h quantised in the epilogue) and once for Linear-2.
+// Persistent CTAs, one per SM, tiles assigned round-robin (tile t goes to CTA t mod grid).  A tile is 128 rows of one
+// expert x 192 accumulator columns: Linear-1 pairs 96 gate columns with the same 96 up columns, so a tile yields
+// 96 columns of h = three whole 32-element scale blocks, which the epilogue quantises straight from the fp32
+// accumulator (h never exists in bf16); Linear-2 writes 192 bf16 columns of y_perm.
+//
+// Roles (320 threads): warp 0 = TMA producer (codes of A and of two 96-row weight boxes per 128-element K stage),
+// warps 6-9 = scale loaders (one 4-byte cp.async per operand row per stage, written in the 512-byte layout
+// tcgen05.cp expects; they arrive on the stage's full barrier when their copies land), warp 1 = MMA issuer (per
+// stage: three tcgen05.cp of scales into tensor memory, then four MMAs picking scale byte 0..3), warps 2-5 =
+// epilogue.  Tensor memory: two accumulators of 192 columns, 4 columns of A scales, 8 of B scales.
+// Every wait is bounded; a wait that gives up is reported through the status word and the CTA unwinds.
+#include <cuda_bf16.h>
+
+#include "moe_internal.h"
+#include "mx_quant.cuh"
+#include "ptx_sm100.cuh"
+
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int BM = 128;                 // rows per tile
+constexpr int BNH = 96;                 // rows of one weight box
+constexpr int BN = 2 * BNH;             // accumulator columns
+constexpr int BK = 128;                 // K elements (= bytes) per stage: one 128-byte swizzle row
+constexpr int UMMA_K = 32;
+constexpr int kABytes = BM * BK;
+constexpr int kBBoxBytes = BNH * BK;
+constexpr int kOperandBytes = kABytes + 2 * kBBoxBytes;
+constexpr int kSfABytes = 512;          // 128 rows x 4 scale bytes
+constexpr int kSfBytes = kSfABytes + 1024;
+constexpr int kStages = 5;
+constexpr int kTmemCols = 512;
+constexpr uint32_t kTmemSfA = 2 * BN;   // column of the A scales
+constexpr uint32_t kTmemSfB = 2 * BN + 4;
+constexpr int kSfThreads = 128;
+constexpr int kKernelIdMx = 9;          // in the detail word of a time-out: 9 * 65536 + role
+
+struct MxParams {
+  const int32_t* offsets;   // [E+1]
+  int E;
+  int N;                    // output columns of this GEMM: F (Linear-1) or H (Linear-2)
+  int n_blocks;             // tiles along N: ceil(N / 96) gated, ceil(N / 192) otherwise
+  int k_blocks;             // K / 128
+  long long a_rows;         // R
+  long long b_rows;         // E * N: rows of each weight matrix
+  const uint32_t* sf_a;     // [K/128][R]
+  const uint32_t* sf_b0;    // [K/128][E*N] gate resp. down
+  const uint32_t* sf_b1;    // [K/128][E*N] up resp. down
+  uint4* hq;                // Linear-1 out: E4M3 [R, N]
+  unsigned char* sf_h;      // Linear-1 out: scale bytes, words [N/128][R]
+  float* h_dbg;             // optional fp32 [R, N]
+  __nv_bfloat16* y;         // Linear-2 out: bf16 [R, N]
+  int32_t* status;
+};
+
+struct MxTile {
+  int row0, row_end, n0, w_row0;
+};
+
+struct MxTail {
+  uint64_t full[kStages];
+  uint64_t empty[kStages];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  int32_t blk_prefix[1025];   // exclusive prefix of ceil(count / 128) over experts
+};
+
+__device__ __forceinline__ void mx_timeout(const MxParams& p, int role) {
+  atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
+  atomicCAS(&p.status[1], 0, kKernelIdMx * 65536 + role);
+}
+
+// Tile t of the list ordered by (expert, column tile, row block): row blocks of one expert and column tile are
+// neighbours, so CTAs that run side by side share the weight boxes in L2.
+template <bool kGated>
+__device__ __forceinline__ MxTile decode_tile(int t, const MxTail* st, const MxParams& p) {
+  int lo = 0, hi = p.E;   // invariant: prefix(lo) * n_blocks <= t < prefix(hi) * n_blocks
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (st->blk_prefix[mid] * p.n_blocks <= t) lo = mid; else hi = mid;
+  }
+  const int e = lo;
+  const int blocks_e = st->blk_prefix[e + 1] - st->blk_prefix[e];
+  const int local = t - st->blk_prefix[e] * p.n_blocks;
+  const int nb = local / blocks_e, mb = local - nb * blocks_e;
+  MxTile tile;
+  tile.row0 = p.offsets[e] + mb * BM;
+  tile.row_end = p.offsets[e + 1];
+  tile.n0 = nb * (kGated ? BNH : BN);
+  tile.w_row0 = e * p.N + tile.n0;
+  return tile;
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <bool kGated>
+__global__ void __launch_bounds__(kThreads, 1)
+expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
+                     const __grid_constant__ CUtensorMap tm_b1, const MxParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+  unsigned char* base = smem_raw + pad;                      // 1024-byte aligned: required by the swizzle
+  const uint32_t ring_u32 = raw + pad;                       // kStages operand stages
+  const uint32_t sf_u32 = ring_u32 + kStages * kOperandBytes;   // kStages scale stages
+  MxTail* st = reinterpret_cast<MxTail*>(base + kStages * (kOperandBytes + kSfBytes));
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&st->full[s]), 1 + kSfThreads);   // the TMA arrival + every scale loader
+      ptx::mbar_init(ptx::smem_u32(&st->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(ptx::smem_u32(&st->tmem_full[a]), 1);
+      ptx::mbar_init(ptx::smem_u32(&st->tmem_empty[a]), 4);          // one arrival per epilogue warp
+    }
+    st->abort_flag = 0;
+    st->blk_prefix[0] = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async_smem();
+  }
+  if (warp == 0) {
+    int32_t run = 0;
+    for (int b0 = 0; b0 < p.E; b0 += 32) {
+      const int e = b0 + lane;
+      int32_t v = e < p.E ? (p.offsets[e + 1] - p.offsets[e] + BM - 1) / BM : 0;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int32_t o = __shfl_up_sync(0xFFFFFFFFu, v, off);
+        if (lane >= off) v += o;
+      }
+      if (e < p.E) st->blk_prefix[e + 1] = run + v;
+      run += __shfl_sync(0xFFFFFFFFu, v, 31);
+    }
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tm_a);
+      ptx::prefetch_tensormap(&tm_b0);
+      ptx::prefetch_tensormap(&tm_b1);
+    }
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(&st->tmem_base), kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+
+  const uint32_t tmem_base = st->tmem_base;
+  const int total_tiles = st->blk_prefix[p.E] * p.n_blocks;
+  const int b1_shift = kGated ? 0 : BNH;       // second weight box: same rows of the up matrix, or the next 96 rows
+  volatile int* abort_flag = &st->abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+        const MxTile tile = decode_tile<kGated>(t, st, p);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag)) {
+            mx_timeout(p, 1);
+            ok = false;
+            break;
+          }
+          const uint32_t full = ptx::smem_u32(&st->full[stage]);
+          const uint32_t sa = ring_u32 + stage * kOperandBytes;
+          ptx::mbar_expect_tx(full, kOperandBytes);
+          ptx::tma_load_2d(sa, &tm_a, full, kb * BK, tile.row0);
+          ptx::tma_load_2d(sa + kABytes, &tm_b0, full, kb * BK, tile.w_row0);
+          ptx::tma_load_2d(sa + kABytes + kBBoxBytes, &tm_b1, full, kb * BK, tile.w_row0 + b1_shift);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+        if (!ptx::mbar_wait(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) {
+          mx_timeout(p, 2);
+          break;
+        }
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&st->full[stage]), phase, abort_flag)) {
+            mx_timeout(p, 3);
+            ok = false;
+            break;
+          }
+          ptx::fence_proxy_async_smem();     // the scale words arrived through cp.async, tcgen05.cp reads them
+          ptx::tc_fence_after_sync();
+          const uint32_t sa = ring_u32 + stage * kOperandBytes;
+          const uint32_t sf = sf_u32 + stage * kSfBytes;
+          ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfA, sf);
+          ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB, sf + kSfABytes);
+          ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB + 4, sf + kSfABytes + 512);
+          const uint64_t a_desc = ptx::smem_desc_sw128(sa);
+          const uint64_t b_desc = ptx::smem_desc_sw128(sa + kABytes);
+#pragma unroll
+          for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
+            const uint64_t adv = static_cast<uint64_t>(2 * k4);   // +32 bytes along K inside the swizzle row
+            ptx::tc_mma_mx(d_tmem, a_desc + adv, b_desc + adv, ptx::idesc_mx_e4m3(BM, BN, k4, k4),
+                           tmem_base + kTmemSfA, tmem_base + kTmemSfB, (kb | k4) != 0 ? 1u : 0u);
+          }
+          ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // stage (codes and scales) is free once these are done
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::tc_commit(ptx::smem_u32(&st->tmem_full[acc]));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+    __syncwarp();
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ epilogue (4 warps = 128 rows)
+    const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      const MxTile tile = decode_tile<kGated>(t, st, p);
+      if (!ptx::mbar_wait(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag)) {
+        if (lane == 0) mx_timeout(p, 4);
+        break;
+      }
+      ptx::tc_fence_after_sync();
+      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
+      const int row = tile.row0 + quarter * 32 + lane;
+      const bool row_ok = row < tile.row_end;
+      if constexpr (kGated) {
+#pragma unroll 1
+        for (int j = 0; j < BNH / 32; ++j) {
+          const int col = tile.n0 + 32 * j;
+          if (col >= p.N) break;                  // N is a multiple of 32: blocks are whole
+          uint32_t g[32], u[32];
+          ptx::tmem_ld_32x32(t_addr + 32 * j, g);
+          ptx::tmem_ld_32x32(t_addr + BNH + 32 * j, u);
+          ptx::tmem_ld_wait();
+          float h[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) h[i] = silu_mul(__uint_as_float(g[i]), __uint_as_float(u[i]));
+          uint32_t c[8];
+          const uint32_t byte = mx::quantize_block(h, c);
+          if (row_ok) {
+            uint4* dst = p.hq + (static_cast<size_t>(row) * p.N + col) / 16;
+            dst[0] = make_uint4(c[0], c[1], c[2], c[3]);
+            dst[1] = make_uint4(c[4], c[5], c[6], c[7]);
+            p.sf_h[mx::scale_byte_index(p.a_rows, row, col >> 5)] = static_cast<unsigned char>(byte);
+            if (p.h_dbg != nullptr) {
+              float4* dbg = reinterpret_cast<float4*>(p.h_dbg + static_cast<size_t>(row) * p.N + col);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) dbg[i] = make_float4(h[4 * i], h[4 * i + 1], h[4 * i + 2], h[4 * i + 3]);
+            }
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          const int col = tile.n0 + c0;
+          if (col >= p.N) break;
+          uint32_t v[32];
+          ptx::tmem_ld_32x32(t_addr + c0, v);
+          ptx::tmem_ld_wait();
+          if (row_ok) {
+            uint4* dst = reinterpret_cast<uint4*>(p.y + static_cast<size_t>(row) * p.N + col);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              dst[i] = make_uint4(pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
+                                  pack_bf16(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
+                                  pack_bf16(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
+                                  pack_bf16(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
+          }
+        }
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  } else {
+    // ------------------------------------------------------------------ scale loaders (4 warps, one operand row each)
+    const int idx = tid - 6 * 32;                 // 0..127
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    // where this thread's words go inside a stage: row r of a 128-row group sits at (r % 32) * 16 + (r / 32) * 4
+    const uint32_t dst_a = (idx & 31) * 16 + (idx >> 5) * 4;
+    const int n1 = idx + kSfThreads;              // second weight row of this thread (only below 192)
+    const uint32_t dst_b1 = 512 + (n1 & 31) * 16 + ((n1 & 127) >> 5) * 4;
+    for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+      const MxTile tile = decode_tile<kGated>(t, st, p);
+      const long long a_row = static_cast<long long>(tile.row0) + idx;
+      // weight row n of the tile: rows 0..95 come from the first box, 96..191 from the second
+      const long long b_row_0 = idx < BNH ? static_cast<long long>(tile.w_row0) + idx
+                                          : static_cast<long long>(tile.w_row0) + b1_shift + (idx - BNH);
+      const uint32_t* b_src_0 = idx < BNH ? p.sf_b0 : p.sf_b1;
+      const long long b_row_1 = static_cast<long long>(tile.w_row0) + b1_shift + (n1 - BNH);
+      const bool a_ok = a_row < p.a_rows, b0_ok = b_row_0 < p.b_rows, b1_ok = n1 < BN && b_row_1 < p.b_rows;
+      for (int kb = 0; kb < p.k_blocks; ++kb) {
+        if (!ptx::mbar_wait(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag)) {
+          if (lane == 0) mx_timeout(p, 5);
+          ok = false;
+          break;
+        }
+        const uint32_t sf = sf_u32 + stage * kSfBytes;
+        ptx::cp_async_4(sf + dst_a, p.sf_a + (a_ok ? kb * p.a_rows + a_row : 0), a_ok ? 4u : 0u);
+        ptx::cp_async_4(sf + kSfABytes + dst_a, b_src_0 + (b0_ok ? kb * p.b_rows + b_row_0 : 0), b0_ok ? 4u : 0u);
+        if (n1 < BN) ptx::cp_async_4(sf + kSfABytes + dst_b1, p.sf_b1 + (b1_ok ? kb * p.b_rows + b_row_1 : 0), b1_ok ? 4u : 0u);
+        ptx::cp_async_arrive_noinc(ptx::smem_u32(&st->full[stage]));
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  }
+
+  __syncthreads();
+  if (st->abort_flag) {
+    // a wait gave up: give copies still in flight time to land before the shared memory is released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Tensor map over a row-major [rows, cols] matrix of E4M3 bytes: boxes of box_rows x 128 bytes, 128-byte swizzle.
+CUresult encode_bytes(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), box_rows};
+  const cuuint32_t elem[2] = {1u, 1u};
+  return ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * (kOperandBytes + kSfBytes) + sizeof(MxTail);
+
+}  // namespace
+
+namespace moe {
+
+cudaError_t prepare_expert_ffn_mx(moe_ctx* ctx) {
+  (void)ctx;
+  cudaError_t e = cudaFuncSetAttribute(expert_ffn_mx_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(kSmemBytes));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(expert_ffn_mx_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(kSmemBytes));
+}
+
+moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, cudaStream_t stream) {
+  const moe_shape& s = ctx->shape;
+  const uint64_t R = static_cast<uint64_t>(s.T) * s.k;
+  CUtensorMap tm_x, tm_wg, tm_wu, tm_h, tm_wd;
+  if (encode_bytes(ctx, &tm_x, a->xq_perm, R, s.H, BM) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_bytes(ctx, &tm_wg, a->wq_gate, static_cast<uint64_t>(s.E) * s.F, s.H, BNH) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_bytes(ctx, &tm_wu, a->wq_up, static_cast<uint64_t>(s.E) * s.F, s.H, BNH) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_bytes(ctx, &tm_h, a->hq_ws, R, s.F, BM) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  if (encode_bytes(ctx, &tm_wd, a->wq_down, static_cast<uint64_t>(s.E) * s.H, s.F, BNH) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+
+  MxParams p1{};
+  p1.offsets = a->offsets;
+  p1.E = s.E;
+  p1.N = s.F;
+  p1.n_blocks = (s.F + BNH - 1) / BNH;
+  p1.k_blocks = s.H / BK;
+  p1.a_rows = static_cast<long long>(R);
+  p1.b_rows = static_cast<long long>(s.E) * s.F;
+  p1.sf_a = a->sfx_perm;
+  p1.sf_b0 = a->sf_gate;
+  p1.sf_b1 = a->sf_up;
+  p1.hq = static_cast<uint4*>(a->hq_ws);
+  p1.sf_h = reinterpret_cast<unsigned char*>(a->sfh_ws);
+  p1.h_dbg = a->h_fp32_debug;
+  p1.status = ctx->d_status;
+
+  MxParams p2{};
+  p2.offsets = p1.offsets;
+  p2.E = s.E;
+  p2.N = s.H;
+  p2.n_blocks = (s.H + BN - 1) / BN;
+  p2.k_blocks = s.F / BK;
+  p2.a_rows = static_cast<long long>(R);
+  p2.b_rows = static_cast<long long>(s.E) * s.H;
+  p2.sf_a = a->sfh_ws;
+  p2.sf_b0 = a->sf_down;
+  p2.sf_b1 = p2.sf_b0;
+  p2.y = static_cast<__nv_bfloat16*>(a->y_perm);
+  p2.status = ctx->d_status;
+
+  const int grid = ctx->num_sms;
+  expert_ffn_mx_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, p1);
+  moe_mark(ctx, 5, stream);
+  expert_ffn_mx_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(tm_h, tm_wd, tm_wd, p2);
+  moe_mark(ctx, 6, stream);
+  ctx->last_launches += 2;
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+}  // namespace moe

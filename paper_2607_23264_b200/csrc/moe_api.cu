@@ -166,6 +166,7 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   ok = ok && cudaMemset(ctx->d_router_done, 0, done_bytes) == cudaSuccess;
   ok = ok && moe::prepare_expert_ffn(ctx) == cudaSuccess;
   ok = ok && moe::prepare_router(ctx) == cudaSuccess;
+  ok = ok && moe::prepare_expert_ffn_mx(ctx) == cudaSuccess;
   for (int i = 0; ok && i <= kMoeKernels; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) == cudaSuccess;
@@ -567,6 +568,145 @@ moe_status moe_fused_forward_fp8(moe_ctx* ctx, const void* x, const float* logit
   a.sh_ws = reinterpret_cast<float*>(ws + L.sh);
   a.y_perm = ws + L.y_perm;
   st = moe::launch_expert_ffn_fp8(ctx, &a, tuning, cs);
+  if (st != MOE_OK) return st;
+  if (moe::launch_combine(ctx, ws + L.y_perm, inv_perm, topk_w, out, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ MXFP8 variant
+}  // extern "C"
+namespace {
+void fill_layout_mx(const moe_shape& s, moe_workspace_layout_mx* L) {
+  const size_t T = s.T, H = s.H, F = s.F, E = s.E, k = s.k, R = T * k;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t at = off; off += up256(bytes); return at; };
+  L->topk_ids = take(R * 4);
+  L->topk_w = take(R * 4);
+  L->counts = take(E * 4);
+  L->offsets = take((E + 1) * 4);
+  L->perm = take(R * 4);
+  L->inv_perm = take(R * 4);
+  L->xq = take(T * H);
+  L->sfx = take(H / 128 * T * 4);
+  L->xq_perm = take(R * H);
+  L->sfx_perm = take(H / 128 * R * 4);
+  L->hq = take(R * F);
+  L->sfh = take(F / 128 * R * 4);
+  L->y_perm = take(R * H * 2);
+  L->total = off;
+}
+moe_status check_mx_shape(const moe_ctx* ctx) {
+  return (ctx->shape.H % 128 == 0 && ctx->shape.F % 128 == 0) ? MOE_OK : MOE_ERR_UNSUPPORTED_SHAPE;
+}
+}  // namespace
+extern "C" {
+
+moe_status moe_quantize_rows_mx(moe_ctx* ctx, const void* in_bf16, int64_t rows, int32_t cols, void* codes,
+                                uint32_t* sf_words, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  ctx->last_launches = 0;
+  if (rows < 0 || cols <= 0 || cols % 128 != 0) return MOE_ERR_INVALID_ARG;
+  if (rows == 0) return MOE_OK;
+  if (!in_bf16 || !codes || !sf_words || !aligned16(in_bf16) || !aligned16(codes) || !aligned16(sf_words))
+    return MOE_ERR_INVALID_ARG;
+  return moe::launch_quantize_rows_mx(ctx, in_bf16, rows, cols, codes, sf_words, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_dispatch_mx(moe_ctx* ctx, const void* xq, const uint32_t* sfx, const int32_t* inv_perm, void* xq_perm,
+                           uint32_t* sfx_perm, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  st = check_mx_shape(ctx);
+  if (st != MOE_OK) return st;
+  begin_call(ctx, 3, stream);
+  if (ctx->shape.T == 0) return MOE_OK;
+  const void* ptrs[] = {xq, sfx, inv_perm, xq_perm, sfx_perm};
+  for (const void* q : ptrs)
+    if (!q || !aligned16(q)) return MOE_ERR_INVALID_ARG;
+  return moe::launch_dispatch_mx(ctx, xq, sfx, inv_perm, xq_perm, sfx_perm, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+moe_status moe_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  st = check_mx_shape(ctx);
+  if (st != MOE_OK) return st;
+  begin_call(ctx, 4, stream);
+  if (!a) return MOE_ERR_INVALID_ARG;
+  if (ctx->shape.T == 0) return MOE_OK;
+  const void* ptrs[] = {a->xq_perm, a->sfx_perm, a->offsets, a->wq_gate, a->sf_gate, a->wq_up, a->sf_up,
+                        a->wq_down, a->sf_down, a->hq_ws, a->sfh_ws, a->y_perm};
+  for (const void* q : ptrs)
+    if (!q || !aligned16(q)) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(a->h_fp32_debug)) return MOE_ERR_INVALID_ARG;
+  return moe::launch_expert_ffn_mx(ctx, a, static_cast<cudaStream_t>(stream));
+}
+
+moe_status moe_get_workspace_layout_mx(const moe_shape* shape, moe_workspace_layout_mx* out_layout) {
+  if (!out_layout) return MOE_ERR_INVALID_ARG;
+  std::memset(out_layout, 0, sizeof(*out_layout));
+  const moe_status st = check_shape(shape);
+  if (st != MOE_OK) return st;
+  if (shape->H % 128 != 0 || shape->F % 128 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
+  fill_layout_mx(*shape, out_layout);
+  return MOE_OK;
+}
+
+moe_status moe_fused_forward_mx(moe_ctx* ctx, const void* x, const float* logits, const void* wq_gate,
+                                const uint32_t* sf_gate, const void* wq_up, const uint32_t* sf_up, const void* wq_down,
+                                const uint32_t* sf_down, void* out, void* workspace, size_t workspace_bytes,
+                                void* stream) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  st = check_mx_shape(ctx);
+  if (st != MOE_OK) return st;
+  const moe_shape& s = ctx->shape;
+  if (s.T == 0) { ctx->last_launches = 0; return MOE_OK; }
+  const void* ptrs[] = {x, logits, wq_gate, sf_gate, wq_up, sf_up, wq_down, sf_down, out};
+  for (const void* q : ptrs)
+    if (!q || !aligned16(q)) return MOE_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MOE_ERR_INVALID_ARG;
+  moe_workspace_layout_mx L;
+  fill_layout_mx(s, &L);
+  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE_TOO_SMALL;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  int32_t* topk_ids = reinterpret_cast<int32_t*>(ws + L.topk_ids);
+  float* topk_w = reinterpret_cast<float*>(ws + L.topk_w);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+  int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
+  int32_t* perm = reinterpret_cast<int32_t*>(ws + L.perm);
+  int32_t* inv_perm = reinterpret_cast<int32_t*>(ws + L.inv_perm);
+  uint32_t* sfx = reinterpret_cast<uint32_t*>(ws + L.sfx);
+  uint32_t* sfx_perm = reinterpret_cast<uint32_t*>(ws + L.sfx_perm);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  begin_call(ctx, 0, stream);
+  if (moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (moe::launch_quantize_rows_mx(ctx, x, s.T, s.H, ws + L.xq, sfx, cs) != cudaSuccess) return MOE_ERR_CUDA;
+  if (moe::launch_dispatch_mx(ctx, ws + L.xq, sfx, inv_perm, ws + L.xq_perm, sfx_perm, cs) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  moe_mx_ffn_args a{};
+  a.xq_perm = ws + L.xq_perm;
+  a.sfx_perm = sfx_perm;
+  a.offsets = offsets;
+  a.wq_gate = wq_gate;
+  a.sf_gate = sf_gate;
+  a.wq_up = wq_up;
+  a.sf_up = sf_up;
+  a.wq_down = wq_down;
+  a.sf_down = sf_down;
+  a.hq_ws = ws + L.hq;
+  a.sfh_ws = reinterpret_cast<uint32_t*>(ws + L.sfh);
+  a.y_perm = ws + L.y_perm;
+  a.h_fp32_debug = nullptr;
+  st = moe::launch_expert_ffn_mx(ctx, &a, cs);
   if (st != MOE_OK) return st;
   if (moe::launch_combine(ctx, ws + L.y_perm, inv_perm, topk_w, out, cs) != cudaSuccess) return MOE_ERR_CUDA;
   return MOE_OK;

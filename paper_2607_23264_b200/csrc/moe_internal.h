@@ -99,6 +99,14 @@ moe_status launch_router(moe_ctx* ctx, const void* x, const void* w_split, const
                          float* logits_out, int32_t* topk_ids, float* topk_w, cudaStream_t stream);
 cudaError_t prepare_router(moe_ctx* ctx);      // one-time kernel attributes
 
+// Block-scaled FP8 (MXFP8): row quantisation in 32-element blocks, dispatch of quantised rows, the two GEMMs.
+cudaError_t launch_quantize_rows_mx(moe_ctx* ctx, const void* in_bf16, long long rows, int cols, void* codes,
+                                    uint32_t* sf_words, cudaStream_t stream);
+cudaError_t launch_dispatch_mx(moe_ctx* ctx, const void* xq, const uint32_t* sfx, const int32_t* inv_perm,
+                               void* xq_perm, uint32_t* sfx_perm, cudaStream_t stream);
+moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* args, cudaStream_t stream);
+cudaError_t prepare_expert_ffn_mx(moe_ctx* ctx);
+
 cudaError_t prepare_expert_ffn(moe_ctx* ctx);  // one-time kernel attributes (dynamic shared memory size)
 
 }  // namespace moe

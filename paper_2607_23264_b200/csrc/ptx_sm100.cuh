@@ -250,4 +250,46 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N) {
          (static_cast<uint32_t>(M >> 4) << 24);
 }
 
+// ---------------------------------------------------------------- block-scaled MMA (kind::mxf8f6f4)
+// D[tmem] (+)= (A * 2^sfa) * (B * 2^sfb)^T: E4M3 operands from shared memory, K = 32 per instruction, one E8M0
+// scale per operand row per instruction, read from tensor memory: for an operand of R rows the scales sit in R/32
+// consecutive 32-bit columns; row r is lane r % 32 (replicated in all four lane quarters) of column r / 32, and
+// the four bytes of that word are the scales of four consecutive K = 32 steps, selected by the sf id fields of the
+// instruction descriptor.
+__device__ __forceinline__ void tc_mma_mx(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %6, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%4], [%5], p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+// Instruction descriptor of the block-scaled form: E4M3 x E4M3 (format code 0), both K-major, E8M0 scales, tile
+// M x N, scale byte a_sf / b_sf (0..3) of the scale words.  The accumulator is always fp32.
+__host__ __device__ constexpr uint32_t idesc_mx_e4m3(int M, int N, int a_sf, int b_sf) {
+  return (static_cast<uint32_t>(b_sf) << 4) | (static_cast<uint32_t>(N >> 3) << 17) | (1u << 23) |
+         (static_cast<uint32_t>(M >> 4) << 24) | (static_cast<uint32_t>(a_sf) << 29);
+}
+// Shared memory -> tensor memory: 32 rows of 16 bytes (512 contiguous bytes, no swizzle) become four 32-bit
+// columns of lanes 0..31, replicated into all four lane quarters.  Issued by one thread; ordered with the MMAs
+// the same thread issues before and after it.
+__device__ __forceinline__ void tc_cp_32x128b_warpx4(uint32_t taddr, uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+  d |= static_cast<uint64_t>(128 >> 4) << 32;                // 8-row groups are 128 bytes apart
+  d |= static_cast<uint64_t>(1) << 46;                       // descriptor version for sm_100
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
+}
+// 4-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros and reads nothing.
+__device__ __forceinline__ void cp_async_4(uint32_t dst_smem, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
+}
+// One arrival on `bar` (already counted in its expected arrivals) once this thread's earlier cp.async copies landed.
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 }  // namespace ptx

@@ -1,0 +1,183 @@
+"""Block-scaled FP8 (MXFP8) experts on the GPU against the oracle.
+
+Codes and scale bytes are integer decisions taken in fp32 on both sides: compared bit for bit (x, the weights, the
+dispatched rows, and h re-quantised by the oracle from the GPU's own fp32 h).  The GEMMs are compared on identical
+quantised operands (fp32 accumulation and bf16 output rounding only), and the whole layer in norm against the fully
+independent oracle, where a last-bit difference in h can move an E4M3 code by one step."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as orc
+from oracle import mx_oracle as mx
+from paper_2607_23264_b200 import binding, inputs as gen
+from moe_testlib import DEV, TOL_FRO, TOL_OUT, Layer, assert_out_close, bits_to_dev, dev_bf16_to_f64, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+def words_to_bytes(words: torch.Tensor, rows: int) -> np.ndarray:
+    """scale words [K/128][rows] (device) -> scale bytes [rows, K/32] as the oracle orders them."""
+    w = words.cpu().numpy().view(np.uint8).reshape(-1, rows, 4)
+    return np.ascontiguousarray(w.transpose(1, 0, 2)).reshape(rows, -1)
+
+
+def bytes_to_words(b: np.ndarray) -> torch.Tensor:
+    rows, nb = b.shape
+    w = np.ascontiguousarray(b.reshape(rows, nb // 4, 4).transpose(1, 0, 2)).reshape(nb // 4, rows * 4)
+    return torch.from_numpy(w.view(np.uint32).reshape(nb // 4, rows).copy().view(np.int32)).to(DEV)
+
+
+def quantize_on_gpu(ctx, t_bf16: torch.Tensor):
+    rows, cols = t_bf16.shape
+    codes = torch.full((rows, cols), 0x7F, dtype=torch.uint8, device=DEV)
+    words = torch.full((cols // 128, rows), -1, dtype=torch.int32, device=DEV)
+    ctx.moe_quantize_rows_mx(t_bf16, rows, cols, codes, words)
+    torch.cuda.synchronize()
+    return codes, words
+
+
+class MxLayer:
+    def __init__(self, cfg):
+        self.cfg = cfg
+        self.L = Layer(cfg)
+        L, E, F, H = self.L, cfg.E, cfg.F, cfg.H
+        self.q = {}
+        for name, t, rows, cols in (("gate", L.w_gate, E * F, H), ("up", L.w_up, E * F, H), ("down", L.w_down, E * H, F)):
+            self.q[name] = quantize_on_gpu(L.ctx, t.view(rows, cols))
+
+        self._wq = {}
+
+    def oracle_weights(self, e):
+        if e not in self._wq:
+            self._wq[e] = mx.quantize_weights(*self.L.weights(e))
+        return self._wq[e]
+
+
+def small_cfg(T, H, F, E, k, seed, router="xWr"):
+    return gen.MoEConfig(name="mx", T=T, H=H, F=F, E=E, k=k, seed=seed, router=router)
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 128), (37, 256), (300, 1024)])
+def test_quantize_rows_mx_bits(rows, cols):
+    rng = np.random.default_rng(rows)
+    v = (rng.standard_normal((rows, cols)) * np.exp(rng.uniform(-8, 8, (rows, 1)))).astype(np.float32)
+    v[0, :32] = 0.0                                               # an all-zero block
+    if rows > 2:
+        v[2, 32:64] = np.float32(448.0) * np.float32(2.0) ** rng.integers(-5, 5, 32)   # exact boundary values
+    bits = gen.f32_to_bf16_bits(v)
+    ctx = binding.Context(8, 128, 128, 2, 1)
+    codes, words = quantize_on_gpu(ctx, bits_to_dev(bits))
+    ref_c, ref_s = mx.quantize_rows(gen.bf16_bits_to_f32(bits))
+    assert np.array_equal(codes.cpu().numpy(), ref_c)
+    assert np.array_equal(words_to_bytes(words, rows), ref_s)
+
+
+@pytest.mark.parametrize("T,H,F,E,k,router", [
+    (64, 128, 128, 4, 2, "xWr"),        # one K stage per GEMM; Linear-1 tiles of 96 + 32 columns; Linear-2 tile wider than H
+    (300, 512, 384, 8, 2, "xWr"),       # several row blocks per expert, ragged tails, whole column tiles
+    (129, 256, 640, 16, 4, "xWr_zipf"), # skewed: empty experts, experts of one row
+    (5, 384, 256, 6, 6, "xWr"),         # k = E, five rows per expert
+])
+def test_expert_ffn_mx_parity(T, H, F, E, k, router):
+    cfg = small_cfg(T, H, F, E, k, seed=T + H, router=router)
+    M = MxLayer(cfg)
+    L, ctx = M.L, M.L.ctx
+    L.plan()
+    ref = mx.forward_mx(L.x_bits, L.logits, k, L.weights)
+    R = cfg.R
+    # x: quantise and dispatch on the GPU, bit for bit
+    xq, sfx = quantize_on_gpu(ctx, L.x)
+    assert np.array_equal(xq.cpu().numpy(), ref["xq"]) and np.array_equal(words_to_bytes(sfx, T), ref["sx"])
+    xq_perm = torch.full((R, H), 0x7F, dtype=torch.uint8, device=DEV)
+    sfx_perm = torch.full((H // 128, R), -1, dtype=torch.int32, device=DEV)
+    ctx.moe_dispatch_mx(xq, sfx, L.inv_perm, xq_perm, sfx_perm)
+    torch.cuda.synchronize()
+    assert np.array_equal(xq_perm.cpu().numpy(), ref["xq_perm"])
+    assert np.array_equal(words_to_bytes(sfx_perm, R), ref["sx_perm"])
+    # weights: the GPU's codes are the oracle's
+    for e in (0, E - 1):
+        (gq, gs), (uq, us), (dq, ds) = M.oracle_weights(e)
+        assert np.array_equal(M.q["gate"][0][e * F:(e + 1) * F].cpu().numpy(), gq)
+        assert np.array_equal(words_to_bytes(M.q["down"][1], E * H)[e * H:(e + 1) * H], ds)
+    # the two GEMMs
+    hq = torch.full((R, F), 0x7F, dtype=torch.uint8, device=DEV)
+    sfh = torch.full((F // 128, R), -1, dtype=torch.int32, device=DEV)
+    y = L.nan_bf16(R, H)
+    h_dbg = torch.full((R, F), float("nan"), device=DEV)
+    ctx.moe_expert_ffn_mx(xq_perm, sfx_perm, L.offsets, *M.q["gate"], *M.q["up"], *M.q["down"], hq, sfh, y, h_dbg)
+    torch.cuda.synchronize()
+    L.check_device_status()
+    h_gpu = h_dbg.cpu().numpy()
+    assert np.isfinite(h_gpu).all()
+    assert rel_fro(h_gpu.astype(np.float64), ref["h"]) <= TOL_FRO
+    # h's codes and scales are the oracle's quantisation of the GPU's own fp32 h
+    req_c, req_s = mx.quantize_rows(h_gpu)
+    assert np.array_equal(hq.cpu().numpy(), req_c)
+    assert np.array_equal(words_to_bytes(sfh, R), req_s)
+    # Linear-2 on the GPU's own codes
+    y_gpu = dev_bf16_to_f64(y)
+    assert np.isfinite(y_gpu).all()
+    offsets = L.offsets.cpu().numpy()
+    y_ref = np.zeros((R, H))
+    for e in range(E):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        if hi > lo:
+            dq, ds = M.oracle_weights(e)[2]
+            y_ref[lo:hi] = mx.gemm(req_c[lo:hi], req_s[lo:hi], dq, ds)
+    assert rel_fro(y_gpu, y_ref) <= TOL_FRO
+    assert_out_close(y_gpu, y_ref, "Linear-2 on the GPU's codes")
+    # and against the fully independent oracle, in norm
+    assert rel_fro(y_gpu, ref["y_perm"]) <= 2e-2
+
+
+def test_fused_forward_mx_and_sampled_rows_at_full_k():
+    # C2's hidden size with two experts: K loops of 32 and 11 stages (the 5-stage ring wraps many times), 15 column
+    # tiles of Linear-1 with a ragged last one (1408 = 14 * 96 + 64), 22 of Linear-2 (4096 = 21 * 192 + 64)
+    cfg = small_cfg(1024, 4096, 1408, 2, 2, seed=9)
+    M = MxLayer(cfg)
+    L, ctx = M.L, M.L.ctx
+    lay = ctx.workspace_layout_mx()
+    ws = torch.empty(lay["total"], dtype=torch.uint8, device=DEV)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    ctx.moe_fused_forward_mx(L.x, L.d_logits, *M.q["gate"], *M.q["up"], *M.q["down"], out, ws)
+    torch.cuda.synchronize()
+    L.check_device_status()
+    assert ctx.moe_last_launch_count() == 8
+    out_gpu = dev_bf16_to_f64(out)
+    assert np.isfinite(out_gpu).all()
+    # oracle on a sample of tokens (rows are independent)
+    ids, w = orc.topk_route(L.logits, cfg.k)
+    counts, offsets, perm, inv_perm = orc.plan_permutation(ids, cfg.E)
+    rng = np.random.default_rng(0)
+    toks = np.sort(rng.choice(cfg.T, 48, replace=False))
+    xq, sx = mx.quantize_rows(orc.bf16_to_f64(L.x_bits[toks]))
+    wq = {e: M.oracle_weights(e) for e in range(cfg.E)}
+    ref = np.zeros((len(toks), cfg.H))
+    for i, t in enumerate(toks):
+        for j in range(cfg.k):
+            r = mx.expert_ffn_rows(xq[i:i + 1], sx[i:i + 1], wq[int(ids[t, j])])
+            ref[i] += w[t, j] * r["y"][0]
+    assert rel_fro(out_gpu[toks], ref) <= 2e-2
+    # the plan in the workspace is the bf16 path's plan
+    got_perm = ws[lay["perm"]:lay["perm"] + 4 * cfg.R].view(torch.int32).cpu().numpy()
+    assert np.array_equal(got_perm, perm)
+    # determinism
+    out2 = L.nan_bf16(cfg.T, cfg.H)
+    ctx.moe_fused_forward_mx(L.x, L.d_logits, *M.q["gate"], *M.q["up"], *M.q["down"], out2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+
+
+def test_mx_rejects_shapes_it_cannot_tile():
+    ctx = binding.Context(16, 192, 128, 2, 1)       # H is not a multiple of 128
+    t = torch.zeros(64, dtype=torch.uint8, device=DEV)
+    with pytest.raises(binding.MoeError) as e:
+        ctx.moe_dispatch_mx(t, t, t, t, t)
+    assert e.value.code == 2
+    with pytest.raises(binding.MoeError) as e:
+        ctx.workspace_layout_mx()
+    assert e.value.code == 2
+    with pytest.raises(binding.MoeError) as e:
+        ctx.moe_quantize_rows_mx(t, 1, 96, t, t)
+    assert e.value.code == 1
