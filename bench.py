@@ -208,10 +208,17 @@ def main():
     dev = f"cuda:{local_rank}"
     if args.probe_mma:
         pctx = binding.Context(128, 64, 64, 1, 1, device=local_rank)
-        rows = [{"M": M, "N": N, "clocks_per_mma": pctx.moe_probe_mma_cycles(M, N)}
+        # the first launches run while the clocks ramp: warm up, then keep the smallest of several runs per point
+        for _ in range(20):
+            pctx.moe_probe_mma_cycles(128, 256, 16384)
+        best = lambda fn: min(fn() for _ in range(7))
+        rows = [{"M": M, "N": N, "clocks_per_mma": best(lambda: pctx.moe_probe_mma_cycles(M, N))}
                 for M in (128, 64) for N in (16, 32, 64, 128, 256)]
+        kinds = ((1, "kind::f8f6f4 (E4M3), 128xNx32"), (2, "kind::mxf8f6f4.block_scale (E4M3, E8M0 scales), 128xNx32"))
+        rows8 = [{"kind": name, "N": N, "clocks_per_mma": best(lambda: pctx.moe_probe_mma_cycles_kind(kind, 128, N))}
+                 for kind, name in kinds for N in (32, 64, 96, 128, 192, 256)]
         print(json.dumps({"probe": "tcgen05.mma kind::f16 MxNx16, one CTA, operands resident in shared memory",
-                          "rows": rows}), flush=True)
+                          "rows": rows, "fp8_rows": rows8}), flush=True)
         return
     if args.xstage_probe:
         run_xstage_probe(dev)
@@ -547,7 +554,12 @@ def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
     ws = torch.empty(ctx.workspace_layout_fp8()["total"], dtype=torch.uint8, device=dev)
     tn = binding.make_tuning(args.burst, args.mode, args.ik, debug_flags={"auto": 0, "on": 8, "off": 16}[args.pairs])
     step = lambda: ctx.moe_fused_forward_fp8(x, d_logits, *wq, out, ws, tuning=tn)
+    sampler = ClockSampler(torch.cuda.current_device())
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
     ms = timed(step, args.steps, args.warmup) / args.steps
+    clocks = sampler.stop() if rank == 0 else None
     ctx.moe_set_kernel_timing(True)
     per = []
     for _ in range(args.steps):
@@ -575,7 +587,7 @@ def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         "roofline": {"kernel": "expert FFN Linear-1 launch, E4M3 operands", "bound": "tensor", "achieved": l1_tf,
                      "peak": peak, "unit": "TFLOP/s", "frac": l1_tf / peak, "traffic": None,
                      "peak_source": f"2 x {kind} bf16_tflops (burst): nominal fp8 / bf16 ratio"},
-        "gpu_launches": ctx.moe_last_launch_count() * args.steps,
+        "gpu_launches": ctx.moe_last_launch_count() * args.steps, "clocks": clocks,
     }
     print(json.dumps(line), flush=True)
 
@@ -595,7 +607,12 @@ def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
     del w_gate, w_up, w_down
     ws = torch.empty(ctx.workspace_layout_mx()["total"], dtype=torch.uint8, device=dev)
     step = lambda: ctx.moe_fused_forward_mx(x, d_logits, *wq, out, ws)
+    sampler = ClockSampler(torch.cuda.current_device())
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
     ms = timed(step, args.steps, args.warmup) / args.steps
+    clocks = sampler.stop() if rank == 0 else None
     ctx.moe_set_kernel_timing(True)
     per = []
     for _ in range(args.steps):
@@ -624,7 +641,7 @@ def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         "roofline": {"kernel": "expert FFN Linear-1 launch, block-scaled E4M3 operands", "bound": "tensor",
                      "achieved": l1_tf, "peak": peak, "unit": "TFLOP/s", "frac": l1_tf / peak, "traffic": None,
                      "peak_source": f"2 x {kind} bf16_tflops (burst): nominal fp8 / bf16 ratio"},
-        "gpu_launches": ctx.moe_last_launch_count() * args.steps,
+        "gpu_launches": ctx.moe_last_launch_count() * args.steps, "clocks": clocks,
     }
     print(json.dumps(line), flush=True)
 

@@ -28,7 +28,7 @@ EXPORTS = (
     "moe_dispatch_fp8", "moe_expert_ffn_fp8", "moe_get_workspace_layout_fp8", "moe_fused_forward_fp8",
     "moe_set_active_tokens", "moe_plan_routing_from_topk", "moe_router_weight_bytes", "moe_router_scratch_bytes",
     "moe_router_prepare", "moe_route_tokens", "moe_fused_forward_routed", "moe_quantize_rows_mx", "moe_dispatch_mx",
-    "moe_expert_ffn_mx", "moe_get_workspace_layout_mx", "moe_fused_forward_mx",
+    "moe_expert_ffn_mx", "moe_get_workspace_layout_mx", "moe_fused_forward_mx", "moe_probe_mma_cycles_kind",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -137,6 +137,7 @@ def load_library() -> C.CDLL:
     lib.moe_set_kernel_timing.argtypes = [vp, C.c_int32]
     lib.moe_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32]
     lib.moe_probe_mma_cycles.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_double), vp]
+    lib.moe_probe_mma_cycles_kind.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_double), vp]
     lib.moe_get_ffn_order.argtypes = [vp, C.POINTER(C.c_int32), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.moe_get_ffn_trace.argtypes = [vp, C.POINTER(C.c_uint64), C.c_int32, C.POINTER(C.c_int32), vp]
     for name in EXPORTS:
@@ -426,6 +427,13 @@ class Context:
         out = C.c_double(0.0)
         _check(self._lib.moe_probe_mma_cycles(self._handle, M, N, iters, C.byref(out), _stream(stream)),
                "moe_probe_mma_cycles")
+        return out.value
+
+    def moe_probe_mma_cycles_kind(self, kind: int, M: int, N: int, iters: int = 4096, stream=None) -> float:
+        """kind 0 bf16, 1 E4M3, 2 block-scaled E4M3."""
+        out = C.c_double(0.0)
+        _check(self._lib.moe_probe_mma_cycles_kind(self._handle, kind, M, N, iters, C.byref(out), _stream(stream)),
+               "moe_probe_mma_cycles_kind")
         return out.value
 
     def moe_set_kernel_timing(self, enable: bool):

@@ -936,6 +936,7 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
 
 // Calibration probe: one CTA issues `iters` tcgen05.mma of shape M x N x 16 back to back on resident
 // shared-memory operands and reports the SM clocks from the first issue to the completion of the last.
+template <int kKind>
 __global__ void __launch_bounds__(128, 1) mma_cycle_probe(int M, int N, int iters, long long* out) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ uint64_t bar;
@@ -961,12 +962,30 @@ __global__ void __launch_bounds__(128, 1) mma_cycle_probe(int M, int N, int iter
   ptx::tc_fence_after_sync();
   const uint32_t tb = tmem_base_s;
   if (threadIdx.x == 0) {
-    const uint32_t idesc = ptx::idesc_bf16_f32(M, N);
     const uint64_t a = ptx::smem_desc_sw128(base), b = ptx::smem_desc_sw128(base + kABytes);
+    // block-scaled kind: scale columns behind the accumulator, filled once from the (constant) operand bytes
+    const uint32_t sfa = tb + 256, sfb = tb + 260;
+    if constexpr (kKind == 2) {
+      ptx::tc_cp_32x128b_warpx4(sfa, base);
+      ptx::tc_cp_32x128b_warpx4(sfb, base + 512);
+      ptx::tc_cp_32x128b_warpx4(sfb + 4, base + 1024);
+    }
+    // descriptors out of the loop: the loop must cost less than the instruction it times
+    uint32_t idesc[4];
+#pragma unroll
+    for (int k4 = 0; k4 < 4; ++k4)
+      idesc[k4] = kKind == 0 ? ptx::idesc_bf16_f32(M, N) : kKind == 1 ? ptx::idesc_e4m3_f32(M, N)
+                                                                      : ptx::idesc_mx_e4m3(M, N, k4, k4);
     const long long t0 = clock64();
-    for (int i = 0; i < iters; ++i) {
-      const uint64_t adv = static_cast<uint64_t>(2 * (i & 3));
-      ptx::tc_mma_bf16(tb, a + adv, b + adv, idesc, i > 0 ? 1u : 0u);
+    for (int i = 0; i < iters; i += 4) {
+#pragma unroll
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const uint64_t adv = static_cast<uint64_t>(2 * k4);
+        const uint32_t acc = (i | k4) != 0 ? 1u : 0u;
+        if constexpr (kKind == 0) ptx::tc_mma_bf16(tb, a + adv, b + adv, idesc[k4], acc);
+        else if constexpr (kKind == 1) ptx::tc_mma_e4m3(tb, a + adv, b + adv, idesc[k4], acc);
+        else ptx::tc_mma_mx(tb, a + adv, b + adv, idesc[k4], sfa, sfb, acc);
+      }
     }
     ptx::tc_commit(ptx::smem_u32(&bar));
     ptx::mbar_wait(ptx::smem_u32(&bar), 0, &abort_flag);
@@ -996,16 +1015,23 @@ CUresult encode_2d(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t ro
 
 extern "C" moe_status moe_probe_mma_cycles(moe_ctx* ctx, int32_t M, int32_t N, int32_t iters, double* cycles_per_mma,
                                            void* stream) {
+  return moe_probe_mma_cycles_kind(ctx, 0, M, N, iters, cycles_per_mma, stream);
+}
+
+extern "C" moe_status moe_probe_mma_cycles_kind(moe_ctx* ctx, int32_t kind, int32_t M, int32_t N, int32_t iters,
+                                                double* cycles_per_mma, void* stream) {
   if (!ctx || !cycles_per_mma) return MOE_ERR_INVALID_ARG;
+  if (kind < 0 || kind > 2 || (kind == 2 && M != 128)) return MOE_ERR_INVALID_ARG;
   if (!(M == 64 || M == 128) || N < 16 || N > 256 || N % 16 != 0 || iters < 1 || iters > (1 << 20))
     return MOE_ERR_INVALID_ARG;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   long long* d_out = reinterpret_cast<long long*>(ctx->d_trace);   // reuse the first trace word as the result slot
   const size_t smem = 1024 + kStageBytes;
-  if (cudaFuncSetAttribute(mma_cycle_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
-      cudaSuccess)
+  auto kernel = kind == 0 ? mma_cycle_probe<0> : kind == 1 ? mma_cycle_probe<1> : mma_cycle_probe<2>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
     return MOE_ERR_CUDA;
-  mma_cycle_probe<<<1, 128, smem, cs>>>(M, N, iters, d_out);
+  iters = (iters + 3) / 4 * 4;
+  kernel<<<1, 128, smem, cs>>>(M, N, iters, d_out);
   long long clocks = 0;
   if (cudaMemcpyAsync(&clocks, d_out, sizeof(clocks), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return MOE_ERR_CUDA;
   if (cudaStreamSynchronize(cs) != cudaSuccess) return MOE_ERR_CUDA;
