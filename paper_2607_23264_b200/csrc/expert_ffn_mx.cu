@@ -9,7 +9,8 @@
 //
 // Roles (320 threads): warp 0 = TMA producer (codes of A and of two 96-row weight boxes per 128-element K stage),
 // warps 6-9 = scale loaders (one 4-byte cp.async per operand row per stage, written in the 512-byte layout
-// tcgen05.cp expects; they arrive on the stage's full barrier when their copies land), warp 1 = MMA issuer (per
+// tcgen05.cp expects, into a ring of their own that is twice as deep as the operand ring; they arrive on its full
+// barrier when their copies land), warp 1 = MMA issuer (per
 // stage: three tcgen05.cp of scales into tensor memory, then four MMAs picking scale byte 0..3), warps 2-5 =
 // epilogue.  Tensor memory: two accumulators of 192 columns, 4 columns of A scales, 8 of B scales.
 // Every wait is bounded; a wait that gives up is reported through the status word and the CTA unwinds.
@@ -33,6 +34,7 @@ constexpr int kOperandBytes = kABytes + 2 * kBBoxBytes;
 constexpr int kSfABytes = 512;          // 128 rows x 4 scale bytes
 constexpr int kSfBytes = kSfABytes + 1024;
 constexpr int kStages = 5;
+constexpr int kSfStages = 10;           // the scale ring is deeper than the operand ring: scale loads run further ahead
 constexpr int kTmemCols = 512;
 constexpr uint32_t kTmemSfA = 2 * BN;   // column of the A scales
 constexpr uint32_t kTmemSfB = 2 * BN + 4;
@@ -64,6 +66,8 @@ struct MxTile {
 struct MxTail {
   uint64_t full[kStages];
   uint64_t empty[kStages];
+  uint64_t sf_full[kSfStages];
+  uint64_t sf_empty[kSfStages];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint32_t tmem_base;
@@ -113,15 +117,19 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   unsigned char* base = smem_raw + pad;                      // 1024-byte aligned: required by the swizzle
   const uint32_t ring_u32 = raw + pad;                       // kStages operand stages
-  const uint32_t sf_u32 = ring_u32 + kStages * kOperandBytes;   // kStages scale stages
-  MxTail* st = reinterpret_cast<MxTail*>(base + kStages * (kOperandBytes + kSfBytes));
+  const uint32_t sf_u32 = ring_u32 + kStages * kOperandBytes;   // kSfStages scale stages
+  MxTail* st = reinterpret_cast<MxTail*>(base + kStages * kOperandBytes + kSfStages * kSfBytes);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&st->full[s]), 1 + kSfThreads);   // the TMA arrival + every scale loader
+      ptx::mbar_init(ptx::smem_u32(&st->full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&st->empty[s]), 1);
+    }
+    for (int s = 0; s < kSfStages; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&st->sf_full[s]), kSfThreads);    // every scale loader, when its copies have landed
+      ptx::mbar_init(ptx::smem_u32(&st->sf_empty[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(ptx::smem_u32(&st->tmem_full[a]), 1);
@@ -194,6 +202,8 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
+      int sf_stage = 0;
+      uint32_t sf_phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
@@ -210,10 +220,15 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             ok = false;
             break;
           }
+          if (!ptx::mbar_wait(ptx::smem_u32(&st->sf_full[sf_stage]), sf_phase, abort_flag)) {
+            mx_timeout(p, 6);
+            ok = false;
+            break;
+          }
           ptx::fence_proxy_async_smem();     // the scale words arrived through cp.async, tcgen05.cp reads them
           ptx::tc_fence_after_sync();
           const uint32_t sa = ring_u32 + stage * kOperandBytes;
-          const uint32_t sf = sf_u32 + stage * kSfBytes;
+          const uint32_t sf = sf_u32 + sf_stage * kSfBytes;
           ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfA, sf);
           ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB, sf + kSfABytes);
           ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB + 4, sf + kSfABytes + 512);
@@ -225,8 +240,10 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             ptx::tc_mma_mx(d_tmem, a_desc + adv, b_desc + adv, ptx::idesc_mx_e4m3(BM, BN, k4, k4),
                            tmem_base + kTmemSfA, tmem_base + kTmemSfB, (kb | k4) != 0 ? 1u : 0u);
           }
-          ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // stage (codes and scales) is free once these are done
+          ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // codes and scales are free once these are done
+          ptx::tc_commit(ptx::smem_u32(&st->sf_empty[sf_stage]));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++sf_stage == kSfStages) { sf_stage = 0; sf_phase ^= 1u; }
         }
         if (!ok) break;
         ptx::tc_commit(ptx::smem_u32(&st->tmem_full[acc]));
@@ -321,7 +338,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       const long long b_row_1 = static_cast<long long>(tile.w_row0) + b1_shift + (n1 - BNH);
       const bool a_ok = a_row < p.a_rows, b0_ok = b_row_0 < p.b_rows, b1_ok = n1 < BN && b_row_1 < p.b_rows;
       for (int kb = 0; kb < p.k_blocks; ++kb) {
-        if (!ptx::mbar_wait(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag)) {
+        if (!ptx::mbar_wait(ptx::smem_u32(&st->sf_empty[stage]), phase ^ 1u, abort_flag)) {
           if (lane == 0) mx_timeout(p, 5);
           ok = false;
           break;
@@ -330,8 +347,8 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         ptx::cp_async_4(sf + dst_a, p.sf_a + (a_ok ? kb * p.a_rows + a_row : 0), a_ok ? 4u : 0u);
         ptx::cp_async_4(sf + kSfABytes + dst_a, b_src_0 + (b0_ok ? kb * p.b_rows + b_row_0 : 0), b0_ok ? 4u : 0u);
         if (n1 < BN) ptx::cp_async_4(sf + kSfABytes + dst_b1, p.sf_b1 + (b1_ok ? kb * p.b_rows + b_row_1 : 0), b1_ok ? 4u : 0u);
-        ptx::cp_async_arrive_noinc(ptx::smem_u32(&st->full[stage]));
-        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        ptx::cp_async_arrive_noinc(ptx::smem_u32(&st->sf_full[stage]));
+        if (++stage == kSfStages) { stage = 0; phase ^= 1u; }
       }
     }
   }
@@ -359,7 +376,7 @@ CUresult encode_bytes(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * (kOperandBytes + kSfBytes) + sizeof(MxTail);
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kOperandBytes + kSfStages * kSfBytes + sizeof(MxTail);
 
 }  // namespace
 
