@@ -181,3 +181,26 @@ def test_mx_rejects_shapes_it_cannot_tile():
     with pytest.raises(binding.MoeError) as e:
         ctx.moe_quantize_rows_mx(t, 1, 96, t, t)
     assert e.value.code == 1
+
+
+def test_mx_smaller_batches_on_one_context():
+    # a context created for T tokens runs any smaller batch (and an empty one) through the block-scaled path
+    cfg = small_cfg(96, 256, 256, 4, 2, seed=21)
+    M = MxLayer(cfg)
+    L, ctx = M.L, M.L.ctx
+    ws = torch.empty(ctx.workspace_layout_mx()["total"], dtype=torch.uint8, device=DEV)
+    for tokens in (96, 33, 1, 0):
+        ctx.moe_set_active_tokens(tokens)
+        out = L.nan_bf16(max(tokens, 1), cfg.H)
+        ctx.moe_fused_forward_mx(L.x[:tokens].contiguous() if tokens else L.x, L.d_logits[:tokens].contiguous() if tokens
+                                 else L.d_logits, *M.q["gate"], *M.q["up"], *M.q["down"], out, ws)
+        torch.cuda.synchronize()
+        L.check_device_status()
+        if tokens == 0:
+            assert ctx.moe_last_launch_count() == 0
+            continue
+        ref = mx.forward_mx(L.x_bits[:tokens], L.logits[:tokens], cfg.k, L.weights)
+        got = dev_bf16_to_f64(out)[:tokens]
+        assert np.isfinite(got).all()
+        assert rel_fro(got, ref["out"]) <= 2.5e-2
+    ctx.moe_set_active_tokens(cfg.T)

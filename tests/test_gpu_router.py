@@ -192,3 +192,29 @@ def test_router_argument_errors():
     torch.cuda.synchronize()
     assert int(c.counts.abs().sum()) == 0 and int(c.offsets.abs().sum()) == 0
     assert c.ctx.moe_last_launch_count() == 0
+
+
+def test_router_smaller_batches_on_one_context():
+    c = RouterCase(300, 256, 24, 3, seed=17, bias=True)
+    c.route()
+    full_ids = c.topk_ids.clone()
+    full_logits = c.logits.clone()
+    for tokens in (129, 128, 7):
+        c.ctx.moe_set_active_tokens(tokens)
+        c.topk_ids.fill_(-1)
+        c.logits.fill_(float("nan"))
+        c.ctx.moe_route_tokens(c.x, c.w_split, c.d_bias, c.scratch, c.logits, c.topk_ids, c.topk_w, c.counts, c.offsets,
+                               c.perm, c.inv_perm)
+        torch.cuda.synchronize()
+        code, _ = c.ctx.moe_last_device_status()
+        assert code == 0
+        # rows are independent and the K split is the same for every batch size here (H = 256 has four K blocks,
+        # which caps the split at 4), so the first `tokens` tokens get the same logit bits as in the full batch
+        ids = c.topk_ids.view(-1)[: tokens * 3].view(tokens, 3)
+        assert torch.equal(ids, full_ids[:tokens])
+        lg = c.logits.view(-1)[: tokens * 24].view(tokens, 24)
+        assert torch.equal(lg.view(torch.int32), full_logits[:tokens].view(torch.int32))
+        counts, offsets, perm, inv_perm = moe_oracle.plan_permutation(ids.cpu().numpy(), 24)
+        assert np.array_equal(c.counts.cpu().numpy(), counts)
+        assert np.array_equal(c.perm.cpu().numpy()[: tokens * 3], perm)
+    c.ctx.moe_set_active_tokens(300)
