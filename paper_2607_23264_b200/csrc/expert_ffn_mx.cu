@@ -8,9 +8,9 @@
 // accumulator (h never exists in bf16); Linear-2 writes 192 bf16 columns of y_perm.
 //
 // Roles (320 threads): warp 0 = TMA producer (codes of A and of two 96-row weight boxes per 128-element K stage),
-// warps 6-9 = scale loaders (one 4-byte cp.async per operand row per stage, written in the 512-byte layout
-// tcgen05.cp expects, into a ring of their own that is twice as deep as the operand ring; they arrive on its full
-// barrier when their copies land), warp 1 = MMA issuer (per
+// warps 6-9 = scale loaders (one word per operand row per stage, loaded four stages ahead into registers and
+// stored in the 512-byte layout tcgen05.cp expects, into a ring of their own that is twice as deep as the operand
+// ring), warp 1 = MMA issuer (per
 // stage: three tcgen05.cp of scales into tensor memory, then four MMAs picking scale byte 0..3), warps 2-5 =
 // epilogue.  Tensor memory: two accumulators of 192 columns, 4 columns of A scales, 8 of B scales.
 // Every wait is bounded; a wait that gives up is reported through the status word and the CTA unwinds.
@@ -128,7 +128,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       ptx::mbar_init(ptx::smem_u32(&st->empty[s]), 1);
     }
     for (int s = 0; s < kSfStages; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&st->sf_full[s]), kSfThreads);    // every scale loader, when its copies have landed
+      ptx::mbar_init(ptx::smem_u32(&st->sf_full[s]), kSfThreads);    // every scale loader, after its stores
       ptx::mbar_init(ptx::smem_u32(&st->sf_empty[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -225,7 +225,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             ok = false;
             break;
           }
-          ptx::fence_proxy_async_smem();     // the scale words arrived through cp.async, tcgen05.cp reads them
+          ptx::fence_proxy_async_smem();     // the scale words were stored through the generic proxy, tcgen05.cp reads them
           ptx::tc_fence_after_sync();
           const uint32_t sa = ring_u32 + stage * kOperandBytes;
           const uint32_t sf = sf_u32 + sf_stage * kSfBytes;
@@ -320,35 +320,72 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     }
   } else {
     // ------------------------------------------------------------------ scale loaders (4 warps, one operand row each)
-    const int idx = tid - 6 * 32;                 // 0..127
-    int stage = 0;
-    uint32_t phase = 0;
-    bool ok = true;
-    // where this thread's words go inside a stage: row r of a 128-row group sits at (r % 32) * 16 + (r / 32) * 4
+    const int w4 = warp - 6;                      // 0..3
+    // Row of a 128-row group this thread serves.  Row r sits at (r % 32) * 16 + (r / 32) * 4 inside the group's
+    // 512 bytes; with r = 32 * (lane % 4) + 8 * w4 + lane / 4 the 32 lanes of a warp store 32 consecutive words (one
+    // shared-memory wavefront) and read four runs of eight consecutive rows from global memory.  Plain loads into
+    // registers, kPrefetch stages ahead, then plain stores: a 4-byte cp.async costs 16 shared-memory wavefronts
+    // per warp whatever the addresses, a quarter of the shared-memory pipe at this kernel's rate.
+    const int idx = 32 * (lane & 3) + 8 * w4 + (lane >> 2);
     const uint32_t dst_a = (idx & 31) * 16 + (idx >> 5) * 4;
     const int n1 = idx + kSfThreads;              // second weight row of this thread (only below 192)
     const uint32_t dst_b1 = 512 + (n1 & 31) * 16 + ((n1 & 127) >> 5) * 4;
-    for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
-      const MxTile tile = decode_tile<kGated>(t, st, p);
+    constexpr int kPrefetch = 4;
+
+    // prefetch cursor: the (tile, K block) whose scale words are loaded next
+    int pf_t = blockIdx.x, pf_kb = 0;
+    const uint32_t *pf_a = nullptr, *pf_b0 = nullptr, *pf_b1 = nullptr;   // null = outside the operand: scale byte 0
+    auto pf_setup = [&]() {
+      if (pf_t >= total_tiles) return;
+      const MxTile tile = decode_tile<kGated>(pf_t, st, p);
       const long long a_row = static_cast<long long>(tile.row0) + idx;
       // weight row n of the tile: rows 0..95 come from the first box, 96..191 from the second
       const long long b_row_0 = idx < BNH ? static_cast<long long>(tile.w_row0) + idx
                                           : static_cast<long long>(tile.w_row0) + b1_shift + (idx - BNH);
-      const uint32_t* b_src_0 = idx < BNH ? p.sf_b0 : p.sf_b1;
       const long long b_row_1 = static_cast<long long>(tile.w_row0) + b1_shift + (n1 - BNH);
-      const bool a_ok = a_row < p.a_rows, b0_ok = b_row_0 < p.b_rows, b1_ok = n1 < BN && b_row_1 < p.b_rows;
-      for (int kb = 0; kb < p.k_blocks; ++kb) {
+      pf_a = a_row < p.a_rows ? p.sf_a + a_row : nullptr;
+      pf_b0 = b_row_0 < p.b_rows ? (idx < BNH ? p.sf_b0 : p.sf_b1) + b_row_0 : nullptr;
+      pf_b1 = (n1 < BN && b_row_1 < p.b_rows) ? p.sf_b1 + b_row_1 : nullptr;
+    };
+    auto pf_load = [&](uint32_t (&w)[3]) {
+      w[0] = pf_a ? __ldg(pf_a + pf_kb * p.a_rows) : 0u;
+      w[1] = pf_b0 ? __ldg(pf_b0 + pf_kb * p.b_rows) : 0u;
+      w[2] = pf_b1 ? __ldg(pf_b1 + pf_kb * p.b_rows) : 0u;
+      if (++pf_kb == p.k_blocks) {
+        pf_kb = 0;
+        pf_t += gridDim.x;
+        pf_setup();
+      }
+    };
+    pf_setup();
+    uint32_t buf[kPrefetch][3];
+#pragma unroll
+    for (int u = 0; u < kPrefetch; ++u) {
+      buf[u][0] = buf[u][1] = buf[u][2] = 0u;
+      if (pf_t < total_tiles) pf_load(buf[u]);
+    }
+    long long remaining = 0;                      // stages this CTA runs in all
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) remaining += p.k_blocks;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    while (ok && remaining > 0) {
+#pragma unroll
+      for (int u = 0; u < kPrefetch; ++u) {
+        if (remaining <= 0) break;
         if (!ptx::mbar_wait(ptx::smem_u32(&st->sf_empty[stage]), phase ^ 1u, abort_flag)) {
           if (lane == 0) mx_timeout(p, 5);
           ok = false;
           break;
         }
-        const uint32_t sf = sf_u32 + stage * kSfBytes;
-        ptx::cp_async_4(sf + dst_a, p.sf_a + (a_ok ? kb * p.a_rows + a_row : 0), a_ok ? 4u : 0u);
-        ptx::cp_async_4(sf + kSfABytes + dst_a, b_src_0 + (b0_ok ? kb * p.b_rows + b_row_0 : 0), b0_ok ? 4u : 0u);
-        if (n1 < BN) ptx::cp_async_4(sf + kSfABytes + dst_b1, p.sf_b1 + (b1_ok ? kb * p.b_rows + b_row_1 : 0), b1_ok ? 4u : 0u);
-        ptx::cp_async_arrive_noinc(ptx::smem_u32(&st->sf_full[stage]));
+        unsigned char* sf = base + kStages * kOperandBytes + stage * kSfBytes;
+        *reinterpret_cast<uint32_t*>(sf + dst_a) = buf[u][0];
+        *reinterpret_cast<uint32_t*>(sf + kSfABytes + dst_a) = buf[u][1];
+        if (n1 < BN) *reinterpret_cast<uint32_t*>(sf + kSfABytes + dst_b1) = buf[u][2];
+        ptx::mbar_arrive(ptx::smem_u32(&st->sf_full[stage]));       // release: the stores above are visible to the waiter
         if (++stage == kSfStages) { stage = 0; phase ^= 1u; }
+        --remaining;
+        if (pf_t < total_tiles) pf_load(buf[u]);
       }
     }
   }
