@@ -214,7 +214,8 @@ def main():
         best = lambda fn: min(fn() for _ in range(7))
         rows = [{"M": M, "N": N, "clocks_per_mma": best(lambda: pctx.moe_probe_mma_cycles(M, N))}
                 for M in (128, 64) for N in (16, 32, 64, 128, 256)]
-        kinds = ((1, "kind::f8f6f4 (E4M3), 128xNx32"), (2, "kind::mxf8f6f4.block_scale (E4M3, E8M0 scales), 128xNx32"))
+        kinds = ((1, "kind::f8f6f4 (E4M3), 128xNx32"), (2, "kind::mxf8f6f4.block_scale (E4M3, E8M0 scales), 128xNx32"),
+                 (3, "kind::mxf8f6f4.block_scale with 3 tcgen05.cp scale copies per 4 instructions, 128xNx32"))
         rows8 = [{"kind": name, "N": N, "clocks_per_mma": best(lambda: pctx.moe_probe_mma_cycles_kind(kind, 128, N))}
                  for kind, name in kinds for N in (32, 64, 96, 128, 192, 256)]
         print(json.dumps({"probe": "tcgen05.mma kind::f16 MxNx16, one CTA, operands resident in shared memory",
@@ -620,6 +621,16 @@ def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         per.append(ctx.moe_get_kernel_times())
     ctx.moe_set_kernel_timing(False)
     km = [float(np.mean([p[i] for p in per])) for i in range(len(binding.KERNEL_NAMES))]
+    # the GEMMs' own wait counters (recorded while per-kernel timing is on), averaged over CTAs, as shares of the span
+    tr = ctx.moe_get_ffn_trace().astype(np.float64)
+    waits = {}
+    for gi, gname in enumerate(("linear1", "linear2")):
+        span = np.maximum(tr[gi, :, 0], 1.0)
+        waits[gname] = {"span_clocks": float(span.mean()), "tiles_per_cta": float(tr[gi, :, 6].mean()),
+                        "mma_waits_operands": float((tr[gi, :, 2] / span).mean()),
+                        "mma_waits_accumulator": float((tr[gi, :, 3] / span).mean()),
+                        "producer_waits_stage": float((tr[gi, :, 1] / span).mean()),
+                        "epilogue_busy": float((tr[gi, :, 5] / span).mean())}
     code, detail = ctx.moe_last_device_status()
     if code != 0:
         raise RuntimeError(f"device status {code} detail {detail:#x}")
@@ -641,7 +652,7 @@ def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         "roofline": {"kernel": "expert FFN Linear-1 launch, block-scaled E4M3 operands", "bound": "tensor",
                      "achieved": l1_tf, "peak": peak, "unit": "TFLOP/s", "frac": l1_tf / peak, "traffic": None,
                      "peak_source": f"2 x {kind} bf16_tflops (burst): nominal fp8 / bf16 ratio"},
-        "gpu_launches": ctx.moe_last_launch_count() * args.steps, "clocks": clocks,
+        "gpu_launches": ctx.moe_last_launch_count() * args.steps, "clocks": clocks, "gemm_waits": waits,
     }
     print(json.dumps(line), flush=True)
 

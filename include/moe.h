@@ -455,7 +455,9 @@ moe_status moe_get_ffn_order(moe_ctx* ctx, int32_t* codes_host, int32_t capacity
 moe_status moe_probe_mma_cycles(moe_ctx* ctx, int32_t M, int32_t N, int32_t iters, double* cycles_per_mma,
                                 void* stream);
 /* The same probe for the other operand kinds: kind 0 = bf16 (K = 16 per instruction), 1 = E4M3 (kind::f8f6f4,
- * K = 32), 2 = block-scaled E4M3 (kind::mxf8f6f4.block_scale, K = 32, M = 128 only; scales resident in tensor memory). */
+ * K = 32), 2 = block-scaled E4M3 (kind::mxf8f6f4.block_scale, K = 32, M = 128 only; scales resident in tensor memory),
+ * 3 = the same with three tcgen05.cp scale copies (512 bytes each) in front of every four instructions, as one K stage
+ * of the block-scaled GEMM issues them. */
 moe_status moe_probe_mma_cycles_kind(moe_ctx* ctx, int32_t kind, int32_t M, int32_t N, int32_t iters,
                                      double* cycles_per_mma, void* stream);
 

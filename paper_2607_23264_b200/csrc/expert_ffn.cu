@@ -965,7 +965,7 @@ __global__ void __launch_bounds__(128, 1) mma_cycle_probe(int M, int N, int iter
     const uint64_t a = ptx::smem_desc_sw128(base), b = ptx::smem_desc_sw128(base + kABytes);
     // block-scaled kind: scale columns behind the accumulator, filled once from the (constant) operand bytes
     const uint32_t sfa = tb + 256, sfb = tb + 260;
-    if constexpr (kKind == 2) {
+    if constexpr (kKind >= 2) {
       ptx::tc_cp_32x128b_warpx4(sfa, base);
       ptx::tc_cp_32x128b_warpx4(sfb, base + 512);
       ptx::tc_cp_32x128b_warpx4(sfb + 4, base + 1024);
@@ -978,6 +978,11 @@ __global__ void __launch_bounds__(128, 1) mma_cycle_probe(int M, int N, int iter
                                                                       : ptx::idesc_mx_e4m3(M, N, k4, k4);
     const long long t0 = clock64();
     for (int i = 0; i < iters; i += 4) {
+      if constexpr (kKind == 3) {        // as a K stage of the block-scaled GEMM: three scale copies, then four MMAs
+        ptx::tc_cp_32x128b_warpx4(sfa, base);
+        ptx::tc_cp_32x128b_warpx4(sfb, base + 512);
+        ptx::tc_cp_32x128b_warpx4(sfb + 4, base + 1024);
+      }
 #pragma unroll
       for (int k4 = 0; k4 < 4; ++k4) {
         const uint64_t adv = static_cast<uint64_t>(2 * k4);
@@ -1021,13 +1026,13 @@ extern "C" moe_status moe_probe_mma_cycles(moe_ctx* ctx, int32_t M, int32_t N, i
 extern "C" moe_status moe_probe_mma_cycles_kind(moe_ctx* ctx, int32_t kind, int32_t M, int32_t N, int32_t iters,
                                                 double* cycles_per_mma, void* stream) {
   if (!ctx || !cycles_per_mma) return MOE_ERR_INVALID_ARG;
-  if (kind < 0 || kind > 2 || (kind == 2 && M != 128)) return MOE_ERR_INVALID_ARG;
+  if (kind < 0 || kind > 3 || (kind >= 2 && M != 128)) return MOE_ERR_INVALID_ARG;
   if (!(M == 64 || M == 128) || N < 16 || N > 256 || N % 16 != 0 || iters < 1 || iters > (1 << 20))
     return MOE_ERR_INVALID_ARG;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   long long* d_out = reinterpret_cast<long long*>(ctx->d_trace);   // reuse the first trace word as the result slot
   const size_t smem = 1024 + kStageBytes;
-  auto kernel = kind == 0 ? mma_cycle_probe<0> : kind == 1 ? mma_cycle_probe<1> : mma_cycle_probe<2>;
+  auto kernel = kind == 0 ? mma_cycle_probe<0> : kind == 1 ? mma_cycle_probe<1> : kind == 2 ? mma_cycle_probe<2> : mma_cycle_probe<3>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
     return MOE_ERR_CUDA;
   iters = (iters + 3) / 4 * 4;

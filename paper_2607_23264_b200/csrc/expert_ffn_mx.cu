@@ -9,8 +9,7 @@
 //
 // Roles (320 threads): warp 0 = TMA producer (codes of A and of two 96-row weight boxes per 128-element K stage),
 // warps 6-9 = scale loaders (one word per operand row per stage, loaded four stages ahead into registers and
-// stored in the 512-byte layout tcgen05.cp expects, into a ring of their own that is twice as deep as the operand
-// ring), warp 1 = MMA issuer (per
+// stored in the 512-byte layout tcgen05.cp expects, then a proxy fence and an arrival on the stage's full barrier), warp 1 = MMA issuer (per
 // stage: three tcgen05.cp of scales into tensor memory, then four MMAs picking scale byte 0..3), warps 2-5 =
 // epilogue.  Tensor memory: two accumulators of 192 columns, 4 columns of A scales, 8 of B scales.
 // Every wait is bounded; a wait that gives up is reported through the status word and the CTA unwinds.
@@ -34,7 +33,6 @@ constexpr int kOperandBytes = kABytes + 2 * kBBoxBytes;
 constexpr int kSfABytes = 512;          // 128 rows x 4 scale bytes
 constexpr int kSfBytes = kSfABytes + 1024;
 constexpr int kStages = 5;
-constexpr int kSfStages = 10;           // the scale ring is deeper than the operand ring: scale loads run further ahead
 constexpr int kTmemCols = 512;
 constexpr uint32_t kTmemSfA = 2 * BN;   // column of the A scales
 constexpr uint32_t kTmemSfB = 2 * BN + 4;
@@ -57,6 +55,7 @@ struct MxParams {
   float* h_dbg;             // optional fp32 [R, N]
   __nv_bfloat16* y;         // Linear-2 out: bf16 [R, N]
   int32_t* status;
+  unsigned long long* trace;   // null, or [CTAs][kMoeTraceFields] wait counters (the fields of the bf16 kernel)
 };
 
 struct MxTile {
@@ -66,8 +65,6 @@ struct MxTile {
 struct MxTail {
   uint64_t full[kStages];
   uint64_t empty[kStages];
-  uint64_t sf_full[kSfStages];
-  uint64_t sf_empty[kSfStages];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint32_t tmem_base;
@@ -117,19 +114,15 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   unsigned char* base = smem_raw + pad;                      // 1024-byte aligned: required by the swizzle
   const uint32_t ring_u32 = raw + pad;                       // kStages operand stages
-  const uint32_t sf_u32 = ring_u32 + kStages * kOperandBytes;   // kSfStages scale stages
-  MxTail* st = reinterpret_cast<MxTail*>(base + kStages * kOperandBytes + kSfStages * kSfBytes);
+  const uint32_t sf_u32 = ring_u32 + kStages * kOperandBytes;   // kStages scale stages
+  MxTail* st = reinterpret_cast<MxTail*>(base + kStages * (kOperandBytes + kSfBytes));
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&st->full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&st->full[s]), 1 + kSfThreads);   // the TMA arrival + every scale loader
       ptx::mbar_init(ptx::smem_u32(&st->empty[s]), 1);
-    }
-    for (int s = 0; s < kSfStages; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&st->sf_full[s]), kSfThreads);    // every scale loader, after its stores
-      ptx::mbar_init(ptx::smem_u32(&st->sf_empty[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(ptx::smem_u32(&st->tmem_full[a]), 1);
@@ -178,10 +171,12 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      long long w_empty = 0;
+      const long long t_begin = clock64();
       for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
         const MxTile tile = decode_tile<kGated>(t, st, p);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag)) {
+          if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, &w_empty)) {
             mx_timeout(p, 1);
             ok = false;
             break;
@@ -195,6 +190,10 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
+      if (p.trace) {
+        p.trace[blockIdx.x * kMoeTraceFields + 0] = static_cast<unsigned long long>(clock64() - t_begin);
+        p.trace[blockIdx.x * kMoeTraceFields + 1] = static_cast<unsigned long long>(w_empty);
+      }
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -202,33 +201,27 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      int sf_stage = 0;
-      uint32_t sf_phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      long long w_full = 0, w_tmem = 0;
+      unsigned long long n_tiles = 0;
       for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
-        if (!ptx::mbar_wait(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) {
+        if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, &w_tmem)) {
           mx_timeout(p, 2);
           break;
         }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&st->full[stage]), phase, abort_flag)) {
+          if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), phase, abort_flag, &w_full)) {
             mx_timeout(p, 3);
             ok = false;
             break;
           }
-          if (!ptx::mbar_wait(ptx::smem_u32(&st->sf_full[sf_stage]), sf_phase, abort_flag)) {
-            mx_timeout(p, 6);
-            ok = false;
-            break;
-          }
-          ptx::fence_proxy_async_smem();     // the scale words were stored through the generic proxy, tcgen05.cp reads them
           ptx::tc_fence_after_sync();
           const uint32_t sa = ring_u32 + stage * kOperandBytes;
-          const uint32_t sf = sf_u32 + sf_stage * kSfBytes;
+          const uint32_t sf = sf_u32 + stage * kSfBytes;
           ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfA, sf);
           ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB, sf + kSfABytes);
           ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB + 4, sf + kSfABytes + 512);
@@ -241,14 +234,18 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                            tmem_base + kTmemSfA, tmem_base + kTmemSfB, (kb | k4) != 0 ? 1u : 0u);
           }
           ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // codes and scales are free once these are done
-          ptx::tc_commit(ptx::smem_u32(&st->sf_empty[sf_stage]));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          if (++sf_stage == kSfStages) { sf_stage = 0; sf_phase ^= 1u; }
         }
         if (!ok) break;
         ptx::tc_commit(ptx::smem_u32(&st->tmem_full[acc]));
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
+        ++n_tiles;
+      }
+      if (p.trace) {
+        p.trace[blockIdx.x * kMoeTraceFields + 2] = static_cast<unsigned long long>(w_full);
+        p.trace[blockIdx.x * kMoeTraceFields + 3] = static_cast<unsigned long long>(w_tmem);
+        p.trace[blockIdx.x * kMoeTraceFields + 6] = n_tiles;
       }
     }
     __syncwarp();
@@ -257,13 +254,15 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     int acc = 0;
     uint32_t acc_phase = 0;
+    long long w_acc = 0, busy = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
       const MxTile tile = decode_tile<kGated>(t, st, p);
-      if (!ptx::mbar_wait(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag)) {
+      if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, &w_acc)) {
         if (lane == 0) mx_timeout(p, 4);
         break;
       }
       ptx::tc_fence_after_sync();
+      const long long t_drain = clock64();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
       const int row = tile.row0 + quarter * 32 + lane;
       const bool row_ok = row < tile.row_end;
@@ -315,8 +314,13 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
+      busy += clock64() - t_drain;
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
+    }
+    if (p.trace && warp == 2 && lane == 0) {
+      p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
+      p.trace[blockIdx.x * kMoeTraceFields + 5] = static_cast<unsigned long long>(busy);
     }
   } else {
     // ------------------------------------------------------------------ scale loaders (4 warps, one operand row each)
@@ -373,7 +377,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
 #pragma unroll
       for (int u = 0; u < kPrefetch; ++u) {
         if (remaining <= 0) break;
-        if (!ptx::mbar_wait(ptx::smem_u32(&st->sf_empty[stage]), phase ^ 1u, abort_flag)) {
+        if (!ptx::mbar_wait(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag)) {
           if (lane == 0) mx_timeout(p, 5);
           ok = false;
           break;
@@ -382,8 +386,9 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         *reinterpret_cast<uint32_t*>(sf + dst_a) = buf[u][0];
         *reinterpret_cast<uint32_t*>(sf + kSfABytes + dst_a) = buf[u][1];
         if (n1 < BN) *reinterpret_cast<uint32_t*>(sf + kSfABytes + dst_b1) = buf[u][2];
-        ptx::mbar_arrive(ptx::smem_u32(&st->sf_full[stage]));       // release: the stores above are visible to the waiter
-        if (++stage == kSfStages) { stage = 0; phase ^= 1u; }
+        ptx::fence_proxy_async_smem();      // the words were stored through the generic proxy, tcgen05.cp reads them
+        ptx::mbar_arrive(ptx::smem_u32(&st->full[stage]));
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
         --remaining;
         if (pf_t < total_tiles) pf_load(buf[u]);
       }
@@ -413,7 +418,7 @@ CUresult encode_bytes(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kOperandBytes + kSfStages * kSfBytes + sizeof(MxTail);
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * (kOperandBytes + kSfBytes) + sizeof(MxTail);
 
 }  // namespace
 
@@ -453,6 +458,7 @@ moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, cudaStre
   p1.sf_h = reinterpret_cast<unsigned char*>(a->sfh_ws);
   p1.h_dbg = a->h_fp32_debug;
   p1.status = ctx->d_status;
+  p1.trace = ctx->timing ? ctx->d_trace : nullptr;   // per-kernel timing also turns the wait counters on
 
   MxParams p2{};
   p2.offsets = p1.offsets;
@@ -467,8 +473,12 @@ moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, cudaStre
   p2.sf_b1 = p2.sf_b0;
   p2.y = static_cast<__nv_bfloat16*>(a->y_perm);
   p2.status = ctx->d_status;
+  p2.trace = ctx->timing ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
 
   const int grid = ctx->num_sms;
+  if (ctx->timing &&
+      cudaMemsetAsync(ctx->d_trace, 0, static_cast<size_t>(2) * ctx->num_sms * kMoeTraceFields * 8, stream) != cudaSuccess)
+    return MOE_ERR_CUDA;
   expert_ffn_mx_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(tm_x, tm_wg, tm_wu, p1);
   moe_mark(ctx, 5, stream);
   expert_ffn_mx_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(tm_h, tm_wd, tm_wd, p2);
