@@ -160,6 +160,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="C2", choices=sorted(gen.CONFIGS))
+    ap.add_argument("--tokens", type=int, default=0, help="run --config's layer at this batch size instead of its own T")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=128, help="tokens per step of the reference (oracle) arm")
     ap.add_argument("--cpu-baseline-tokens", type=int, default=384)
@@ -193,6 +194,10 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     cfg = gen.CONFIGS[args.config]
+    if args.tokens:
+        # the same layer at another batch size (a serving batch): same seed and weights, T tokens
+        import dataclasses
+        cfg = dataclasses.replace(cfg, name=f"{cfg.name}@T={args.tokens}", T=args.tokens)
     if args.warmup < 3 and args.impl == "b200" and not args.sweep:
         args.warmup = 3   # timing rule: at least three warm-up steps
 

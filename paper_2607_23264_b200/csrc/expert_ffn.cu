@@ -35,6 +35,7 @@
 
 #include <climits>
 
+#include "ffn_math.cuh"
 #include "moe_internal.h"
 #include "ptx_sm100.cuh"
 
@@ -175,13 +176,6 @@ __device__ __forceinline__ Tile decode_tile(int code, const SharedTail* st, cons
   const int local = tile - nb * prefix[e];
   const int n_blk = local / mb;
   return make_tile(phase, e, local - n_blk * mb, n_blk, st, p);
-}
-
-__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
-
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 __device__ __forceinline__ void report_timeout(const FfnParams& p, int role) {

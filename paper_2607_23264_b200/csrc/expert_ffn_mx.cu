@@ -15,6 +15,7 @@
 // Every wait is bounded; a wait that gives up is reported through the status word and the CTA unwinds.
 #include <cuda_bf16.h>
 
+#include "ffn_math.cuh"
 #include "moe_internal.h"
 #include "mx_quant.cuh"
 #include "ptx_sm100.cuh"
@@ -96,13 +97,6 @@ __device__ __forceinline__ MxTile decode_tile(int t, const MxTail* st, const MxP
   tile.n0 = nb * (kGated ? BNH : BN);
   tile.w_row0 = e * p.N + tile.n0;
   return tile;
-}
-
-__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
-
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 template <bool kGated>
