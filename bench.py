@@ -573,6 +573,22 @@ def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         per.append(ctx.moe_get_kernel_times())
     ctx.moe_set_kernel_timing(False)
     km = [float(np.mean([p[i] for p in per])) for i in range(len(binding.KERNEL_NAMES))]
+    waits = None
+    if args.trace:
+        # one traced step: the GEMMs' own wait counters, averaged over CTAs, as shares of the producer's span
+        ttn = binding.make_tuning(args.burst, args.mode, args.ik,
+                                  debug_flags={"auto": 0, "on": 8, "off": 16}[args.pairs] | 1)
+        ctx.moe_fused_forward_fp8(x, d_logits, *wq, out, ws, tuning=ttn)
+        tr = ctx.moe_get_ffn_trace().astype(np.float64)
+        waits = {}
+        for gi, gname in enumerate(("linear1", "linear2")):
+            live = tr[gi, :, 0] > 0
+            span = np.maximum(tr[gi, live, 0], 1.0)
+            waits[gname] = {"span_clocks": float(span.mean()), "tiles_per_cta": float(tr[gi, live, 6].mean()),
+                            "mma_waits_operands": float((tr[gi, live, 2] / span).mean()),
+                            "mma_waits_accumulator": float((tr[gi, live, 3] / span).mean()),
+                            "producer_waits_stage": float((tr[gi, live, 1] / span).mean()),
+                            "epilogue_busy": float((tr[gi, live, 5] / span).mean())}
     code, detail = ctx.moe_last_device_status()
     if code != 0:
         raise RuntimeError(f"device status {code} detail {detail:#x}")
@@ -593,7 +609,7 @@ def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         "roofline": {"kernel": "expert FFN Linear-1 launch, E4M3 operands", "bound": "tensor", "achieved": l1_tf,
                      "peak": peak, "unit": "TFLOP/s", "frac": l1_tf / peak, "traffic": None,
                      "peak_source": f"2 x {kind} bf16_tflops (burst): nominal fp8 / bf16 ratio"},
-        "gpu_launches": ctx.moe_last_launch_count() * args.steps, "clocks": clocks,
+        "gpu_launches": ctx.moe_last_launch_count() * args.steps, "clocks": clocks, "gemm_waits": waits,
     }
     print(json.dumps(line), flush=True)
 

@@ -234,12 +234,19 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
       ptx::tmem_ld_wait();
       if constexpr (kFp8) {
         const float rs = row_ok ? d.row_scale[row] : 0.f;
-        const int w0 = t.w_row0 + c * kChunkCols;
+        // the chunk's 32 column scales of each matrix as eight 16-byte loads (the same addresses in every lane);
+        // N is a multiple of 32, so a chunk is inside the matrix or outside as a whole
+        const bool in = t.n0 + c * kChunkCols < d.N;
+        const float4* g4 = reinterpret_cast<const float4*>(d.col_scale0 + t.w_row0 + c * kChunkCols);
+        const float4* u4 = reinterpret_cast<const float4*>(d.col_scale1 + t.w_row0 + c * kChunkCols);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const bool in = t.n0 + c * kChunkCols + i < d.N;
-          const float sg = in ? d.col_scale0[w0 + i] : 0.f, su = in ? d.col_scale1[w0 + i] : 0.f;
-          o[i] = silu_mul(__uint_as_float(v[i]) * (rs * sg), __uint_as_float(u[i]) * (rs * su));
+        for (int q = 0; q < 8; ++q) {
+          const float4 sg = in ? __ldg(g4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 su = in ? __ldg(u4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+          o[4 * q + 0] = silu_mul(__uint_as_float(v[4 * q + 0]) * (rs * sg.x), __uint_as_float(u[4 * q + 0]) * (rs * su.x));
+          o[4 * q + 1] = silu_mul(__uint_as_float(v[4 * q + 1]) * (rs * sg.y), __uint_as_float(u[4 * q + 1]) * (rs * su.y));
+          o[4 * q + 2] = silu_mul(__uint_as_float(v[4 * q + 2]) * (rs * sg.z), __uint_as_float(u[4 * q + 2]) * (rs * su.z));
+          o[4 * q + 3] = silu_mul(__uint_as_float(v[4 * q + 3]) * (rs * sg.w), __uint_as_float(u[4 * q + 3]) * (rs * su.w));
         }
       } else {
 #pragma unroll
@@ -251,11 +258,15 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
       if constexpr (kFp8) {
         const float rs = row_ok ? d.row_scale[row] : 0.f;
         // columns 0..127 of the tile come from the first weight box, 128..255 from the second (same matrix)
-        const int w0 = t.w_row0 + c * kChunkCols;
+        const bool in = t.n0 + c * kChunkCols < d.N;
+        const float4* s4 = reinterpret_cast<const float4*>(d.col_scale0 + t.w_row0 + c * kChunkCols);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const bool in = t.n0 + c * kChunkCols + i < d.N;
-          o[i] = __uint_as_float(v[i]) * (rs * (in ? d.col_scale0[w0 + i] : 0.f));
+        for (int q = 0; q < 8; ++q) {
+          const float4 sc = in ? __ldg(s4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+          o[4 * q + 0] = __uint_as_float(v[4 * q + 0]) * (rs * sc.x);
+          o[4 * q + 1] = __uint_as_float(v[4 * q + 1]) * (rs * sc.y);
+          o[4 * q + 2] = __uint_as_float(v[4 * q + 2]) * (rs * sc.z);
+          o[4 * q + 3] = __uint_as_float(v[4 * q + 3]) * (rs * sc.w);
         }
       } else {
 #pragma unroll
