@@ -55,7 +55,7 @@ constexpr int kTmemCols = 512;
 constexpr int kChunkCols = 32;     // accumulator columns per tcgen05.ld = columns of one store tile
 constexpr int kRing = 4;           // tile codes the producer may publish ahead of the consumers
 constexpr int kHotBlocks = 2;      // experts with at least this many 128-row blocks count as tensor-bound
-constexpr int kSwapRows = 64;      // experts with at most this many rows run with swapped operands
+constexpr int kSwapRows = 64;      // row blocks with at most this many rows (small experts, short last blocks) run with swapped operands
 constexpr int kPhaseShift = 30;    // tile code = phase << 30 | index in the phase's tile list; -1 = no more tiles
 
 struct SharedTail {
@@ -144,8 +144,8 @@ __device__ __forceinline__ Tile make_tile(int phase, int e, int m_blk, int n_blk
   t.n0 = n_blk * d.out_cols_per_tile;
   t.w_row0 = e * d.N + t.n0;
   t.block = st->hot_prefix[e] + st->cold_prefix[e] + m_blk;
-  const int rows = t.row_end - p.offsets[e];                      // the whole expert
-  t.n_pad = rows <= kSwapRows ? ((rows + 15) & ~15) : 0;          // few rows: swapped operands (m_blk is 0 then)
+  const int rows = min(t.row_end - t.row0, BM);                   // rows of this block: a whole small expert, or the
+  t.n_pad = rows <= kSwapRows ? ((rows + 15) & ~15) : 0;          // short last block of a larger one: swapped operands
   return t;
 }
 
