@@ -283,13 +283,4 @@ __device__ __forceinline__ void tc_cp_32x128b_warpx4(uint32_t taddr, uint32_t sm
   d |= static_cast<uint64_t>(1) << 46;                       // descriptor version for sm_100
   asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
 }
-// 4-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros and reads nothing.
-__device__ __forceinline__ void cp_async_4(uint32_t dst_smem, const void* src, uint32_t src_bytes) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
-}
-// One arrival on `bar` (already counted in its expected arrivals) once this thread's earlier cp.async copies landed.
-__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
-  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
-}
-
 }  // namespace ptx
