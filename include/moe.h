@@ -368,7 +368,7 @@ typedef struct {
 } moe_mx_ffn_args;
 
 /* Linear-1 (block-scaled MMA, SiLU*mul, h quantised in the epilogue) and Linear-2 (-> y_perm bf16): two launches,
- * 128 x 192 tiles, Expert-Wave order.  For expert e and its rows r, with deq() the dequantised operands:
+ * 128 x 256 tiles, Expert-Wave order.  For expert e and its rows r, with deq() the dequantised operands:
  *   h[r,f] = silu(sum_c deq(x)[r,c] deq(w_gate)[e,f,c]) * (sum_c deq(x)[r,c] deq(w_up)[e,f,c]),
  *   y_perm[r,c] = sum_f deq(hq)[r,f] deq(w_down)[e,c,f]   (fp32 accumulation, bf16 out). */
 moe_status moe_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* args, void* stream);

@@ -3,15 +3,21 @@
 //
 // One kernel, launched once for Linear-1 (gate | up, SwiGLU, h quantised in the epilogue) and once for Linear-2.
 // Persistent CTAs, one per SM, tiles assigned round-robin (tile t goes to CTA t mod grid).  A tile is 128 rows of one
-// expert x 192 accumulator columns: Linear-1 pairs 96 gate columns with the same 96 up columns, so a tile yields
-// 96 columns of h = three whole 32-element scale blocks, which the epilogue quantises straight from the fp32
-// accumulator (h never exists in bf16); Linear-2 writes 192 bf16 columns of y_perm.
+// expert x 256 accumulator columns: Linear-1 pairs 128 gate columns with the same 128 up columns, so a tile yields
+// 128 columns of h = four whole 32-element scale blocks, which the epilogue quantises straight from the fp32
+// accumulator (h never exists in bf16); Linear-2 writes 256 bf16 columns of y_perm.
 //
-// Roles (320 threads): warp 0 = TMA producer (codes of A and of two 96-row weight boxes per 128-element K stage),
+// Tensor memory (512 columns) holds ONE 256-column accumulator plus 4 columns of A scales and 8 of B scales; two
+// accumulators and the scales do not fit, and a 192-column tile with two accumulators was measured 13-15 % slower:
+// an MMA costs about the same clocks in the running kernel at N = 192 as at N = 256.  So the epilogue does not
+// overlap the next tile's mainloop; eight epilogue warps (two per lane quarter, half of the columns each) keep it
+// short (the MMA thread waits for the accumulator 14 % of the time in Linear-1 on the Mixtral-like layer).
+//
+// Roles (448 threads): warp 0 = TMA producer (codes of A and of two 128-row weight boxes per 128-element K stage),
 // warps 6-9 = scale loaders (one word per operand row per stage, loaded four stages ahead into registers and
-// stored in the 512-byte layout tcgen05.cp expects, then a proxy fence and an arrival on the stage's full barrier), warp 1 = MMA issuer (per
-// stage: three tcgen05.cp of scales into tensor memory, then four MMAs picking scale byte 0..3), warps 2-5 =
-// epilogue.  Tensor memory: two accumulators of 192 columns, 4 columns of A scales, 8 of B scales.
+// stored in the 512-byte layout tcgen05.cp expects, then a proxy fence and an arrival on the stage's full barrier),
+// warp 1 = MMA issuer (per stage: three tcgen05.cp of scales into tensor memory, then four MMAs picking scale byte
+// 0..3), warps 2-5 and 10-13 = epilogue.  Four stages of 49.5 KB.
 // Every wait is bounded; a wait that gives up is reported through the status word and the CTA unwinds.
 #include <cuda_bf16.h>
 
@@ -22,9 +28,9 @@
 
 namespace {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 448;
 constexpr int BM = 128;                 // rows per tile
-constexpr int BNH = 96;                 // rows of one weight box
+constexpr int BNH = 128;                // rows of one weight box
 constexpr int BN = 2 * BNH;             // accumulator columns
 constexpr int BK = 128;                 // K elements (= bytes) per stage: one 128-byte swizzle row
 constexpr int UMMA_K = 32;
@@ -33,10 +39,11 @@ constexpr int kBBoxBytes = BNH * BK;
 constexpr int kOperandBytes = kABytes + 2 * kBBoxBytes;
 constexpr int kSfABytes = 512;          // 128 rows x 4 scale bytes
 constexpr int kSfBytes = kSfABytes + 1024;
-constexpr int kStages = 5;
+constexpr int kStages = 4;
+constexpr int kAccBufs = 1;               // accumulators in tensor memory (two would leave no room for the scales)
 constexpr int kTmemCols = 512;
-constexpr uint32_t kTmemSfA = 2 * BN;   // column of the A scales
-constexpr uint32_t kTmemSfB = 2 * BN + 4;
+constexpr uint32_t kTmemSfA = kAccBufs * BN;   // column of the A scales
+constexpr uint32_t kTmemSfB = kAccBufs * BN + 4;
 constexpr int kSfThreads = 128;
 constexpr int kKernelIdMx = 9;          // in the detail word of a time-out: 9 * 65536 + role
 
@@ -44,7 +51,7 @@ struct MxParams {
   const int32_t* offsets;   // [E+1]
   int E;
   int N;                    // output columns of this GEMM: F (Linear-1) or H (Linear-2)
-  int n_blocks;             // tiles along N: ceil(N / 96) gated, ceil(N / 192) otherwise
+  int n_blocks;             // tiles along N: ceil(N / 128) gated, ceil(N / 256) otherwise
   int k_blocks;             // K / 128
   long long a_rows;         // R
   long long b_rows;         // E * N: rows of each weight matrix
@@ -120,7 +127,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(ptx::smem_u32(&st->tmem_full[a]), 1);
-      ptx::mbar_init(ptx::smem_u32(&st->tmem_empty[a]), 4);          // one arrival per epilogue warp
+      ptx::mbar_init(ptx::smem_u32(&st->tmem_empty[a]), 8);          // one arrival per epilogue warp
     }
     st->abort_flag = 0;
     st->blk_prefix[0] = 0;
@@ -156,7 +163,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
 
   const uint32_t tmem_base = st->tmem_base;
   const int total_tiles = st->blk_prefix[p.E] * p.n_blocks;
-  const int b1_shift = kGated ? 0 : BNH;       // second weight box: same rows of the up matrix, or the next 96 rows
+  const int b1_shift = kGated ? 0 : BNH;       // second weight box: same rows of the up matrix, or the next 128 rows
   volatile int* abort_flag = &st->abort_flag;
 
   if (warp == 0) {
@@ -232,8 +239,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         }
         if (!ok) break;
         ptx::tc_commit(ptx::smem_u32(&st->tmem_full[acc]));
-        acc ^= 1;
-        if (acc == 0) acc_phase ^= 1u;
+        if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
         ++n_tiles;
       }
       if (p.trace) {
@@ -243,9 +249,10 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       }
     }
     __syncwarp();
-  } else if (warp < 6) {
-    // ------------------------------------------------------------------ epilogue (4 warps = 128 rows)
+  } else if (warp < 6 || warp >= 10) {
+    // ------------------------------------------------------------------ epilogue (2 x 4 warps: 128 rows x two column halves)
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
+    const int half = warp >= 10 ? 1 : 0;          // which half of the tile's columns this warp drains
     int acc = 0;
     uint32_t acc_phase = 0;
     long long w_acc = 0, busy = 0;
@@ -262,7 +269,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       const bool row_ok = row < tile.row_end;
       if constexpr (kGated) {
 #pragma unroll 1
-        for (int j = 0; j < BNH / 32; ++j) {
+        for (int j = half * (BNH / 64); j < (half + 1) * (BNH / 64); ++j) {
           const int col = tile.n0 + 32 * j;
           if (col >= p.N) break;                  // N is a multiple of 32: blocks are whole
           uint32_t g[32], u[32];
@@ -288,7 +295,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         }
       } else {
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
           const int col = tile.n0 + c0;
           if (col >= p.N) break;
           uint32_t v[32];
@@ -309,8 +316,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
       busy += clock64() - t_drain;
-      acc ^= 1;
-      if (acc == 0) acc_phase ^= 1u;
+      if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
     }
     if (p.trace && warp == 2 && lane == 0) {
       p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
@@ -326,7 +332,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     // per warp whatever the addresses, a quarter of the shared-memory pipe at this kernel's rate.
     const int idx = 32 * (lane & 3) + 8 * w4 + (lane >> 2);
     const uint32_t dst_a = (idx & 31) * 16 + (idx >> 5) * 4;
-    const int n1 = idx + kSfThreads;              // second weight row of this thread (only below 192)
+    const int n1 = idx + kSfThreads;              // second weight row of this thread
     const uint32_t dst_b1 = 512 + (n1 & 31) * 16 + ((n1 & 127) >> 5) * 4;
     constexpr int kPrefetch = 4;
 
@@ -337,7 +343,7 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       if (pf_t >= total_tiles) return;
       const MxTile tile = decode_tile<kGated>(pf_t, st, p);
       const long long a_row = static_cast<long long>(tile.row0) + idx;
-      // weight row n of the tile: rows 0..95 come from the first box, 96..191 from the second
+      // weight row n of the tile: rows 0..127 come from the first box, 128..255 from the second
       const long long b_row_0 = idx < BNH ? static_cast<long long>(tile.w_row0) + idx
                                           : static_cast<long long>(tile.w_row0) + b1_shift + (idx - BNH);
       const long long b_row_1 = static_cast<long long>(tile.w_row0) + b1_shift + (n1 - BNH);
