@@ -11,7 +11,8 @@
 // accumulators and the scales do not fit, and a 192-column tile with two accumulators was measured 13-15 % slower:
 // an MMA costs about the same clocks in the running kernel at N = 192 as at N = 256.  So the epilogue does not
 // overlap the next tile's mainloop; eight epilogue warps (two per lane quarter, half of the columns each) keep it
-// short (the MMA thread waits for the accumulator 14 % of the time in Linear-1 on the Mixtral-like layer).
+// short, and each hands the accumulator back right after its last load from tensor memory (the MMA thread waits
+// for the accumulator 10 % of the time in Linear-1 on the Mixtral-like layer).
 //
 // Roles (448 threads): warp 0 = TMA producer (codes of A and of two 128-row weight boxes per 128-element K stage),
 // warps 6-9 = scale loaders (one word per operand row per stage, loaded four stages ahead into registers and
@@ -267,15 +268,26 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
       const int row = tile.row0 + quarter * 32 + lane;
       const bool row_ok = row < tile.row_end;
+      const uint32_t empty_bar = ptx::smem_u32(&st->tmem_empty[acc]);
+      auto release = [&]() {            // one arrival per warp and tile: its loads from the accumulator are complete
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(empty_bar);
+      };
       if constexpr (kGated) {
+        // this warp's blocks of 32 h columns (N is a multiple of 32: blocks are whole); the accumulator is handed
+        // back right after the warp's last load from tensor memory, before that block is processed and stored
+        const int jb = half * (BNH / 64);
+        const int je = min((half + 1) * (BNH / 64), (p.N - tile.n0) / 32);
+        if (je <= jb) release();
 #pragma unroll 1
-        for (int j = half * (BNH / 64); j < (half + 1) * (BNH / 64); ++j) {
+        for (int j = jb; j < je; ++j) {
           const int col = tile.n0 + 32 * j;
-          if (col >= p.N) break;                  // N is a multiple of 32: blocks are whole
           uint32_t g[32], u[32];
           ptx::tmem_ld_32x32(t_addr + 32 * j, g);
           ptx::tmem_ld_32x32(t_addr + BNH + 32 * j, u);
           ptx::tmem_ld_wait();
+          if (j == je - 1) release();
           float h[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) h[i] = silu_mul(__uint_as_float(g[i]), __uint_as_float(u[i]));
@@ -294,13 +306,16 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
           }
         }
       } else {
+        const int cb = half * (BN / 2);
+        const int ce = min((half + 1) * (BN / 2), p.N - tile.n0);
+        if (ce <= cb) release();
 #pragma unroll 1
-        for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+        for (int c0 = cb; c0 < ce; c0 += 32) {
           const int col = tile.n0 + c0;
-          if (col >= p.N) break;
           uint32_t v[32];
           ptx::tmem_ld_32x32(t_addr + c0, v);
           ptx::tmem_ld_wait();
+          if (c0 + 32 >= ce) release();
           if (row_ok) {
             uint4* dst = reinterpret_cast<uint4*>(p.y + static_cast<size_t>(row) * p.N + col);
 #pragma unroll
@@ -312,9 +327,6 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
           }
         }
       }
-      ptx::tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
       busy += clock64() - t_drain;
       if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
     }
