@@ -80,32 +80,102 @@ route_hist_ids(const int32_t* __restrict__ topk_ids, int T, int E, int k, int to
   for (int e = tid; e < E; e += kRouteThreads) chunk_hist[static_cast<size_t>(chunk) * E + e] = s_hist[e];
 }
 
-// One CTA of 1024 threads, E <= 1024: thread e walks the chunks of expert e, then a block scan over e.
+// One CTA of 1024 threads, E <= 1024.  With few experts (at least 8 threads per expert) and at least 64 chunks the
+// chunks are cut into
+// S = min(1024 / E, num_chunks) segments; thread (expert e, segment s) = e + s * E sums its segment (independent
+// loads, consecutive e side by side), the segment sums are scanned over s in shared memory, then the thread writes
+// the exclusive prefixes of its chunks.  With many experts one thread per expert walks all chunks once.  A block scan
+// over the experts' totals gives the offsets.
 __global__ void __launch_bounds__(1024)
 route_scan(const int32_t* __restrict__ chunk_hist, int32_t* __restrict__ chunk_base, int num_chunks, int E,
            int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
   __shared__ int32_t s_warp[32];
-  const int e = threadIdx.x, lane = e & 31, warp = e >> 5;
-  int32_t total = 0;
-  if (e < E) {
-    // eight chunks per step: the loads are independent, only the running sum is serial
-    int c = 0;
-    for (; c + 8 <= num_chunks; c += 8) {
+  __shared__ int32_t s_seg[2][1024];      // [buffer][s * E + e]: inclusive scan over s, ping-pong
+  __shared__ int32_t s_total[1024];       // per expert
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int S = 1024 / E;
+  if (S > num_chunks) S = num_chunks;
+  if (S < 1) S = 1;
+  // many experts or few chunks: one thread per expert walks all chunks once (no second pass, no segment scan)
+  if (S < 8 || num_chunks < 64) S = 1;
+  const int seg_len = (num_chunks + S - 1) / S;
+  const int e_of = tid % E, seg = tid / E;
+  const bool active = seg < S;
+  const int c_begin = seg * seg_len;
+  const int c_end = min(num_chunks, c_begin + seg_len);
+  int32_t sum = 0;
+  if (S == 1) {
+    // single pass: the prefix is written while summing
+    if (active) {
+      int c = 0;
+      for (; c + 8 <= num_chunks; c += 8) {
+        int32_t v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = chunk_hist[static_cast<size_t>(c + u) * E + e_of];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          chunk_base[static_cast<size_t>(c + u) * E + e_of] = sum;
+          sum += v[u];
+        }
+      }
+      for (; c < num_chunks; ++c) {
+        const size_t i = static_cast<size_t>(c) * E + e_of;
+        const int32_t v = chunk_hist[i];
+        chunk_base[i] = sum;
+        sum += v;
+      }
+      s_total[e_of] = sum;
+    }
+  } else if (active) {
+    int c = c_begin;
+    for (; c + 8 <= c_end; c += 8) {        // eight independent loads per step
       int32_t v[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = chunk_hist[static_cast<size_t>(c + u) * E + e];
+      for (int u = 0; u < 8; ++u) v[u] = chunk_hist[static_cast<size_t>(c + u) * E + e_of];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) sum += v[u];
+    }
+    for (; c < c_end; ++c) sum += chunk_hist[static_cast<size_t>(c) * E + e_of];
+    s_seg[0][tid] = sum;
+  }
+  __syncthreads();
+  // inclusive scan over the segments of each expert (entries e + s * E, stride E); nothing to do for one segment
+  int cur = 0;
+  for (int off = 1; off < S; off <<= 1) {
+    if (active) {
+      int32_t v = s_seg[cur][tid];
+      if (seg >= off) v += s_seg[cur][tid - off * E];
+      s_seg[cur ^ 1][tid] = v;
+    }
+    cur ^= 1;
+    __syncthreads();
+  }
+  if (active && S > 1) {
+    int32_t running = s_seg[cur][tid] - sum;                 // slots of this expert in earlier segments
+    int c = c_begin;
+    for (; c + 8 <= c_end; c += 8) {        // eight loads in flight, then the eight prefixes
+      int32_t v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = chunk_hist[static_cast<size_t>(c + u) * E + e_of];
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
-        chunk_base[static_cast<size_t>(c + u) * E + e] = total;
-        total += v[u];
+        chunk_base[static_cast<size_t>(c + u) * E + e_of] = running;
+        running += v[u];
       }
     }
-    for (; c < num_chunks; ++c) {
-      const size_t i = static_cast<size_t>(c) * E + e;
+    for (; c < c_end; ++c) {
+      const size_t i = static_cast<size_t>(c) * E + e_of;
       const int32_t v = chunk_hist[i];
-      chunk_base[i] = total;
-      total += v;
+      chunk_base[i] = running;
+      running += v;
     }
+    if (seg == S - 1) s_total[e_of] = s_seg[cur][tid];       // inclusive over all segments = the expert's count
+  }
+  __syncthreads();
+  const int e = tid;
+  int32_t total = 0;
+  if (e < E) {
+    total = s_total[e];
     counts[e] = total;
   }
   int32_t incl = total;
