@@ -488,6 +488,12 @@ def main():
             "bytes_per_launch": l1_bytes, "ms_per_launch": kernel_ms[4], "nonempty_experts": nonempty,
             "tensor_tflops": l1_tf,
         }
+    # The cuBLAS peak was measured at its own SM clock under the power cap; this kernel ran at sm_mhz_kernel (its
+    # clock64 span over its CUDA-event time).  frac x (peak's clock / this clock) compares flops per clock.
+    peak_mhz = float((peaks.get("clocks_under_load") or {}).get("sm_mhz_median") or 0.0)
+    if roofline["bound"] == "tensor" and peak_mhz > 0 and clocks and clocks.get("sm_mhz_kernel"):
+        roofline["peak_sm_mhz"] = peak_mhz
+        roofline["frac_at_equal_clock"] = roofline["frac"] * peak_mhz / clocks["sm_mhz_kernel"]
     line = {
         "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
