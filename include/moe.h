@@ -62,10 +62,10 @@ typedef struct {
   int32_t interleave_mode;         /* 0 or 1 */
   int32_t interleave_k;            /* 1, 2 or 4; used when interleave_mode == 1 */
   int32_t schedule;                /* 0 = Expert-Wave order (Sec. 4.3): all Linear-1 tiles, then all Linear-2 tiles;
-                                      1 = interleaved order (Algorithm 1): every CTA g of G walks strided cursors
-                                      k1, k2 += G over the row-major Linear-1 / Linear-2 tile lists (a row is one
-                                      128-row block) and emits the Linear-2 tile only while Linear-1 leads by
-                                      dep_lead_D rows; one launch, Linear-2 tiles wait for their row's h.
+                                      1 = interleaved order (Algorithm 1): both tile lists row-major (a row is one
+                                      128-row block), CTA g of G owns tiles g, g+G, ... of each and places its
+                                      Linear-2 tiles between its Linear-1 tiles as early as a lead of dep_lead_D
+                                      rows allows; one launch, Linear-2 tiles wait for their row's h.
                                       Values are bitwise identical for both schedules. */
   int32_t dep_lead_D;              /* schedule 1: minimum row lead D >= 1 of Linear-1 over Linear-2; 0 = the
                                       anti-starvation knee ceil(128 * SMs / (2 F)) (App. A.2).  Must be 0 for
@@ -79,6 +79,19 @@ typedef struct {
                                       the CTA-pair kernel for two-launch runs, bit 4: never use it (by default it
                                       runs when the layer averages at least 1024 rows per expert); other bits 0 */
 } moe_tuning;
+
+/*
+ * Environment override for sweeps (no counterpart in the paper).  moe_create reads the variable MOE_TUNING once:
+ * a comma-separated list of key=value entries with the keys burst, mode, k, schedule, lead, flags (the six fields
+ * above, in that order; fields not named keep their defaults 1, 0, 1, 0, 0, 0).  The result replaces the built-in
+ * default that a call uses when it is given tuning = NULL; a call that passes a moe_tuning is not affected.
+ * Entries "x.<name>=<int>" are development knobs of individual kernels (unstable, undocumented on purpose: they
+ * select between variants under measurement and never change results).  An unknown key, a malformed number or a
+ * combination moe_tuning does not allow makes moe_create return MOE_ERR_INVALID_ARG.
+ * moe_parse_tuning applies the same parser to `text` (NULL = empty) without touching the environment or a device:
+ * *out_tuning receives the fields, *out_named_field (may be NULL) 1 when at least one of the six keys was named.
+ */
+moe_status moe_parse_tuning(const char* text, moe_tuning* out_tuning, int32_t* out_named_field);
 
 /* Byte offsets of the slices of the workspace used by moe_fused_forward (each 256-byte aligned). */
 typedef struct {
@@ -167,8 +180,10 @@ moe_status moe_plan_routing_from_topk(moe_ctx* ctx, const int32_t* topk_ids, int
  * Same inputs, outputs and results as moe_plan_routing (shape->T, E, k are used; H and F are ignored).
  *   - Limit: ceil(T / floor(256/k)) * E <= 65536, e.g. T <= 8192 at E = 256, k = 8.  Beyond it the call
  *     returns MOE_ERR_STATIC_SCRATCH_TOO_SMALL and launches nothing.
- *   - The first call on each device looks up the array's device address (with that device current).
- *     Make that first call outside any stream capture.
+ *   - The first call on each device that passes the argument checks (a call with T = 0 counts) looks up
+ *     the array's device address, with that device current.  Make that first call outside any stream
+ *     capture.  Host threads may make it concurrently: the lookup is idempotent and its result is
+ *     published atomically.
  *   - All calls on a device share the one array.  Nothing in it has to start at zero (each call
  *     rewrites every entry it later reads), so calls may follow one another on a stream freely; two
  *     calls that overlap on the GPU (different streams, no ordering) race on it and give wrong plans.

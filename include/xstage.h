@@ -73,9 +73,9 @@ double xstage_mma_stall(double t_remote_store_span, double t_cover_mma);
 int64_t xstage_fa_recovery_length(int64_t b_n, double recovery_gap, double sigma);
 
 /*
- * Store microbenchmark on this GPU's own memory (Sec. 3.1's periodic-burst and isolated-burst patterns, run as the
- * paper's local-memory control: same producer count, store width, address generation and loop structure, local
- * destination).  `producers` CTAs of 128 threads, one per SM (producers <= SM count), start together; each
+ * Store microbenchmark on this GPU's own memory: the periodic-burst and isolated-burst patterns of Sec. 3.1, run
+ * the way the paper runs its local-memory control (Sec. 3.2), i.e. the identical store kernel with only the
+ * destination changed from a peer's memory to this GPU's.  `producers` CTAs of 128 threads, one per SM (producers <= SM count), start together; each
  * repeats `periods` times: issue bytes_per_burst bytes (a multiple of 16) as 16-byte stores into its own slice of
  * device_buffer (DEVICE pointer, 16-byte aligned, buffer_bytes / producers >= bytes_per_burst; slices are walked
  * and wrap, so a buffer well above the L2 size keeps the stores going to HBM), then spin gap_clocks SM clocks
@@ -84,7 +84,8 @@ int64_t xstage_fa_recovery_length(int64_t b_n, double recovery_gap, double sigma
  * mean / maximum over producers of the sender-visible issue span of burst n (first store issued to last store
  * issued, not completion); period_mean_clocks = mean period n (issue + gap).  *clocks_per_us (may be NULL) = SM
  * clocks per microsecond during the run (clock64 against globaltimer).  Allocates and frees a small device result
- * buffer, runs on the current device, synchronises `stream`.  Returns 0, -1 bad argument, -2 CUDA error,
+ * buffer, runs on the current device, synchronises `stream`.  gap_clocks x periods is limited to 4e9 clocks (about
+ * two seconds of spinning on every SM); more is a bad argument.  Returns 0, -1 bad argument, -2 CUDA error,
  * -3 the producers could not be started together within the wait budget.
  */
 int xstage_store_probe(int32_t producers, int64_t bytes_per_burst, int64_t gap_clocks, int32_t periods,

@@ -29,6 +29,7 @@ EXPORTS = (
     "moe_set_active_tokens", "moe_plan_routing_from_topk", "moe_router_weight_bytes", "moe_router_scratch_bytes",
     "moe_router_prepare", "moe_route_tokens", "moe_fused_forward_routed", "moe_quantize_rows_mx", "moe_dispatch_mx",
     "moe_expert_ffn_mx", "moe_get_workspace_layout_mx", "moe_fused_forward_mx", "moe_probe_mma_cycles_kind",
+    "moe_parse_tuning",
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
@@ -173,6 +174,15 @@ def _check(code: int, where: str):
 
 def make_tuning(store_burst_tiles=1, interleave_mode=0, interleave_k=1, schedule=0, dep_lead_D=0, debug_flags=0):
     return moe_tuning(store_burst_tiles, interleave_mode, interleave_k, schedule, dep_lead_D, debug_flags)
+
+
+def moe_parse_tuning(text):
+    """Parse a MOE_TUNING string.  Returns (moe_tuning, named_field: bool); raises MoeError on a bad string."""
+    t = moe_tuning()
+    named = C.c_int32(0)
+    _check(load_library().moe_parse_tuning(None if text is None else text.encode(), C.byref(t), C.byref(named)),
+           "moe_parse_tuning")
+    return t, bool(named.value)
 
 
 def _tuning_ref(tuning):

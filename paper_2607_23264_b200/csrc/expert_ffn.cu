@@ -22,9 +22,9 @@
 //      the order merges the hot and the cold tile lists at a fixed ratio so that both finish together, and
 //      CTAs draw tiles dynamically from one atomic counter.  Run as two launches (the kernel boundary is the
 //      Linear-1 -> Linear-2 dependency) or as one launch with per-block ready counters.
-//   1  Interleaved (Algorithm 1 of the paper): each CTA g of G walks two strided cursors k1, k2 over the
-//      row-major Linear-1 and Linear-2 tile lists (row = one 128-row block) and emits the Linear-2 tile only
-//      while Linear-1 leads by D rows, else the next Linear-1 tile.  One launch; a Linear-2 tile waits (bounded)
+//   1  Interleaved (Algorithm 1 of the paper): both GEMMs' tiles are listed row-major (row = one 128-row block),
+//      CTA g of G owns tiles g, g+G, ... of each list and splices its Linear-2 tiles between its Linear-1 tiles as
+//      early as a row lead of D allows (InterleaveCursor below).  One launch; a Linear-2 tile waits (bounded)
 //      until all Linear-1 tiles of its row have published their h rows.
 // An expert with at most 64 rows is computed with the operands swapped: each 128-row weight box is the MMA's M
 // side and the expert's rows, padded to a multiple of 16, its N side.  A tcgen05.mma costs 128 clocks at N = 256 but
@@ -32,8 +32,6 @@
 // shared-memory stage is the same three boxes, only the MMA issue and the epilogue (lane = output column) differ.
 // Layers whose experts hold many rows run the CTA-pair variant further down (256-row tiles, cta_group::2).
 #include <cuda_bf16.h>
-
-#include <climits>
 
 #include "ffn_math.cuh"
 #include "moe_internal.h"
@@ -177,6 +175,29 @@ __device__ __forceinline__ Tile decode_tile(int code, const SharedTail* st, cons
   const int n_blk = local / mb;
   return make_tile(phase, e, local - n_blk * mb, n_blk, st, p);
 }
+
+// Schedule 1 (the paper's Algorithm 1): a CTA owns every stride-th tile of each GEMM's row-major tile list and keeps
+// the tiles of one GEMM in list order; what is decided per draw is only which GEMM goes next.  Linear-2 goes when
+// it has a tile left whose row lies at least `lead` rows behind the row of the CTA's pending Linear-1 tile (or
+// Linear-1 has none left); otherwise Linear-1 goes.  Returns the tile code, -1 when both lists are exhausted.
+struct InterleaveCursor {
+  int next1, next2;   // this CTA's pending tile of Linear-1 / Linear-2
+  int stride;         // scheduler instances = CTAs of the launch
+  __device__ __forceinline__ int draw(int tiles1, int tiles2, int per_row1, int per_row2, int lead) {
+    const bool left1 = next1 < tiles1, left2 = next2 < tiles2;
+    if (!left1 && !left2) return -1;
+    const bool linear2_may_go = left2 && (!left1 || next2 / per_row2 + lead <= next1 / per_row1);
+    int code;
+    if (linear2_may_go) {
+      code = (1 << kPhaseShift) | next2;
+      next2 += stride;
+    } else {
+      code = next1;
+      next1 += stride;
+    }
+    return code;
+  }
+};
 
 __device__ __forceinline__ void report_timeout(const FfnParams& p, int role) {
   atomicCAS(&p.status[0], 0, MOE_ERR_TIMEOUT);
@@ -446,7 +467,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       uint32_t ring_phase = 0;
       bool ok = true;
       long long w_empty = 0;
-      int k1 = blockIdx.x, k2 = blockIdx.x;   // Algorithm 1 cursors of scheduler instance g = blockIdx.x
+      InterleaveCursor cursor{static_cast<int>(blockIdx.x), static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)};
       int n_drawn = 0;
       const long long t_begin = clock64();
       while (ok) {
@@ -457,17 +478,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // ---- next tile of this CTA
         int code = -1;
         if (p.schedule == 1) {
-          if (k1 < tiles1 || k2 < tiles2) {
-            const int p1 = k1 < tiles1 ? k1 / p.ph[0].n_blocks : INT_MAX;   // row of the next Linear-1 tile
-            const int p2 = k2 / p.ph[1].n_blocks;
-            if (k2 < tiles2 && p2 <= p1 - p.lead_D) {
-              code = (1 << kPhaseShift) | k2;
-              k2 += gridDim.x;
-            } else {
-              code = k1;
-              k1 += gridDim.x;
-            }
-          }
+          code = cursor.draw(tiles1, tiles2, p.ph[0].n_blocks, p.ph[1].n_blocks, p.lead_D);
         } else {
           const int pos = atomicAdd(&p.sched[0], 1);
           if (pos < tiles1) code = pos;
@@ -1123,8 +1134,8 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   const moe_shape& s = ctx->shape;
   const uint64_t R = static_cast<uint64_t>(s.T) * s.k;
   if (R == 0) return MOE_OK;
-  moe_tuning tn = {1, 0, 1, 0, 0, 0};
-  if (tuning) tn = *tuning;
+  const moe_tuning tn = moe_effective_tuning(ctx, tuning);
+  if (c.fp8 && (tn.schedule != 0 || (tn.debug_flags & 6) != 0)) return MOE_ERR_UNSUPPORTED;   // bf16-only modes
   const int eb = c.fp8 ? 1 : 2;
   const int k_elems = 128 / eb;
 

@@ -1,5 +1,7 @@
 // Host side of the C ABI (include/moe.h): argument validation, context, workspace carving, call order.
+#include <climits>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -29,6 +31,52 @@ moe_status check_tuning(const moe_tuning* t) {
   if (t->dep_lead_D < 0 || (t->schedule == 0 && t->dep_lead_D != 0) || (t->debug_flags & ~31) != 0)
     return MOE_ERR_INVALID_ARG;
   return MOE_OK;
+}
+
+// One "key=value" entry of MOE_TUNING.  Returns false on an unknown key or a malformed number.
+bool apply_tuning_entry(const char* key, size_t key_len, const char* val, moe_tuning* t, int* named_field,
+                        moe_knob* knobs, int* num_knobs) {
+  char* end = nullptr;
+  const long v = std::strtol(val, &end, 0);
+  if (end == val || (*end != 0 && *end != ',') || v < INT32_MIN || v > INT32_MAX) return false;
+  auto is = [&](const char* name) { return std::strlen(name) == key_len && std::strncmp(key, name, key_len) == 0; };
+  int32_t* field = is("burst") ? &t->store_burst_tiles : is("mode") ? &t->interleave_mode : is("k") ? &t->interleave_k
+                 : is("schedule") ? &t->schedule : is("lead") ? &t->dep_lead_D : is("flags") ? &t->debug_flags : nullptr;
+  if (field) {
+    *field = static_cast<int32_t>(v);
+    *named_field = 1;
+    return true;
+  }
+  if (key_len > 2 && key[0] == 'x' && key[1] == '.' && key_len - 2 < sizeof(knobs[0].name)) {
+    if (!knobs || !num_knobs) return true;
+    if (*num_knobs >= kMoeMaxKnobs) return false;
+    moe_knob& k = knobs[(*num_knobs)++];
+    std::memcpy(k.name, key + 2, key_len - 2);
+    k.name[key_len - 2] = 0;
+    k.value = static_cast<int32_t>(v);
+    return true;
+  }
+  return false;
+}
+
+moe_status parse_tuning_text(const char* text, moe_tuning* t, int* named_field, moe_knob* knobs, int* num_knobs) {
+  *t = moe_tuning{1, 0, 1, 0, 0, 0};
+  *named_field = 0;
+  if (num_knobs) *num_knobs = 0;
+  if (!text) return MOE_OK;
+  const char* p = text;
+  while (*p) {
+    while (*p == ',' || *p == ' ') ++p;
+    if (!*p) break;
+    const char* eq = p;
+    while (*eq && *eq != '=' && *eq != ',') ++eq;
+    if (*eq != '=' || eq == p) return MOE_ERR_INVALID_ARG;
+    if (!apply_tuning_entry(p, static_cast<size_t>(eq - p), eq + 1, t, named_field, knobs, num_knobs))
+      return MOE_ERR_INVALID_ARG;
+    p = eq + 1;
+    while (*p && *p != ',') ++p;
+  }
+  return *named_field ? check_tuning(t) : MOE_OK;
 }
 
 moe_status check_ctx(const moe_ctx* ctx) {
@@ -114,11 +162,24 @@ moe_status moe_get_workspace_layout(const moe_shape* shape, moe_workspace_layout
   return MOE_OK;
 }
 
+moe_status moe_parse_tuning(const char* text, moe_tuning* out_tuning, int32_t* out_named_field) {
+  if (!out_tuning) return MOE_ERR_INVALID_ARG;
+  int named = 0;
+  const moe_status st = parse_tuning_text(text, out_tuning, &named, nullptr, nullptr);
+  if (out_named_field) *out_named_field = named;
+  return st;
+}
+
 moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   if (!out_ctx) return MOE_ERR_INVALID_ARG;
   *out_ctx = nullptr;
   const moe_status st = check_shape(shape);
   if (st != MOE_OK) return st;
+  moe_tuning env_tuning;
+  moe_knob env_knobs[kMoeMaxKnobs];
+  int env_named = 0, env_knob_count = 0;
+  if (parse_tuning_text(std::getenv("MOE_TUNING"), &env_tuning, &env_named, env_knobs, &env_knob_count) != MOE_OK)
+    return MOE_ERR_INVALID_ARG;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
   if (dev != device) return MOE_ERR_INVALID_ARG;
@@ -128,6 +189,10 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   ctx->shape = *shape;
   ctx->device = device;
   ctx->last_launches = 0;
+  ctx->has_env_tuning = env_named;
+  ctx->env_tuning = env_tuning;
+  ctx->num_knobs = env_knob_count;
+  std::memcpy(ctx->knobs, env_knobs, sizeof(env_knobs));
   if (cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
     delete ctx;
     return MOE_ERR_CUDA;

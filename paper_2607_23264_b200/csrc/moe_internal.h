@@ -23,8 +23,19 @@ typedef CUresult (*moe_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuin
                                         CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                         CUtensorMapFloatOOBfill);
 
+// Development knobs given as "x.<name>=<int>" entries of the MOE_TUNING environment variable (see moe_create).
+constexpr int kMoeMaxKnobs = 16;
+struct moe_knob {
+  char name[24];
+  int32_t value;
+};
+
 struct moe_ctx {
   moe_shape shape;
+  int has_env_tuning;    // MOE_TUNING named at least one moe_tuning field: env_tuning replaces the defaults of a
+  moe_tuning env_tuning; // call that passes tuning = NULL
+  int num_knobs;
+  moe_knob knobs[kMoeMaxKnobs];
   int device;
   int num_sms;
   int max_pairs;         // CTA pairs (clusters of two) of the pair kernel that can be resident at once
@@ -50,6 +61,23 @@ struct moe_ctx {
   uint32_t ev_recorded;          // bit i set when ev[i] was recorded by the last call
   cudaEvent_t ev[kMoeKernels + 1];
 };
+
+// Value of the development knob "x.<name>" from MOE_TUNING, or dflt.
+inline int moe_knob_value(const moe_ctx* ctx, const char* name, int dflt) {
+  for (int i = 0; i < ctx->num_knobs; ++i) {
+    const char *a = ctx->knobs[i].name, *b = name;
+    while (*a && *a == *b) { ++a; ++b; }
+    if (*a == 0 && *b == 0) return ctx->knobs[i].value;
+  }
+  return dflt;
+}
+
+// The tuning a call runs with: the caller's, else the one MOE_TUNING gave at moe_create, else the built-in default.
+inline moe_tuning moe_effective_tuning(const moe_ctx* ctx, const moe_tuning* given) {
+  if (given) return *given;
+  if (ctx->has_env_tuning) return ctx->env_tuning;
+  return moe_tuning{1, 0, 1, 0, 0, 0};
+}
 
 // Record timing mark i on the stream when per-kernel timing is enabled.
 inline void moe_mark(moe_ctx* ctx, int i, cudaStream_t stream) {
@@ -89,7 +117,7 @@ cudaError_t launch_quantize_rows(moe_ctx* ctx, const void* in_bf16, long long ro
 cudaError_t launch_dispatch_fp8(moe_ctx* ctx, const void* xq, const float* sx, const int32_t* inv_perm,
                                 void* xq_perm, float* sx_perm, cudaStream_t stream);
 
-// Router front end.  Sizes of the prepared weights (three bf16 terms of W_r, expert rows padded) and of the scratch
+// Router front end.  Sizes of the prepared weights (two bf16 terms of W_r, expert rows padded) and of the scratch
 // for the K-split partial logits; the split of W_r; logits + top-k in one kernel (ids and weights only: the plan's
 // histogram, scan and scatter follow through launch_plan_from_topk).
 size_t router_weight_bytes(const moe_shape& s);

@@ -11,6 +11,8 @@
 //                        the chunk) + (earlier lanes in the warp, from a match-any ballot).
 // Everything is integer work on identical fp32 inputs, so ids, counts, offsets and both permutations are
 // reproducible bit for bit.
+#include <atomic>
+
 #include "moe_internal.h"
 #include "route_select.cuh"
 
@@ -286,7 +288,24 @@ constexpr int kStaticScratchInts = 65536;
 static __device__ __align__(256) int32_t g_route_static_scratch[2 * kStaticScratchInts];
 
 constexpr int kMaxDevices = 64;
-int32_t* g_route_static_addr[kMaxDevices] = {};   // device address of the array, per device, once resolved
+// device address of the array, per device, once resolved (host threads may race to resolve it: they store the
+// same value)
+std::atomic<int32_t*> g_route_static_addr[kMaxDevices];
+
+// Set-up, once per device, with that device current: in host code the array's name is only a stand-in, the address
+// a kernel may use comes from cudaGetSymbolAddress.  Returns nullptr on failure.
+int32_t* static_scratch_address() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  int32_t* scratch = g_route_static_addr[dev].load(std::memory_order_acquire);
+  if (!scratch) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_route_static_scratch) != cudaSuccess || !addr) return nullptr;
+    scratch = static_cast<int32_t*>(addr);
+    g_route_static_addr[dev].store(scratch, std::memory_order_release);
+  }
+  return scratch;
+}
 
 }  // namespace
 
@@ -300,6 +319,9 @@ extern "C" moe_status moe_plan_routing_static(const moe_shape* shape, const floa
   if (!counts || !offsets) return MOE_ERR_INVALID_ARG;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   const int T = shape->T, E = shape->E, k = shape->k;
+  // resolved before anything else that can succeed, so that any first call (an empty batch included) is the set-up
+  int32_t* scratch = static_scratch_address();
+  if (!scratch) return MOE_ERR_CUDA;
   if (T == 0) {
     if (cudaMemsetAsync(counts, 0, static_cast<size_t>(E) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
     if (cudaMemsetAsync(offsets, 0, static_cast<size_t>(E + 1) * 4, cs) != cudaSuccess) return MOE_ERR_CUDA;
@@ -314,17 +336,6 @@ extern "C" moe_status moe_plan_routing_static(const moe_shape* shape, const floa
   const long long num_chunks = (static_cast<long long>(T) + tokens_per_chunk - 1) / tokens_per_chunk;
   if (num_chunks * E > kStaticScratchInts) return MOE_ERR_STATIC_SCRATCH_TOO_SMALL;
 
-  // Set-up, once per device, with that device current: in host code the array's name is only a
-  // stand-in, the address a kernel may use comes from cudaGetSymbolAddress.
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MOE_ERR_CUDA;
-  int32_t* scratch = g_route_static_addr[dev];
-  if (!scratch) {
-    void* addr = nullptr;
-    if (cudaGetSymbolAddress(&addr, g_route_static_scratch) != cudaSuccess || !addr) return MOE_ERR_CUDA;
-    scratch = static_cast<int32_t*>(addr);
-    g_route_static_addr[dev] = scratch;
-  }
   int32_t* chunk_hist = scratch;                        // [num_chunks, E], every entry rewritten by kernel 1
   int32_t* chunk_base = scratch + kStaticScratchInts;   // [num_chunks, E], every entry rewritten by kernel 2
 

@@ -13,6 +13,7 @@ namespace {
 
 constexpr int kProbeThreads = 128;
 constexpr long long kStartBudget = 2000000000LL;   // clocks a producer waits for the others at the aligned start
+constexpr long long kMaxGapBudget = 4000000000LL;  // gap_clocks x periods may not exceed this (about 2 s of spinning)
 
 struct ProbeHeader {
   int arrived;        // producers that reached the start line
@@ -91,6 +92,8 @@ extern "C" int xstage_store_probe(int32_t producers, int64_t bytes_per_burst, in
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return -2;
   if (producers > sms) return -1;                      // one resident producer per SM, or the start line never fills
+  // the gaps are busy-waits on every SM: a gap given in the wrong unit must not occupy a shared GPU for minutes
+  if (gap_clocks > kMaxGapBudget / periods) return -1;
   const long long vec_per_burst = bytes_per_burst / 16;
   const long long vec_per_producer = static_cast<long long>(buffer_bytes / 16) / producers;
   if (vec_per_producer < vec_per_burst || (reinterpret_cast<uintptr_t>(device_buffer) & 15u)) return -1;

@@ -102,19 +102,38 @@ def assert_plan_matches(layer: Layer, ref: dict):
     assert np.abs(w - ref["topk_w"]).max() <= TOL_W
 
 
-def sample_tokens(cfg: gen.MoEConfig, plan: dict, n_random: int, seed: int, max_boundary: int = 64) -> np.ndarray:
-    """Tokens for the row-sampled oracle: seeded random ones plus owners of rows at expert and 128-row
-    tile boundaries (first/last rows of experts, rows next to a tile edge)."""
+def stratified_rows(cfg: gen.MoEConfig, plan: dict, seed: int) -> np.ndarray:
+    """Rows of the expert-contiguous buffer that between them touch every tile class of the grouped GEMMs:
+    the first and the last row of every non-empty expert, and one seeded-random row inside every 128-row block of
+    every expert.  A 128-row block is the unit every variant of the kernel is built from: each half of a 256-row
+    CTA-pair tile is one block, a block with few rows is a swapped-operand tile, the short last block of a larger
+    expert is its own tile; so no tile of the launch is left without a checked row."""
     rng = np.random.default_rng(seed)
-    toks = set(rng.choice(cfg.T, size=min(n_random, cfg.T), replace=False).tolist())
-    perm, offsets = plan["perm"], plan["offsets"]
+    offsets = plan["offsets"]
     rows = []
-    nonempty = [e for e in range(cfg.E) if offsets[e + 1] > offsets[e]]
-    for e in rng.permutation(nonempty)[:max_boundary // 4]:
+    for e in range(cfg.E):
         lo, hi = int(offsets[e]), int(offsets[e + 1])
+        if hi == lo:
+            continue
         rows += [lo, hi - 1]
-        if hi - lo > 128:
-            rows += [lo + 127, lo + 128]
-    for r in rows[:max_boundary]:
-        toks.add(int(perm[r]) // cfg.k)
-    return np.array(sorted(toks), dtype=np.int64)
+        for b0 in range(lo, hi, 128):
+            rows.append(int(rng.integers(b0, min(b0 + 128, hi))))
+    return np.unique(np.array(rows, dtype=np.int64))
+
+
+def stratified_tokens(cfg: gen.MoEConfig, plan: dict, n_random: int, seed: int):
+    """(tokens, rows): the owners of stratified_rows plus n_random seeded-random tokens, ascending."""
+    rows = stratified_rows(cfg, plan, seed)
+    rng = np.random.default_rng(seed + 1)
+    toks = set((plan["perm"][rows].astype(np.int64) // cfg.k).tolist())
+    toks.update(rng.choice(cfg.T, size=min(n_random, cfg.T), replace=False).tolist())
+    return np.array(sorted(toks), dtype=np.int64), rows
+
+
+def assert_rows_close(got: np.ndarray, ref: np.ndarray, what: str, tol: float = TOL_FRO):
+    """Relative Frobenius error over all rows together and of every row on its own."""
+    assert rel_fro(got, ref) <= tol, f"{what}: relative Frobenius error {rel_fro(got, ref):.2e}"
+    num = np.linalg.norm(got - ref, axis=1)
+    den = np.maximum(np.linalg.norm(ref, axis=1), 1e-30)
+    worst = int(np.argmax(num / den))
+    assert (num / den).max() <= tol, f"{what}: row {worst} has relative error {(num / den).max():.2e}"

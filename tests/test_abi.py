@@ -85,6 +85,23 @@ def test_null_arguments(lib):
     assert lib.moe_plan_routing(None, None, None, None, None, None, None, None, None) == 1
 
 
+def test_tuning_string_parser(lib):
+    """The parser behind the MOE_TUNING environment override (pure host code)."""
+    t, named = binding.moe_parse_tuning(None)
+    assert not named and (t.store_burst_tiles, t.interleave_mode, t.interleave_k, t.schedule, t.dep_lead_D,
+                          t.debug_flags) == (1, 0, 1, 0, 0, 0)
+    t, named = binding.moe_parse_tuning("burst=4,mode=1,k=2")
+    assert named and (t.store_burst_tiles, t.interleave_mode, t.interleave_k) == (4, 1, 2) and t.schedule == 0
+    t, named = binding.moe_parse_tuning("schedule=1, lead=8,flags=0x1")
+    assert named and (t.schedule, t.dep_lead_D, t.debug_flags) == (1, 8, 1)
+    t, named = binding.moe_parse_tuning("x.some_knob=3")
+    assert not named, "development knobs alone do not replace the default tuning"
+    for bad in ("burst=3", "bogus=1", "burst", "burst=", "k=1x", "lead=4", "mode=2", "=1"):
+        with pytest.raises(binding.MoeError) as ei:     # lead without schedule 1, values moe_tuning does not allow
+            binding.moe_parse_tuning(bad)
+        assert ei.value.code == 1, bad
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "_LIB_PATH", str(tmp_path / "nope.so"))

@@ -11,26 +11,39 @@ def all_orders(G, P, P1, P2, D):
     return [so.algorithm1_order(g, G, P, P1, P2, D) for g in range(G)]
 
 
-def test_every_tile_exactly_once_and_lead_respected():
-    for (G, P, P1, P2, D) in [(1, 3, 2, 1, 1), (4, 7, 5, 3, 2), (148, 37, 16, 28, 5), (148, 130, 112, 16, 1),
-                              (8, 1, 3, 2, 1), (5, 9, 4, 4, 0), (3, 6, 2, 5, 100)]:
-        orders = all_orders(G, P, P1, P2, D)
-        seen = [set(), set()]
-        for seq in orders:
-            done_l1_row = -1   # rows fully behind this instance's Linear-1 cursor
-            k1_next = None
-            emitted_l1 = [k for ph, k in seq if ph == 0]
-            for i, (ph, k) in enumerate(seq):
-                assert k not in seen[ph]
-                seen[ph].add(k)
+CASES = [(1, 3, 2, 1, 1), (4, 7, 5, 3, 2), (148, 37, 16, 28, 5), (148, 130, 112, 16, 1), (8, 1, 3, 2, 1),
+         (5, 9, 4, 4, 0), (3, 6, 2, 5, 100), (7, 11, 3, 9, 3), (2, 5, 1, 1, 2)]
+
+
+def test_every_tile_exactly_once_and_streams_keep_their_order():
+    for (G, P, P1, P2, D) in CASES:
+        seen = [[], []]
+        for g, seq in enumerate(all_orders(G, P, P1, P2, D)):
+            for ph in (0, 1):
+                own = [k for q, k in seq if q == ph]
+                assert own == list(range(g, P * (P1, P2)[ph], G)), "an instance walks its own stride, in order"
+                seen[ph] += own
+        assert sorted(seen[0]) == list(range(P * P1)) and sorted(seen[1]) == list(range(P * P2))
+
+
+def test_lead_is_respected_and_linear2_goes_at_the_first_chance():
+    """The two properties that, with the per-stream order above, fix the merge uniquely: a Linear-2 tile of row p
+    is never emitted while the instance's pending Linear-1 tile lies before row p + D (dependency lead), and a
+    Linear-1 tile is never emitted while the pending Linear-2 tile could already go (no idle Linear-2 work)."""
+    for (G, P, P1, P2, D) in CASES:
+        for g, seq in enumerate(all_orders(G, P, P1, P2, D)):
+            l1 = [k for ph, k in seq if ph == 0]
+            l2 = [k for ph, k in seq if ph == 1]
+            n1 = n2 = 0                      # tiles of each stream emitted so far
+            for ph, k in seq:
+                pending_row1 = l1[n1] // P1 if n1 < len(l1) else math.inf
+                may_go = n2 < len(l2) and l2[n2] // P2 + D <= pending_row1
                 if ph == 1:
-                    # the instance's next Linear-1 tile at this point
-                    n_l1_before = sum(1 for ph2, _ in seq[:i] if ph2 == 0)
-                    nxt = emitted_l1[n_l1_before] if n_l1_before < len(emitted_l1) else None
-                    p1 = nxt // P1 if nxt is not None else math.inf
-                    # if the cursor ran off the end without emitting, p1 is infinite as well
-                    assert k // P2 + D <= p1
-        assert seen[0] == set(range(P * P1)) and seen[1] == set(range(P * P2))
+                    assert may_go, (G, P, P1, P2, D, g, k)
+                    n2 += 1
+                else:
+                    assert not may_go, (G, P, P1, P2, D, g, k)
+                    n1 += 1
 
 
 def test_hand_worked_small_case():
@@ -42,6 +55,16 @@ def test_hand_worked_small_case():
     # (row 1) has to wait until the Linear-1 cursor has run off the end.
     assert so.algorithm1_order(1, 2, 2, 2, 2, 1) == [(0, 1), (1, 1), (0, 3), (1, 3)]
     assert so.algorithm1_order(0, 2, 2, 2, 2, 1) == [(0, 0), (1, 0), (0, 2), (1, 2)]
+
+
+def test_zero_lead_one_instance_alternates_rows_linear2_first():
+    # D = 0: a Linear-2 tile may go as soon as the pending Linear-1 tile is in its own row, so row p's Linear-2
+    # tiles precede row p's Linear-1 tiles (an order no kernel may run: the data does not exist yet)
+    P, P1, P2 = 3, 2, 2
+    want = []
+    for p in range(P):
+        want += [(1, p * P2 + c) for c in range(P2)] + [(0, p * P1 + c) for c in range(P1)]
+    assert so.algorithm1_order(0, 1, P, P1, P2, 0) == want
 
 
 def test_large_lead_is_expert_wave_and_mix_is_preserved():

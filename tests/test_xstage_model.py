@@ -214,3 +214,5 @@ def test_store_probe_runs_and_reports_consistent_spans():
         xstage.xstage_store_probe(sms + 1, 8192, 0, 1, buf)
     with pytest.raises(RuntimeError):
         xstage.xstage_store_probe(sms, 24, 0, 1, buf)
+    with pytest.raises(RuntimeError):      # a gap in the wrong unit: 1e9 clocks x 100 periods is refused, not spun through
+        xstage.xstage_store_probe(sms, 8192, 10**9, 100, buf)
