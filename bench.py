@@ -30,11 +30,21 @@ from paper_2607_23264_b200 import inputs as gen  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one expert_gemm_kernel<true> (Linear-1) launch on the
-# C2 workload: the ncu capture of the two-expert case P1 (511.7 MB read + 109.9 MB written, see
-# profiles/expert_gemm_P1_ncu_full.md) scaled by 4, since DRAM traffic is per expert and C2 has four times
-# P1's experts at the same rows per expert.  C3: one-pass DRAM counters on the full layer (same file).
-LINEAR1_DRAM_TRAFFIC_BYTES = {"C2": 4 * (511_678_208 + 109_886_720), "C3": 11_263_676_672 + 136_142_592}
+def dram_traffic_per_expert(kernel: str):
+    """ncu DRAM bytes (read + write) of one Linear-1 launch, per non-empty expert, for `kernel`, from the committed
+    summary of the capture (a table row per kernel: name | case | experts | dram read bytes | dram write bytes).
+    None when the summary or the row is missing."""
+    path = os.path.join(ROOT, "profiles", "linear1_dram_traffic.md")
+    try:
+        with open(path) as fh:
+            for line in fh:
+                cells = [c.strip() for c in line.strip().strip("|").split("|")]
+                if len(cells) >= 5 and cells[0].strip("`") == kernel:
+                    experts, rd, wr = int(cells[2]), int(cells[3].replace(",", "")), int(cells[4].replace(",", ""))
+                    return (rd + wr) / experts
+    except (OSError, ValueError):
+        pass
+    return None
 
 
 def load_peaks():
@@ -133,7 +143,8 @@ def run_reference(args, cfg, rank, world):
     total = sum(times)
     value = n_tok * args.steps / total
     cores = oracle_threads()
-    sample = f"{n_tok} seeded-random tokens of {cfg.name} per step (row-sampled oracle, exact per row)"
+    sample = (f"{n_tok} seeded-random tokens of {cfg.name} per step (row-sampled fp64 oracle, exact per row; the oracle's "
+              "widening of each touched expert's bf16 matrices to fp64 is part of the timed call)")
     line = {
         "impl": "reference", "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
@@ -163,8 +174,11 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="run --config's layer at this batch size instead of its own T")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=128, help="tokens per step of the reference (oracle) arm")
-    ap.add_argument("--cpu-baseline-tokens", type=int, default=384)
+    ap.add_argument("--cpu-baseline-tokens", type=int, default=128,
+                    help="tokens of the cpu_baseline leg (the same sample size as a step of the reference arm)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--heat-seconds", type=float, default=2.0,
+                    help="back-to-back untimed steps before the timed region, until the power cap has settled the clocks")
     ap.add_argument("--burst", type=int, default=1)
     ap.add_argument("--mode", type=int, default=0)
     ap.add_argument("--ik", type=int, default=1)
@@ -189,6 +203,19 @@ def main():
     ap.add_argument("--profile", action="store_true",
                     help="profiler run: warm-up and timed steps only (no per-kernel pass, end-to-end or CPU legs)")
     args = ap.parse_args()
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain script: become the launcher of args.gpus ranks (one per GPU) and pass their output on
+        import socket
+        from paper_2607_23264_b200 import replicas
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        cmd, extra = replicas.launcher_command(args.gpus, os.path.abspath(__file__), sys.argv[1:], port, sys.executable)
+        env = dict(os.environ)
+        for key, val in extra.items():
+            env.setdefault(key, val)
+        sys.exit(subprocess.call(cmd, env=env))
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -292,41 +319,71 @@ def main():
                                  debug_flags=dbg)
     step = lambda: ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tuning)
 
-    # ---- device-resident throughput, with per-kernel events, clocks sampled during the timed region
-    ctx.moe_set_kernel_timing(True)
+    # ---- device-resident throughput.  Four regions, all on the launch stream:
+    #   burst : args.steps steps back to back right after the warm-up (the GPU still in its boost state);
+    #   heat  : at least two seconds of back-to-back steps, untimed, until the 1 kW power cap has settled the clocks;
+    #   steady: args.steps steps back to back, bracketed by a barrier and a synchronize on both sides, one event
+    #           between consecutive steps: ms_per_step = the whole region / steps (this is the line's value), and
+    #           the median of the per-step times is reported beside it;
+    #   kernel passes after the burst and after the steady region: the same steps with the library's per-kernel
+    #           events read after every step.
     for _ in range(args.warmup):
         step()
     barrier()
     sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    per_step_kernel = []
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
-    total_ms = replicas.max_over_ranks(e0.elapsed_time(e1), world, dev)
-    clocks = sampler.stop() if rank == 0 else None
-    launches = ctx.moe_last_launch_count() * args.steps
 
+    def region(steps):
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        marks[0].record(stream)
+        for i in range(steps):
+            step()
+            marks[i + 1].record(stream)
+        barrier()
+        total = replicas.max_over_ranks(marks[0].elapsed_time(marks[-1]), world, dev)
+        return total, [marks[i].elapsed_time(marks[i + 1]) for i in range(steps)]
+
+    def kernel_pass(steps):
+        ctx.moe_set_kernel_timing(True)
+        per = []
+        for _ in range(steps):
+            step()
+            per.append(ctx.moe_get_kernel_times())
+        ctx.moe_set_kernel_timing(False)
+        return [float(np.mean([s[i] for s in per])) for i in range(len(binding.KERNEL_NAMES))]
+
+    burst_total_ms, _ = region(args.steps)
+    launches = ctx.moe_last_launch_count() * args.steps
     if args.profile:
         if rank == 0:
-            print(json.dumps({"profile_run": True, "ms_per_step": total_ms / args.steps,
-                              "config": workload_config(cfg, world), "clocks": clocks}), flush=True)
+            print(json.dumps({"profile_run": True, "ms_per_step": burst_total_ms / args.steps,
+                              "config": workload_config(cfg, world)}), flush=True)
         if world > 1:
             dist.destroy_process_group()
         return
-
-    # per-kernel average launch duration: the same steps again, reading the event pairs after each step
-    for _ in range(args.steps):
-        step()
-        per_step_kernel.append(ctx.moe_get_kernel_times())
+    burst_kernel_ms = kernel_pass(args.steps)
+    if rank == 0:
+        sampler.start()
+    heat_t0, heat_steps = time.time(), 0
+    while time.time() - heat_t0 < args.heat_seconds:
+        for _ in range(10):
+            step()
+        heat_steps += 10
+        torch.cuda.synchronize()
+    total_ms, step_times = region(args.steps)
+    kernel_ms = kernel_pass(args.steps)
+    # SM clock of the steady region from the kernel itself: the Linear-1 producer's clock64 span over the kernel's
+    # CUDA-event time, in one traced step taken while the GPU is still in that state (read, never set)
+    ctx.moe_set_kernel_timing(True)
+    ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws,
+                          tuning=binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule,
+                                                     dep_lead_D=args.lead, debug_flags=dbg | 1))
+    span = float(ctx.moe_get_ffn_trace()[0, :, 0].max())
+    ms4 = ctx.moe_get_kernel_times()[4]
     ctx.moe_set_kernel_timing(False)
-    kernel_ms = [float(np.mean([s[i] for s in per_step_kernel])) for i in range(len(binding.KERNEL_NAMES))]
+    clocks = sampler.stop() if rank == 0 else None
+    if clocks is not None and ms4 > 0:
+        clocks["sm_mhz_kernel"] = span / (ms4 * 1e-3) / 1e6
 
     # per-step statistics with one event pair per step (the paper reports medians of 20 trials, Sec. 5.1); small
     # layers whose working set fits L2 are also timed cold, a 512 MB memset between steps evicting L2
@@ -344,22 +401,12 @@ def main():
             times.append(a.elapsed_time(b))
         return {"median_ms": statistics.median(times), "min_ms": min(times), "max_ms": max(times)}
 
-    step_stats = {"warm": per_step(False)}
+    step_stats = {"steady": {"median_ms": statistics.median(step_times), "min_ms": min(step_times),
+                             "max_ms": max(step_times), "heat_steps_before": heat_steps},
+                  "synchronised_each_step": per_step(False)}
     weights_bytes = 6 * cfg.E * cfg.H * cfg.F
     if weights_bytes < (256 << 20) or cfg.T <= 256:
         step_stats["cold_l2_flushed"] = per_step(True)
-
-    # SM clock while the first grouped-GEMM kernel runs, from the kernel's own clock64 span against its CUDA-event
-    # time (nvidia-smi, sampled every 100 ms, often misses a timed region this short)
-    ctx.moe_set_kernel_timing(True)
-    ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws,
-                          tuning=binding.make_tuning(args.burst, args.mode, args.ik, schedule=args.schedule,
-                                                     dep_lead_D=args.lead, debug_flags=dbg | 1))
-    span = float(ctx.moe_get_ffn_trace()[0, :, 0].max())
-    ms4 = ctx.moe_get_kernel_times()[4]
-    ctx.moe_set_kernel_timing(False)
-    if clocks is not None and ms4 > 0:
-        clocks["sm_mhz_kernel"] = span / (ms4 * 1e-3) / 1e6
 
     # the same step replayed from a CUDA graph (launch overhead off the critical path; matters for small layers)
     try:
@@ -452,7 +499,8 @@ def main():
     move_bytes = 2 * cfg.H * (cfg.T + R)
     disp_gbs = move_bytes / (kernel_ms[3] * 1e-3) / 1e9
     comb_gbs = (move_bytes + 8 * R) / (kernel_ms[6] * 1e-3) / 1e9
-    peak_tf = float(peaks["bf16_tflops"])
+    peak_tf_burst = float(peaks["bf16_tflops"])
+    peak_tf = float(peaks.get("bf16_tflops_sustained", peak_tf_burst))   # the steady region is a long step loop
     peak_hbm = float(peaks["hbm_gbs"])
     lay = ctx.workspace_layout()
     counts = ws[lay["counts"]:lay["counts"] + 4 * cfg.E].view(torch.int32).cpu().numpy()
@@ -465,42 +513,58 @@ def main():
     l1_gbs = l1_bytes / (kernel_ms[4] * 1e-3) / 1e9
     l2_gbs = 0.0 if one_launch else l2_bytes / (kernel_ms[5] * 1e-3) / 1e9
     pair_kernel = not one_launch and (args.pairs == "on" or (args.pairs == "auto" and cfg.R // cfg.E >= 1024))
-    gemm_name = ("expert_ffn_kernel (Linear-1 + SiLU*mul + Linear-2, one launch)" if one_launch
-                 else ("expert_ffn_pair_kernel" if pair_kernel else "expert_ffn_kernel") + ", Linear-1 + SiLU*mul launch")
+    kernel_symbol = "expert_ffn_pair_kernel<false>" if pair_kernel else "expert_ffn_kernel<false>"
+    gemm_name = (kernel_symbol + " (Linear-1 + SiLU*mul + Linear-2, one launch)" if one_launch
+                 else kernel_symbol + ", Linear-1 + SiLU*mul launch")
+    per_expert = None if one_launch else dram_traffic_per_expert(kernel_symbol)
+    traffic = None if per_expert is None else per_expert * nonempty
     # the roofline that binds Linear-1: tensor time at the measured GEMM peak vs HBM time at the measured copy rate
-    t_tensor = l1_flops / (peak_tf * 1e12)
+    t_tensor = l1_flops / (peak_tf_burst * 1e12)
     t_hbm = l1_bytes / (peak_hbm * 1e9)
+    burst_ms4 = burst_kernel_ms[4]
     if t_tensor >= t_hbm:
+        burst_tf = l1_flops / (burst_ms4 * 1e-3) / 1e12
         roofline = {
             "kernel": gemm_name, "bound": "tensor", "achieved": l1_tf,
-            "peak": peak_tf, "unit": "TFLOP/s", "frac": l1_tf / peak_tf,
-            "traffic": None if one_launch else LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name),
-            "peak_source": f"{peak_kind} bf16_tflops (burst)",
-            "frac_of_sustained": l1_tf / float(peaks.get("bf16_tflops_sustained", peak_tf)),
+            "peak": peak_tf, "unit": "TFLOP/s", "frac": l1_tf / peak_tf, "traffic": traffic,
+            "peak_source": f"{peak_kind} bf16_tflops_sustained (cuBLAS in a seconds-long loop): the kernel is timed inside "
+                           "a pre-heated loop of steps",
             "flops_per_launch": l1_flops, "ms_per_launch": kernel_ms[4],
+            "burst": {"achieved": burst_tf, "peak": peak_tf_burst, "frac": burst_tf / peak_tf_burst,
+                      "ms_per_launch": burst_ms4, "peak_source": f"{peak_kind} bf16_tflops (burst)"},
         }
     else:
         roofline = {
             "kernel": gemm_name, "bound": "hbm", "achieved": l1_gbs,
-            "peak": peak_hbm, "unit": "GB/s", "frac": l1_gbs / peak_hbm,
-            "traffic": None if one_launch else LINEAR1_DRAM_TRAFFIC_BYTES.get(cfg.name),
+            "peak": peak_hbm, "unit": "GB/s", "frac": l1_gbs / peak_hbm, "traffic": traffic,
             "peak_source": f"{peak_kind} hbm_gbs (copy)",
             "bytes_per_launch": l1_bytes, "ms_per_launch": kernel_ms[4], "nonempty_experts": nonempty,
             "tensor_tflops": l1_tf,
+            "burst": {"achieved": l1_bytes / (burst_ms4 * 1e-3) / 1e9, "peak": peak_hbm,
+                      "frac": l1_bytes / (burst_ms4 * 1e-3) / 1e9 / peak_hbm, "ms_per_launch": burst_ms4},
         }
+    if traffic is not None:
+        roofline["traffic_source"] = ("profiles/linear1_dram_traffic.md: ncu dram read + write bytes per non-empty expert "
+                                      f"of {kernel_symbol} on its profiler-sized case x {nonempty} experts")
     # The cuBLAS peak was measured at its own SM clock under the power cap; this kernel ran at sm_mhz_kernel (its
     # clock64 span over its CUDA-event time).  frac x (peak's clock / this clock) compares flops per clock.
     peak_mhz = float((peaks.get("clocks_under_load") or {}).get("sm_mhz_median") or 0.0)
     if roofline["bound"] == "tensor" and peak_mhz > 0 and clocks and clocks.get("sm_mhz_kernel"):
         roofline["peak_sm_mhz"] = peak_mhz
         roofline["frac_at_equal_clock"] = roofline["frac"] * peak_mhz / clocks["sm_mhz_kernel"]
+    burst_ms_per_step = burst_total_ms / args.steps
     line = {
         "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": workload_config(cfg, world),
-        "tflops": tflops, "frac_bf16_peak": tflops / world / peak_tf,
+        "tflops": tflops, "frac_bf16_peak": tflops / world / peak_tf, "frac_bf16_peak_of": "bf16_tflops_sustained",
+        "burst_ms_per_step": burst_ms_per_step, "burst_value": cfg.T * world / (burst_ms_per_step * 1e-3),
+        "burst_frac_bf16_peak": cfg.flops / (burst_ms_per_step * 1e-3) / 1e12 / peak_tf_burst,
+        "timed_region": f"{args.steps} back-to-back steps after {heat_steps} untimed pre-heating steps "
+                        f"({args.heat_seconds:.1f} s); burst_* = {args.steps} steps right after the warm-up",
         "kernels_ms": dict(zip(binding.KERNEL_NAMES, kernel_ms)),
+        "burst_kernels_ms": dict(zip(binding.KERNEL_NAMES, burst_kernel_ms)),
         "linear2_tflops": l2_tf, "linear1_gbs": l1_gbs, "linear2_gbs": l2_gbs, "dispatch_gbs": disp_gbs, "combine_gbs": comb_gbs,
         "dispatch_frac_hbm": disp_gbs / float(peaks["hbm_gbs"]), "combine_frac_hbm": comb_gbs / float(peaks["hbm_gbs"]),
         "roofline": roofline,
@@ -519,7 +583,8 @@ def main():
         line["cpu_baseline"] = {
             "value": rate, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
             "sample": f"{min(args.cpu_baseline_tokens, cfg.T)} seeded-random tokens of {cfg.name} (row-sampled fp64 "
-                      f"oracle, {dt:.1f} s)"}
+                      f"oracle, {dt:.1f} s; the oracle's widening of each touched expert's bf16 matrices to fp64 is part "
+                      "of the timed call)"}
     elif want_cpu:
         # many experts: sample tokens until they touch about 64 experts, regenerate those experts' weights on the
         # host first (input generation, not timed), then time the oracle on the sample
@@ -811,9 +876,12 @@ def run_sweep(args, cfg, ctx, binding, bufs, timed, rank):
     The GPU is first brought to its steady power-capped state (about 1.5 s of steps); every point is then
     timed in two passes (forward and reverse order) so that clock drift shows up as spread, not as a trend.
     Per point: median/min ms per step, TFLOP/s, algorithmic HBM GB/s, per-kernel times, and from one traced step
-    the Linear-2 per-tile epilogue store span, pacing hold and MMA wait for a free accumulator (SM clocks)."""
+    the share of each GEMM's span its tensor pipe was busy (MMA instructions issued x the 128 clocks the pipe needs
+    for one, over the CTA's span), the Linear-2 per-tile epilogue store span, pacing hold and MMA wait for a free
+    accumulator (SM clocks), and how many CTAs held stores at all."""
     import torch
     x, d_logits, w_gate, w_up, w_down, out, ws = bufs
+    dbg = {"auto": 0, "on": 8, "off": 16}[args.pairs]
     points = [(b, 0, 1) for b in (1, 2, 4, 8, 16)] + [(b, 1, ik) for b in (1, 2, 4, 8, 16) for ik in (1, 2, 4)]
     run = lambda tn: ctx.moe_fused_forward(x, d_logits, w_gate, w_up, w_down, out, ws, tuning=tn)
     t0 = time.time()
@@ -826,9 +894,10 @@ def run_sweep(args, cfg, ctx, binding, bufs, timed, rank):
     extra = {}
     R = cfg.R
     step_bytes = (6 * cfg.E * cfg.H * cfg.F + 2 * (2 * cfg.T * cfg.H + 4 * R * cfg.H + 2 * R * cfg.F))
+    k_blocks = (cfg.H // 64, cfg.F // 64)
     for order in (points, points[::-1]):
         for pt in order:
-            tn = binding.make_tuning(*pt)
+            tn = binding.make_tuning(*pt, debug_flags=dbg)
             ms = timed(lambda: run(tn), args.steps, max(1, args.warmup)) / args.steps
             samples[pt].append(ms)
             if pt not in extra:
@@ -839,22 +908,33 @@ def run_sweep(args, cfg, ctx, binding, bufs, timed, rank):
                 bits = out.view(torch.int16).clone()
                 if base is None:
                     base = bits
-                run(binding.make_tuning(*pt, debug_flags=1))
+                run(binding.make_tuning(*pt, debug_flags=dbg | 1))
                 tr = ctx.moe_get_ffn_trace().astype(np.float64)
+                pipe = []
+                for gi in (0, 1):
+                    issuing = tr[gi][:, 6] > 0           # CTAs whose MMA warp issued (in a CTA pair: the leader)
+                    span = np.maximum(tr[gi][issuing, 0], 1.0)
+                    pipe.append(float((tr[gi][issuing, 6] * k_blocks[gi] * 4 * 128 / span).mean()) if issuing.any() else 0.0)
                 l2 = tr[1].mean(axis=0)
-                tiles = max(l2[6], 1.0)
+                tiles = max(tr[1][:, 6].sum() / max((tr[1][:, 5] > 0).sum(), 1), 1.0)   # tiles per draining CTA
                 extra[pt] = {"linear1_ms": km[4], "linear2_ms": km[5], "identical_bits": bool(torch.equal(bits, base)),
+                             "tensor_pipe_linear1": pipe[0], "tensor_pipe_linear2": pipe[1],
+                             "ctas_holding_stores": [int((tr[0][:, 7] > 0).sum()), int((tr[1][:, 7] > 0).sum())],
+                             "l1_pacing_hold_clk_per_cta": float(tr[0][:, 7].mean()),
                              "l2_store_span_clk_per_tile": l2[5] / tiles, "l2_pacing_hold_clk_per_tile": l2[7] / tiles,
                              "l2_mma_wait_accumulator_clk_per_tile": l2[3] / tiles,
                              "l2_mma_wait_operands_frac": l2[2] / max(l2[0], 1.0)}
     rows = []
     for pt in points:
         ms = statistics.median(samples[pt])
+        e = extra[pt]
+        pipe_step = (e["tensor_pipe_linear1"] * e["linear1_ms"] + e["tensor_pipe_linear2"] * e["linear2_ms"]) / ms
         rows.append({"burst": pt[0], "mode": pt[1], "k": pt[2], "ms_per_step": ms, "ms_min": min(samples[pt]),
                      "ms_max": max(samples[pt]), "tflops": cfg.flops / (ms * 1e-3) / 1e12,
-                     "hbm_gbs_algorithmic": step_bytes / (ms * 1e-3) / 1e9, **extra[pt]})
+                     "hbm_gbs_algorithmic": step_bytes / (ms * 1e-3) / 1e9, "tensor_pipe_step": pipe_step, **e})
     if rank == 0:
-        print(json.dumps({"sweep": rows, "config": workload_config(cfg, 1), "steps_per_sample": args.steps}), flush=True)
+        print(json.dumps({"sweep": rows, "config": workload_config(cfg, 1), "steps_per_sample": args.steps,
+                          "pairs": args.pairs}), flush=True)
 
 
 if __name__ == "__main__":

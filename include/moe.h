@@ -53,12 +53,16 @@ typedef struct {
  * A "store tile" is 128 rows x 32 output columns of bf16 (8 KiB), the unit one pass of the four epilogue
  * warps drains from tensor memory.  A burst is `store_burst_tiles` store tiles issued back to back by a
  * CTA.  interleave_mode 0 ("after-mainloop"): bursts follow one another with no enforced gap.
- * interleave_mode 1 ("every-k-iterations"): after each burst the epilogue holds further stores until the
- * MMA warp has issued `interleave_k` more 64-deep K-blocks of the next tile's mainloop (or has nothing
- * left to issue).  Pacing never changes values: outputs are bitwise identical for every setting.
+ * interleave_mode 1 ("every-k-iterations"): after each burst the epilogue holds its next store until the
+ * MMA warp has issued `interleave_k` more 64-deep K-blocks (of the following tiles' mainloops) than when
+ * the burst ended, or has nothing left to issue.  In the CTA-pair kernel both CTAs of a pair pace on the
+ * leader's MMA warp, so every CTA that stores is a paced producer in the sense of Eq. 1.  Tiles computed
+ * with swapped operands (a few rows) are not paced.  Pacing never changes values: outputs are bitwise
+ * identical for every setting.
  */
 typedef struct {
-  int32_t store_burst_tiles;       /* 1, 2, 4, 8 or 16 (values above the tiles in one output tile act as that count) */
+  int32_t store_burst_tiles;       /* 1, 2, 4, 8 or 16; a CTA counts its store tiles across output tiles, so a burst
+                                      may span accumulators (an output tile is 4 store tiles in Linear-1, 8 in Linear-2) */
   int32_t interleave_mode;         /* 0 or 1 */
   int32_t interleave_k;            /* 1, 2 or 4; used when interleave_mode == 1 */
   int32_t schedule;                /* 0 = Expert-Wave order (Sec. 4.3): all Linear-1 tiles, then all Linear-2 tiles;

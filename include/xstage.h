@@ -73,6 +73,30 @@ double xstage_mma_stall(double t_remote_store_span, double t_cover_mma);
 int64_t xstage_fa_recovery_length(int64_t b_n, double recovery_gap, double sigma);
 
 /*
+ * Calibration of M_X from microbenchmark rows (Sec. 3.3 "independent calibration", Sec. 3.5: the three parameters
+ * come from the large-gap plateau, the zero-gap runs and the isolated-burst knee).
+ *   Periodic rows (one burst volume at several gaps, gap 0 among them): volume, gap, measured issue span t_iss and
+ *   period t_period.  Isolated rows (one burst from a recovered state), ascending volume: volume, t_iss.
+ *   t_iss0  = median t_iss over the rows whose gap is among the largest third of the distinct gaps (the plateau);
+ *   rate    = median of volume / t_period over the rows with gap 0 (drain-limited steady state); 0 if there is none;
+ *   the recovered issue floor of an isolated burst grows with its volume (the issue loop itself takes time), so it
+ *   is a least-squares line a + b V through the smallest third of the isolated volumes (at least three rows);
+ *   the knee is the last row before the first later row whose t_iss exceeds (1 + knee_tolerance)(a + b V);
+ *   capacity = [V_knee - rate t_iss(V_knee)]_+   (Eq. 6 from a recovered state).
+ * has_knee is 0 (capacity and knee_volume 0) when no row leaves the floor line, when there are fewer than three
+ * isolated rows or when there is no zero-gap row.  Returns 0, or -1 on a bad argument (null pointer, no periodic row,
+ * negative tolerance, a non-positive period in a zero-gap row).
+ */
+typedef struct {
+  double t_iss0, rate, capacity, knee_volume, floor_intercept, floor_per_byte;
+  int32_t has_knee;
+} xstage_calibration;
+
+int xstage_calibrate(int64_t n_periodic, const double* p_volume, const double* p_gap, const double* p_t_iss,
+                     const double* p_t_period, int64_t n_isolated, const double* i_volume, const double* i_t_iss,
+                     double knee_tolerance, xstage_calibration* out);
+
+/*
  * Store microbenchmark on this GPU's own memory: the periodic-burst and isolated-burst patterns of Sec. 3.1, run
  * the way the paper runs its local-memory control (Sec. 3.2), i.e. the identical store kernel with only the
  * destination changed from a peer's memory to this GPU's.  `producers` CTAs of 128 threads, one per SM (producers <= SM count), start together; each

@@ -78,3 +78,36 @@ def mma_stall(t_rs: float, t_cover: float) -> float:
 def fa_recovery_length(b_n: int, g_star: float, sigma: float) -> int:
     """App. C.2: b_n ceil(G*/sigma)."""
     return b_n * math.ceil(g_star / sigma)
+
+
+def calibrate(periodic, isolated, knee_tolerance: float = 0.10):
+    """The three parameters from microbenchmark rows (Sec. 3.3, Sec. 3.5): T0 from the large-gap plateau, R from the
+    zero-gap runs, Q from the isolated-burst knee.
+
+    periodic: (volume, gap, t_iss, t_period) tuples of one burst volume; isolated: (volume, t_iss) tuples, ascending.
+    Plateau = rows whose gap is among the largest third of the distinct gaps.  The recovered floor of an isolated
+    burst is the least-squares line through the smallest third (at least three) of the isolated rows; the knee is the
+    row before the first later row that rises more than knee_tolerance above that line; Q = [V_knee - R t_iss]_+.
+    Returns (t0, rate or None, capacity or None, knee_volume or None)."""
+    import statistics
+
+    import numpy as np
+    gaps = sorted({g for _, g, _, _ in periodic})
+    top = gaps[len(gaps) - max(1, len(gaps) // 3):]
+    t0 = statistics.median(ti for _, g, ti, _ in periodic if g in top)
+    zero_gap = [v / tp for v, g, _, tp in periodic if g == 0]
+    rate = statistics.median(zero_gap) if zero_gap else None
+    if rate is None or len(isolated) < 3:
+        return t0, rate, None, None
+    n = max(3, len(isolated) // 3)
+    vol = np.array([v for v, _ in isolated], dtype=np.float64)
+    iss = np.array([t for _, t in isolated], dtype=np.float64)
+    if np.ptp(vol[:n]) > 0:
+        slope, intercept = np.polyfit(vol[:n], iss[:n], 1)          # library least squares
+    else:
+        slope, intercept = 0.0, float(iss[:n].mean())
+    above = np.flatnonzero(iss[n:] > (1.0 + knee_tolerance) * (intercept + slope * vol[n:]))
+    if above.size == 0:
+        return t0, rate, None, None
+    knee = n + int(above[0]) - 1
+    return t0, rate, pos(float(vol[knee]) - rate * float(iss[knee])), float(vol[knee])

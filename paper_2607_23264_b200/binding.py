@@ -275,7 +275,7 @@ class Context:
         return moe_shape(self.T, self.H, self.F, self.E, self.k, self.ep_size, self.ep_rank)
 
     def router_weight_bytes(self) -> int:
-        """Bytes of the prepared router weights (three bf16 terms of W_r, expert rows padded)."""
+        """Bytes of the prepared router weights (two bf16 terms of W_r, expert rows padded)."""
         return int(self._lib.moe_router_weight_bytes(C.byref(self._shape())))
 
     def router_scratch_bytes(self) -> int:

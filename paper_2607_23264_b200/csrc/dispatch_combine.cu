@@ -45,6 +45,15 @@ dispatch_rows(const uint4* __restrict__ x, const int32_t* __restrict__ inv_perm,
   }
 }
 
+// 16-byte load of data read once: through the read-only path, not kept in L1
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
 __device__ __forceinline__ void fma8(float (&acc)[8], float w, const uint4& v) {
   const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
 #pragma unroll
@@ -55,9 +64,12 @@ __device__ __forceinline__ void fma8(float (&acc)[8], float w, const uint4& v) {
   }
 }
 
-constexpr int kCombVec = 2;                      // vectors per lane per item
-constexpr int kCombPass = 32 * kCombVec;         // vectors per item (1 KiB of bf16 per row)
-
+// One item = one token x (32 * V) 16-byte vectors of its row.  The k expert rows are fetched in batches of kCombBatch
+// rows: all loads of a batch (kCombBatch * V per lane) are issued before the first of its FMAs, which then run in
+// ascending j, so the memory system sees the whole batch at once while the summation order stays the contract's.
+// What bounds the kernel is the bytes an SM keeps in flight (resident warps x loads per lane x 16 bytes), so V and
+// the batch are chosen per k: few rows per token -> more vectors per lane.
+template <int V, int kCombBatch>
 __global__ void __launch_bounds__(kThreads)
 combine_rows(const uint4* __restrict__ y_perm, const int32_t* __restrict__ inv_perm,
              const float* __restrict__ topk_w, uint4* __restrict__ out, int T, int k, int vec_per_row,
@@ -68,31 +80,44 @@ combine_rows(const uint4* __restrict__ y_perm, const int32_t* __restrict__ inv_p
   const long long items = static_cast<long long>(T) * blocks_per_row;
   for (long long item = gwarp; item < items; item += warps_total) {
     const int t = static_cast<int>(item / blocks_per_row);
-    const int v0 = static_cast<int>(item % blocks_per_row) * kCombPass;
+    const int v0 = static_cast<int>(item % blocks_per_row) * (32 * V);
     int my_row = 0;
     float my_w = 0.f;
     if (lane < k) {
-      my_row = inv_perm[static_cast<size_t>(t) * k + lane];
-      my_w = topk_w[static_cast<size_t>(t) * k + lane];
+      my_row = __ldg(inv_perm + static_cast<size_t>(t) * k + lane);
+      my_w = __ldg(topk_w + static_cast<size_t>(t) * k + lane);
     }
-    float acc[kCombVec][8];
+    float acc[V][8];
 #pragma unroll
-    for (int u = 0; u < kCombVec; ++u)
+    for (int u = 0; u < V; ++u)
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[u][i] = 0.f;
-#pragma unroll 4
-    for (int j = 0; j < k; ++j) {                 // ascending j: the summation order is part of the contract
-      const int row = __shfl_sync(0xFFFFFFFFu, my_row, j);
-      const float w = __shfl_sync(0xFFFFFFFFu, my_w, j);
-      const uint4* src = y_perm + static_cast<size_t>(row) * vec_per_row;
+    for (int j0 = 0; j0 < k; j0 += kCombBatch) {
+      uint4 buf[kCombBatch][V];
+      float w[kCombBatch];
 #pragma unroll
-      for (int u = 0; u < kCombVec; ++u) {
-        const int v = v0 + u * 32 + lane;
-        if (v < vec_per_row) fma8(acc[u], w, __ldg(src + v));
+      for (int b = 0; b < kCombBatch; ++b) {
+        const int j = j0 + b;                       // j >= k reads lane j's zeros: row 0, weight 0, skipped below
+        const int row = __shfl_sync(0xFFFFFFFFu, my_row, j & 31);
+        w[b] = __shfl_sync(0xFFFFFFFFu, my_w, j & 31);
+        const uint4* src = y_perm + static_cast<size_t>(row) * vec_per_row;
+#pragma unroll
+        for (int u = 0; u < V; ++u) {
+          const int v = v0 + u * 32 + lane;
+          if (j < k && v < vec_per_row) buf[b][u] = ld_stream(src + v);
+        }
+      }
+#pragma unroll
+      for (int b = 0; b < kCombBatch; ++b) {       // ascending j: the summation order is part of the contract
+        if (j0 + b < k) {
+#pragma unroll
+          for (int u = 0; u < V; ++u)
+            if (v0 + u * 32 + lane < vec_per_row) fma8(acc[u], w[b], buf[b][u]);
+        }
       }
     }
 #pragma unroll
-    for (int u = 0; u < kCombVec; ++u) {
+    for (int u = 0; u < V; ++u) {
       const int v = v0 + u * 32 + lane;
       if (v < vec_per_row) {
         uint4 o;
@@ -128,15 +153,28 @@ cudaError_t launch_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_
                            void* out, cudaStream_t stream) {
   const moe_shape& s = ctx->shape;
   const int vec_per_row = s.H / 8;
-  const int blocks_per_row = (vec_per_row + kCombPass - 1) / kCombPass;
+  // loads a lane keeps in flight = batch x V: about 8, split by k (the batch never exceeds the rows of a token)
+  int batch = s.k >= 8 ? 8 : s.k >= 4 ? 4 : s.k >= 2 ? 2 : 1;
+  int V = 8 / batch > 4 ? 4 : 8 / batch;
+  while (V > 1 && vec_per_row < 32 * V) V >>= 1;
+  const int kv = moe_knob_value(ctx, "combine_vec", 0), kb = moe_knob_value(ctx, "combine_batch", 0);
+  if (kv == 1 || kv == 2 || kv == 4) V = kv;
+  if (kb == 1 || kb == 2 || kb == 4 || kb == 8) batch = kb;
+  const int blocks_per_row = (vec_per_row + 32 * V - 1) / (32 * V);
   const long long items = static_cast<long long>(s.T) * blocks_per_row;
   const int warps_per_block = kThreads / 32;
   long long blocks = (items + warps_per_block - 1) / warps_per_block;
-  const long long cap = static_cast<long long>(ctx->num_sms) * 8;
-  if (blocks > cap) blocks = cap;
-  combine_rows<<<static_cast<int>(blocks), kThreads, 0, stream>>>(
-      static_cast<const uint4*>(y_perm), inv_perm, topk_w, static_cast<uint4*>(out), s.T, s.k, vec_per_row,
-      blocks_per_row);
+  const long long cap = static_cast<long long>(ctx->num_sms) * moe_knob_value(ctx, "combine_ctas_per_sm", 6);
+  if (blocks > cap && cap > 0) blocks = cap;
+  using kernel_t = void (*)(const uint4*, const int32_t*, const float*, uint4*, int, int, int, int);
+  static const kernel_t table[3][4] = {
+      {combine_rows<1, 1>, combine_rows<1, 2>, combine_rows<1, 4>, combine_rows<1, 8>},
+      {combine_rows<2, 1>, combine_rows<2, 2>, combine_rows<2, 4>, combine_rows<2, 8>},
+      {combine_rows<4, 1>, combine_rows<4, 2>, combine_rows<4, 4>, combine_rows<4, 8>}};
+  const kernel_t kernel = table[V == 4 ? 2 : V == 2 ? 1 : 0][batch == 8 ? 3 : batch == 4 ? 2 : batch == 2 ? 1 : 0];
+  kernel<<<static_cast<int>(blocks), kThreads, 0, stream>>>(static_cast<const uint4*>(y_perm), inv_perm, topk_w,
+                                                            static_cast<uint4*>(out), s.T, s.k, vec_per_row,
+                                                            blocks_per_row);
   moe_mark(ctx, 7, stream);
   ctx->last_launches += 1;
   return cudaGetLastError();

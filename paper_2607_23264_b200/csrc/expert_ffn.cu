@@ -106,6 +106,8 @@ struct FfnParams {
   int lead_D;               // Algorithm 1: minimum row lead of Linear-1 over Linear-2 (>= 1)
   int fp8;                  // operands are E4M3 bytes (128 per swizzle row) instead of bf16 (64 per row)
   int k_elems;              // K elements per pipeline stage: 64 (bf16) or 128 (E4M3)
+  int small_a;              // swapped-operand tiles load only their own (padded) rows of A, in 16-row boxes
+  int swap_prefetch;        // swapped-operand tiles ask L2 for their weight boxes this many K blocks ahead (0 = off)
   int withhold_ready;       // host-requested failure drill: Linear-1 never publishes its rows (one-launch runs)
   long long wait_budget;    // clocks a cross-CTA wait may last before it gives up
   int kernel_id;
@@ -204,14 +206,31 @@ __device__ __forceinline__ void report_timeout(const FfnParams& p, int role) {
   atomicCAS(&p.status[1], 0, p.kernel_id * 65536 + role);
 }
 
-// Hold the epilogue until the MMA warp has issued `ik` more K-blocks than at `start`, or cannot advance.
-__device__ __forceinline__ void pace_gap(volatile uint32_t* progress, volatile int* idle, volatile int* aborting,
-                                         uint32_t start, int ik) {
-  for (int spin = 0; spin < (1 << 16); ++spin) {
-    if (*progress - start >= static_cast<uint32_t>(ik) || *idle || *aborting) return;
-    __nanosleep(64);
+// Store pacing of one epilogue warp.  The state lives across the CTA's tiles, so a burst of `burst` store tiles may
+// span accumulators.  After a burst the next store is held until the MMA warp (this CTA's, or the pair leader's: the
+// words are read through their shared::cluster addresses) has issued `ik` more K blocks than when the burst ended,
+// or cannot advance (it waits for an accumulator or has finished), or the CTA is aborting, or a spin cap expires.
+struct Pacer {
+  uint32_t progress_addr, idle_addr;   // shared::cluster addresses of mma_progress / mma_idle
+  int in_burst;                        // store tiles written since the last gap
+  uint32_t burst_end;                  // mma_progress when the current burst was completed
+  long long held;                      // clocks spent holding stores
+  __device__ __forceinline__ void before_store(const int burst, const int ik, volatile int* aborting) {
+    if (in_burst < burst) return;
+    const long long t0 = clock64();
+    for (int spin = 0; spin < (1 << 16); ++spin) {
+      if (ptx::ld_cluster_u32(progress_addr) - burst_end >= static_cast<uint32_t>(ik) ||
+          ptx::ld_cluster_u32(idle_addr) != 0u || *aborting)
+        break;
+      __nanosleep(64);
+    }
+    held += clock64() - t0;
+    in_burst = 0;
   }
-}
+  __device__ __forceinline__ void after_store(const int burst) {
+    if (++in_burst >= burst) burst_end = ptx::ld_cluster_u32(progress_addr);
+  }
+};
 
 // Bounded wait until `*counter` (written by other CTAs with release ordering) reaches `target`.
 __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, volatile int* abort_flag,
@@ -236,18 +255,16 @@ __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target,
 // : 256 plain columns, written as bf16 with 16-byte stores masked to the expert's rows and to N.
 template <bool kGated, bool kFp8>
 __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams& p, uint32_t t_addr, int row,
-                                                  long long* w_gap, volatile uint32_t* progress, volatile int* idle,
-                                                  volatile int* aborting) {
+                                                  Pacer& pacer, volatile int* aborting) {
   const PhaseDesc& d = p.ph[kGated ? 0 : 1];
   const bool row_ok = row < t.row_end;
   __nv_bfloat16* out_row = d.out + static_cast<size_t>(row) * d.N + t.n0;
   constexpr int kChunks = kGated ? (128 / kChunkCols) : (BN_ACC / kChunkCols);
-  int in_burst = 0;
-  uint32_t gap_start = *progress;
 #pragma unroll 1
   for (int c = 0; c < kChunks; ++c) {
     uint32_t v[32];
     float o[32];
+    if (p.mode == 1) pacer.before_store(p.burst, p.ik, aborting);
     if constexpr (kGated) {
       uint32_t u[32];
       ptx::tmem_ld_32x32(t_addr + c * kChunkCols, v);
@@ -319,13 +336,7 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
         }
       }
     }
-    if (p.mode == 1 && ++in_burst >= p.burst && c + 1 < kChunks) {
-      const long long t_gap = clock64();
-      pace_gap(progress, idle, aborting, gap_start, p.ik);
-      *w_gap += clock64() - t_gap;
-      gap_start = *progress;
-      in_burst = 0;
-    }
+    if (p.mode == 1) pacer.after_store(p.burst);
   }
 }
 
@@ -382,7 +393,8 @@ template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wg,
                   const __grid_constant__ CUtensorMap tm_wu, const __grid_constant__ CUtensorMap tm_h,
-                  const __grid_constant__ CUtensorMap tm_wd, const FfnParams p) {
+                  const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_x16,
+                  const __grid_constant__ CUtensorMap tm_h16, const FfnParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -441,6 +453,8 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       ptx::prefetch_tensormap(&tm_wu);
       ptx::prefetch_tensormap(&tm_h);
       ptx::prefetch_tensormap(&tm_wd);
+      ptx::prefetch_tensormap(&tm_x16);
+      ptx::prefetch_tensormap(&tm_h16);
     }
   }
   if (warp == 1) {
@@ -504,7 +518,23 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           }
           ptx::fence_proxy_async_all();   // h was written through the generic proxy, TMA reads through the async one
         }
+        // A tile with swapped operands holds n_pad <= 64 rows: it loads them as n_pad/16 boxes of 16 rows (the same
+        // swizzled layout as the first rows of a 128-row box) instead of 128 rows that are mostly other experts'.
+        const bool small_a = t.n_pad != 0 && p.small_a != 0;
+        const CUtensorMap* ma16 = t.phase == 0 ? &tm_x16 : &tm_h16;
+        const uint32_t stage_tx = small_a ? static_cast<uint32_t>(t.n_pad * 128 + 2 * kBHalfBytes) : kStageBytes;
+        // Such a tile only streams weights it uses once, and what limits it is the bytes one CTA keeps in flight: ask
+        // L2 for the weight boxes a few K blocks ahead of the ring.
+        const int ahead = t.n_pad != 0 ? p.swap_prefetch : 0;
+        for (int kb = 0; kb < ahead && kb < d.k_blocks; ++kb) {
+          ptx::tma_prefetch_l2_2d(mb0, kb * p.k_elems, t.w_row0);
+          ptx::tma_prefetch_l2_2d(mb1, kb * p.k_elems, t.w_row0 + d.b1_row_shift);
+        }
         for (int kb = 0; kb < d.k_blocks; ++kb) {
+          if (kb + ahead < d.k_blocks && ahead > 0) {
+            ptx::tma_prefetch_l2_2d(mb0, (kb + ahead) * p.k_elems, t.w_row0);
+            ptx::tma_prefetch_l2_2d(mb1, (kb + ahead) * p.k_elems, t.w_row0 + d.b1_row_shift);
+          }
           if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, &w_empty)) {
             report_timeout(p, 1);
             ok = false;
@@ -512,8 +542,13 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           }
           const uint32_t full = ptx::smem_u32(&st->full[stage]);
           const uint32_t sa = stage_u32 + stage * kStageBytes;
-          ptx::mbar_expect_tx(full, kStageBytes);
-          ptx::tma_load_2d(sa, ma, full, kb * p.k_elems, t.row0);
+          ptx::mbar_expect_tx(full, stage_tx);
+          if (small_a) {
+            for (int r16 = 0; r16 < t.n_pad; r16 += 16)
+              ptx::tma_load_2d(sa + r16 * 128, ma16, full, kb * p.k_elems, t.row0 + r16);
+          } else {
+            ptx::tma_load_2d(sa, ma, full, kb * p.k_elems, t.row0);
+          }
           ptx::tma_load_2d(sa + kABytes, mb0, full, kb * p.k_elems, t.w_row0);
           ptx::tma_load_2d(sa + kABytes + kBHalfBytes, mb1, full, kb * p.k_elems, t.w_row0 + d.b1_row_shift);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -620,7 +655,8 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     uint32_t acc_phase = 0;
     int slot = 0;
     uint32_t ring_phase = 0;
-    long long w_acc = 0, busy = 0, w_gap = 0;
+    long long w_acc = 0, busy = 0;
+    Pacer pacer{ptx::smem_u32(const_cast<uint32_t*>(&st->mma_progress)), ptx::smem_u32(const_cast<int*>(&st->mma_idle)), 0, 0u, 0};
     while (true) {
       if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
         if (lane == 0) report_timeout(p, 7);
@@ -644,11 +680,9 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         if (t.phase == 0) drain_swapped<true, kFp8>(t, p, t_addr, r_in_tile);
         else drain_swapped<false, kFp8>(t, p, t_addr, r_in_tile);
       } else if (t.phase == 0) {
-        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
-                                      abort_flag);
+        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
       } else {
-        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
-                                       abort_flag);
+        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
       }
       ptx::tc_fence_before_sync();
       if (chained && t.phase == 0) {
@@ -668,7 +702,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     if (p.trace && warp == 2 && lane == 0) {
       p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
       p.trace[blockIdx.x * kMoeTraceFields + 5] = static_cast<unsigned long long>(busy);
-      p.trace[blockIdx.x * kMoeTraceFields + 7] = static_cast<unsigned long long>(w_gap);
+      p.trace[blockIdx.x * kMoeTraceFields + 7] = static_cast<unsigned long long>(pacer.held);
     }
   }
 
@@ -902,7 +936,10 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     const int r_in_tile = quarter * 32 + lane;
     int acc = 0;
     uint32_t acc_phase = 0;
-    long long w_acc = 0, busy = 0, w_gap = 0;
+    long long w_acc = 0, busy = 0;
+    // the MMA warp whose progress paces the stores is the leader's: both CTAs read its words
+    Pacer pacer{ptx::map_to_cta(ptx::smem_u32(const_cast<uint32_t*>(&st->mma_progress)), 0),
+                ptx::map_to_cta(ptx::smem_u32(const_cast<int*>(&st->mma_idle)), 0), 0, 0u, 0};
     const uint32_t empty_leader0 = ptx::map_to_cta(ptx::smem_u32(&st->tmem_empty[0]), 0);
     const uint32_t empty_leader1 = ptx::map_to_cta(ptx::smem_u32(&st->tmem_empty[1]), 0);
     for (int tile = pair; tile < total_tiles; tile += pairs) {
@@ -915,15 +952,10 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       const long long t_store = clock64();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               static_cast<uint32_t>(acc * BN_ACC);
-      // pacing needs the MMA warp's progress counter, which lives in the leader: the peer drains unpaced
-      FfnParams q = p;
-      if (rank != 0) q.mode = 0;
       if (phase == 0)
-        drain_accumulator<true, kFp8>(t, q, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
-                                      abort_flag);
+        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
       else
-        drain_accumulator<false, kFp8>(t, q, t_addr, t.row0 + r_in_tile, &w_gap, &st->mma_progress, &st->mma_idle,
-                                       abort_flag);
+        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(acc ? empty_leader1 : empty_leader0);
@@ -934,7 +966,7 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     if (p.trace && warp == 2 && lane == 0) {
       p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
       p.trace[blockIdx.x * kMoeTraceFields + 5] = static_cast<unsigned long long>(busy);
-      p.trace[blockIdx.x * kMoeTraceFields + 7] = static_cast<unsigned long long>(w_gap);
+      p.trace[blockIdx.x * kMoeTraceFields + 7] = static_cast<unsigned long long>(pacer.held);
     }
   }
 
@@ -1020,16 +1052,40 @@ __global__ void __launch_bounds__(128, 1) mma_cycle_probe(int M, int N, int iter
 }
 
 // Tensor map over a row-major [rows, cols] matrix of bf16 (elem_bytes 2) or E4M3 bytes (elem_bytes 1): boxes of
-// 128 rows x 128 bytes, 128-byte swizzle.
-CUresult encode_2d(moe_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, int elem_bytes) {
+// box_rows rows x 128 bytes, 128-byte swizzle.  Encoding a map costs a few microseconds of host time, and a serving
+// loop calls with the same buffers every step, so the context keeps the last maps it built, keyed by everything
+// that goes into one.
+bool tensor_map_2d(moe_ctx* ctx, const void* base, uint64_t rows, uint64_t cols, int elem_bytes, int box_rows,
+                   CUtensorMap* out) {
+  for (int i = 0; i < ctx->num_maps; ++i) {
+    const moe_map_entry& m = ctx->maps[i];
+    if (m.base == base && m.rows == rows && m.cols == cols && m.elem_bytes == elem_bytes && m.box_rows == box_rows) {
+      *out = m.map;
+      return true;
+    }
+  }
+  moe_map_entry& m = ctx->maps[ctx->num_maps < kMoeMapCache ? ctx->num_maps++ : ctx->next_map_victim++ % kMoeMapCache];
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * static_cast<uint64_t>(elem_bytes)};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes), 128u};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes), static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t elem[2] = {1u, 1u};
-  return ctx->encode_tiled(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
-                           const_cast<void*>(base), dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const CUresult r = ctx->encode_tiled(&m.map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                               : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+                                       const_cast<void*>(base), dims, strides, box, elem,
+                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    m.base = nullptr;
+    m.rows = 0;
+    return false;
+  }
+  m.base = base;
+  m.rows = rows;
+  m.cols = cols;
+  m.elem_bytes = elem_bytes;
+  m.box_rows = box_rows;
+  *out = m.map;
+  return true;
 }
 
 }  // namespace
@@ -1109,10 +1165,13 @@ cudaError_t launch_pair(moe_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b
 }
 }  // namespace
 
-static void launch_single(int grid, const CUtensorMap& x, const CUtensorMap& wg, const CUtensorMap& wu,
-                          const CUtensorMap& h, const CUtensorMap& wd, const FfnParams& p, cudaStream_t stream) {
-  if (p.fp8) expert_ffn_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(x, wg, wu, h, wd, p);
-  else expert_ffn_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(x, wg, wu, h, wd, p);
+struct FfnMaps {
+  CUtensorMap x, wg, wu, h, wd, x16, h16;   // copies: the kernels take them by value
+};
+
+static void launch_single(int grid, const FfnMaps& m, const FfnParams& p, cudaStream_t stream) {
+  if (p.fp8) expert_ffn_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, m.x16, m.h16, p);
+  else expert_ffn_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, m.x16, m.h16, p);
 }
 
 // Everything one expert-FFN call needs on the host side; fp8 selects E4M3 operands with epilogue scales.
@@ -1139,12 +1198,15 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   const int eb = c.fp8 ? 1 : 2;
   const int k_elems = 128 / eb;
 
-  CUtensorMap tm_x, tm_wg, tm_wu, tm_h, tm_wd;
-  if (encode_2d(ctx, &tm_x, c.a1, R, s.H, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
-  if (encode_2d(ctx, &tm_wg, c.w_gate, static_cast<uint64_t>(s.E) * s.F, s.H, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
-  if (encode_2d(ctx, &tm_wu, c.w_up, static_cast<uint64_t>(s.E) * s.F, s.H, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
-  if (encode_2d(ctx, &tm_h, c.a2, R, s.F, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
-  if (encode_2d(ctx, &tm_wd, c.w_down, static_cast<uint64_t>(s.E) * s.H, s.F, eb) != CUDA_SUCCESS) return MOE_ERR_CUDA;
+  FfnMaps m;
+  {
+    const uint64_t EF = static_cast<uint64_t>(s.E) * s.F, EH = static_cast<uint64_t>(s.E) * s.H;
+    const bool ok = tensor_map_2d(ctx, c.a1, R, s.H, eb, 128, &m.x) && tensor_map_2d(ctx, c.w_gate, EF, s.H, eb, 128, &m.wg) &&
+                    tensor_map_2d(ctx, c.w_up, EF, s.H, eb, 128, &m.wu) && tensor_map_2d(ctx, c.a2, R, s.F, eb, 128, &m.h) &&
+                    tensor_map_2d(ctx, c.w_down, EH, s.F, eb, 128, &m.wd) && tensor_map_2d(ctx, c.a1, R, s.H, eb, 16, &m.x16) &&
+                    tensor_map_2d(ctx, c.a2, R, s.F, eb, 16, &m.h16);
+    if (!ok) return MOE_ERR_CUDA;
+  }
 
   FfnParams p{};
   p.offsets = offsets;
@@ -1162,6 +1224,9 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   p.schedule = tn.schedule;
   p.fp8 = c.fp8;
   p.k_elems = k_elems;
+  p.small_a = moe_knob_value(ctx, "small_a", 1);
+  p.swap_prefetch = moe_knob_value(ctx, "swap_prefetch", 0);
+  if (p.swap_prefetch < 0 || p.swap_prefetch > 64) return MOE_ERR_INVALID_ARG;
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
   // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
   p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);
@@ -1190,7 +1255,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.trace = trace ? ctx->d_trace : nullptr;
     p.order_log = trace ? ctx->d_order : nullptr;
     p.kernel_id = 3;
-    launch_single(grid, tm_x, tm_wg, tm_wu, tm_h, tm_wd, p, stream);
+    launch_single(grid, m, p, stream);
     moe_mark(ctx, 5, stream);
     moe_mark(ctx, 6, stream);
     ctx->last_launches += 1;
@@ -1203,9 +1268,9 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.trace = trace ? ctx->d_trace : nullptr;
     p.kernel_id = pairs ? 4 : 1;
     if (pairs) {
-      if (launch_pair(ctx, tm_x, tm_wg, tm_wu, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+      if (launch_pair(ctx, m.x, m.wg, m.wu, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
-      launch_single(grid, tm_x, tm_wg, tm_wu, tm_h, tm_wd, p, stream);
+      launch_single(grid, m, p, stream);
     }
     moe_mark(ctx, 5, stream);
     ctx->last_launches += 1;
@@ -1217,9 +1282,9 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.trace = trace2;
     p.kernel_id = pairs ? 5 : 2;
     if (pairs) {
-      if (launch_pair(ctx, tm_h, tm_wd, tm_wd, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+      if (launch_pair(ctx, m.h, m.wd, m.wd, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
-      launch_single(grid, tm_x, tm_wg, tm_wu, tm_h, tm_wd, p, stream);
+      launch_single(grid, m, p, stream);
     }
     moe_mark(ctx, 6, stream);
     ctx->last_launches += 1;

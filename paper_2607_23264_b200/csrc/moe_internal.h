@@ -30,6 +30,15 @@ struct moe_knob {
   int32_t value;
 };
 
+// Tensor maps the grouped GEMMs built for recent calls (see tensor_map_2d).
+constexpr int kMoeMapCache = 24;
+struct moe_map_entry {
+  const void* base;
+  uint64_t rows, cols;
+  int elem_bytes, box_rows;
+  CUtensorMap map;
+};
+
 struct moe_ctx {
   moe_shape shape;
   int has_env_tuning;    // MOE_TUNING named at least one moe_tuning field: env_tuning replaces the defaults of a
@@ -51,6 +60,9 @@ struct moe_ctx {
   int32_t* d_order;       // [num_sms][kMoeOrderLogCap] tile codes drawn by each CTA in the last traced one-launch run
   unsigned long long* d_trace;   // [2][num_sms][kMoeTraceFields] wait counters of Linear-1 and Linear-2
   moe_encode_tiled_fn encode_tiled;
+  int num_maps;
+  unsigned next_map_victim;
+  moe_map_entry maps[kMoeMapCache];
   int32_t last_launches;
   // Two-deep pipeline of moe_fused_forward_host_pipelined: copy streams, per-slot events, next slot.
   cudaStream_t s_h2d, s_d2h;

@@ -1,6 +1,8 @@
 // Host-side X-Stage (Burst-Gap) calculator: include/xstage.h.  Pure double-precision arithmetic, no GPU work.
+#include <algorithm>
 #include <cmath>
 #include <limits>
+#include <vector>
 
 #include "../../include/xstage.h"
 
@@ -8,9 +10,67 @@ namespace {
 inline double pos(double z) { return z > 0.0 ? z : 0.0; }
 inline bool ok(const xstage_params* m) { return m && m->rate > 0.0 && m->t_iss0 >= 0.0; }
 const double kNaN = std::numeric_limits<double>::quiet_NaN();
+double median_of(std::vector<double> v) {
+  std::sort(v.begin(), v.end());
+  const size_t n = v.size();
+  return n % 2 ? v[n / 2] : 0.5 * (v[n / 2 - 1] + v[n / 2]);
+}
 }  // namespace
 
 extern "C" {
+
+int xstage_calibrate(int64_t n_periodic, const double* p_volume, const double* p_gap, const double* p_t_iss,
+                     const double* p_t_period, int64_t n_isolated, const double* i_volume, const double* i_t_iss,
+                     double knee_tolerance, xstage_calibration* out) {
+  if (!out || n_periodic < 1 || !p_volume || !p_gap || !p_t_iss || !p_t_period || n_isolated < 0 ||
+      (n_isolated > 0 && (!i_volume || !i_t_iss)) || !(knee_tolerance >= 0.0))
+    return -1;
+  *out = xstage_calibration{};
+  // the plateau: rows whose gap is among the largest third of the distinct gaps
+  std::vector<double> gaps(p_gap, p_gap + n_periodic);
+  std::sort(gaps.begin(), gaps.end());
+  gaps.erase(std::unique(gaps.begin(), gaps.end()), gaps.end());
+  const size_t third = std::max<size_t>(1, gaps.size() / 3);
+  const double threshold = gaps[gaps.size() - third];
+  std::vector<double> plateau, rates;
+  for (int64_t i = 0; i < n_periodic; ++i) {
+    if (p_gap[i] >= threshold) plateau.push_back(p_t_iss[i]);
+    if (p_gap[i] == 0.0) {
+      if (!(p_t_period[i] > 0.0)) return -1;
+      rates.push_back(p_volume[i] / p_t_period[i]);
+    }
+  }
+  out->t_iss0 = median_of(plateau);
+  out->rate = rates.empty() ? 0.0 : median_of(rates);
+  if (n_isolated < 3 || rates.empty()) return 0;
+  // least-squares line through the smallest third of the isolated volumes
+  const int64_t n = std::max<int64_t>(3, n_isolated / 3);
+  double mx = 0.0, my = 0.0;
+  for (int64_t i = 0; i < n; ++i) {
+    mx += i_volume[i];
+    my += i_t_iss[i];
+  }
+  mx /= n;
+  my /= n;
+  double sxx = 0.0, sxy = 0.0;
+  for (int64_t i = 0; i < n; ++i) {
+    sxx += (i_volume[i] - mx) * (i_volume[i] - mx);
+    sxy += (i_volume[i] - mx) * (i_t_iss[i] - my);
+  }
+  const double b = sxx > 0.0 ? sxy / sxx : 0.0;
+  const double a = my - b * mx;
+  out->floor_intercept = a;
+  out->floor_per_byte = b;
+  for (int64_t i = n; i < n_isolated; ++i) {
+    if (i_t_iss[i] > (1.0 + knee_tolerance) * (a + b * i_volume[i])) {
+      out->has_knee = 1;
+      out->knee_volume = i_volume[i - 1];
+      out->capacity = pos(i_volume[i - 1] - out->rate * i_t_iss[i - 1]);
+      break;
+    }
+  }
+  return 0;
+}
 
 int xstage_burst_gap(const xstage_params* m, double volume, double gap, double* t_period, double* t_iss) {
   if (!ok(m) || volume < 0.0 || gap < 0.0) return -1;

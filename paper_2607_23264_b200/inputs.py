@@ -68,6 +68,9 @@ CONFIGS = {
     "P1": MoEConfig("P1", T=2048, H=4096, F=14336, E=2, k=2, seed=4, router="xWr"),
     # P2 = C2's row movers (dispatch/combine traffic of a 16384-token batch) with token-sized experts
     "P2": MoEConfig("P2", T=16384, H=4096, F=64, E=8, k=2, seed=5, router="xWr"),
+    # P3 = a slice of the DeepSeek-V3-like layer: the same expert shape and skewed routing over 32 experts (2.8 GB of
+    # weights), which mixes many-row experts, single-block experts and swapped-operand tiles in one launch
+    "P3": MoEConfig("P3", T=256, H=7168, F=2048, E=32, k=8, seed=6, router="xWr_zipf"),
 }
 
 

@@ -47,3 +47,16 @@ def max_over_ranks(value: float, world: int, device="cpu") -> float:
 def job_tokens_per_second(tokens_per_rank: int, world: int, steps: int, slowest_ms: float) -> float:
     """Whole-job throughput: all ranks' tokens over the slowest rank's time."""
     return tokens_per_rank * world * steps / (slowest_ms * 1e-3)
+
+
+def launcher_command(n_gpus: int, script: str, argv, port: int, python: str = "python"):
+    """Command and extra environment that start `script argv` as n_gpus ranks on this node, one per GPU.
+
+    The ranks meet over 127.0.0.1 (a container's host name may not resolve).  NCCL's own log stays on at INFO level
+    unless the caller's environment already sets it, so that a run's output shows how many ranks joined."""
+    if n_gpus < 2:
+        raise ValueError("a launcher is needed for two or more ranks only")
+    cmd = [python, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), script, *argv]
+    env = {"NCCL_DEBUG": "INFO"}
+    return cmd, env

@@ -12,7 +12,7 @@ class xstage_params(C.Structure):
 
 EXPORTS = ("xstage_burst_gap", "xstage_recovery_gap", "xstage_isolated_occupancy", "xstage_audit",
            "xstage_interleaved_gap", "xstage_interleaved_issue_overhead", "xstage_average_rate_feasible",
-           "xstage_lead_knee", "xstage_mma_stall", "xstage_fa_recovery_length", "xstage_store_probe")
+           "xstage_lead_knee", "xstage_mma_stall", "xstage_fa_recovery_length", "xstage_store_probe", "xstage_calibrate")
 
 _ready = False
 
@@ -43,6 +43,8 @@ def _lib():
         lib.xstage_store_probe.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_void_p, C.c_uint64, dp, dp, dp,
                                            dp, C.c_void_p]
         lib.xstage_store_probe.restype = C.c_int
+        lib.xstage_calibrate.argtypes = [C.c_int64, dp, dp, dp, dp, C.c_int64, dp, dp, d, C.c_void_p]
+        lib.xstage_calibrate.restype = C.c_int
         _ready = True
     return lib
 
@@ -122,37 +124,31 @@ def xstage_store_probe(producers, bytes_per_burst, gap_clocks, periods, device_b
     return dict(issue_mean=list(im), issue_max=list(ix), period_mean=list(pm), clocks_per_us=cpu.value)
 
 
-def calibrate(periodic, isolated, knee_tolerance=0.10):
-    """The paper's calibration (Sec. 3.3, Sec. 3.5) from microbenchmark rows.
+class xstage_calibration(C.Structure):
+    _fields_ = [(n, C.c_double) for n in ("t_iss0", "rate", "capacity", "knee_volume", "floor_intercept",
+                                          "floor_per_byte")] + [("has_knee", C.c_int32)]
+
+
+def xstage_calibrate(periodic, isolated, knee_tolerance=0.10):
+    """Calibrate (T_iss^0, R, Q) from microbenchmark rows: marshals the rows into arrays for the C routine.
 
     periodic: rows dict(volume, gap, t_iss, t_period) of one burst volume at several gaps, gap 0 included;
     isolated: rows dict(volume, t_iss) from a recovered state, ascending volume.
-    T_iss^0 = median issue time over the largest third of the gaps (the plateau); R = V / T_period at zero gap
-    (the drain-limited steady state).  Isolated bursts: the recovered issue floor depends on the volume (the
-    issue loop itself takes time), so it is a line a + b V fitted to the smallest third of the volumes; the knee
-    is the largest volume whose issue time stays within (1 + knee_tolerance) of that line before the first one
-    that leaves it; Q = [V_knee - R T_iss(V_knee)]_+ (Eq. 6 from a recovered state).
-    Returns dict(t_iss0, rate, capacity, knee_volume, floor_intercept, floor_per_byte); capacity and knee_volume
-    are None when no row leaves the floor line."""
-    import statistics
-    gaps = sorted({r["gap"] for r in periodic})
-    plateau = [r["t_iss"] for r in periodic if r["gap"] >= gaps[-max(1, len(gaps) // 3)]]
-    t0 = statistics.median(plateau)
-    zero = [r for r in periodic if r["gap"] == 0]
-    rate = statistics.median(r["volume"] / r["t_period"] for r in zero) if zero else None
-    knee, a, b = None, None, None
-    if isolated and rate:
-        fit = isolated[: max(3, len(isolated) // 3)]
-        n = len(fit)
-        mx = sum(r["volume"] for r in fit) / n
-        my = sum(r["t_iss"] for r in fit) / n
-        sxx = sum((r["volume"] - mx) ** 2 for r in fit)
-        b = sum((r["volume"] - mx) * (r["t_iss"] - my) for r in fit) / sxx if sxx > 0 else 0.0
-        a = my - b * mx
-        for i, r in enumerate(isolated):
-            if i >= n and r["t_iss"] > (1.0 + knee_tolerance) * (a + b * r["volume"]):
-                knee = isolated[i - 1]
-                break
-    cap = None if knee is None else max(knee["volume"] - rate * knee["t_iss"], 0.0)
-    return dict(t_iss0=t0, rate=rate, capacity=cap, knee_volume=None if knee is None else knee["volume"],
-                floor_intercept=a, floor_per_byte=b)
+    Returns dict(t_iss0, rate, capacity, knee_volume, floor_intercept, floor_per_byte); rate is None without a
+    zero-gap row, capacity and knee_volume are None when no row leaves the floor line."""
+    col = lambda rows, key: (C.c_double * len(rows))(*[float(r[key]) for r in rows])
+    out = xstage_calibration()
+    lib = _lib()
+    rc = lib.xstage_calibrate(len(periodic), col(periodic, "volume"), col(periodic, "gap"), col(periodic, "t_iss"),
+                              col(periodic, "t_period"), len(isolated), col(isolated, "volume"), col(isolated, "t_iss"),
+                              float(knee_tolerance), C.byref(out))
+    if rc != 0:
+        raise ValueError("xstage_calibrate: bad argument")
+    fitted = len(isolated) >= 3 and out.rate > 0
+    return dict(t_iss0=out.t_iss0, rate=out.rate if out.rate > 0 else None,
+                capacity=out.capacity if out.has_knee else None, knee_volume=out.knee_volume if out.has_knee else None,
+                floor_intercept=out.floor_intercept if fitted else None,
+                floor_per_byte=out.floor_per_byte if fitted else None)
+
+
+calibrate = xstage_calibrate

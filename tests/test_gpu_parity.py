@@ -184,7 +184,7 @@ def test_pipelined_host_calls_match_device_path():
 
 def test_pacing_points_are_bitwise_identical():
     """Store pacing reorders stores in time only: all 20 sweep points give the same bits."""
-    cfg = gen.MoEConfig("pace", T=900, H=512, F=768, E=4, k=2, seed=31, router="xWr")
+    cfg = gen.MoEConfig("pace", T=2400, H=512, F=1024, E=4, k=2, seed=31, router="xWr")   # large enough for two launches
     L = Layer(cfg)
     ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
     base = L.nan_bf16(cfg.T, cfg.H)
@@ -194,13 +194,63 @@ def test_pacing_points_are_bitwise_identical():
     assert_out_close(dev_bf16_to_f64(base), ref["out"], "pacing baseline")
     points = [(b, 0, 1) for b in (1, 2, 4, 8, 16)] + [(b, 1, ik) for b in (1, 2, 4, 8, 16) for ik in (1, 2, 4)]
     assert len(points) == 20
-    for b, mode, ik in points:
-        out = L.nan_bf16(cfg.T, cfg.H)
-        L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws,
-                                tuning=binding.make_tuning(b, mode, ik))
-        torch.cuda.synchronize()
-        assert torch.equal(out.view(torch.int16), base.view(torch.int16)), (b, mode, ik)
+    for pairs in (0, 8):                       # the single-CTA kernel, then the CTA-pair kernel (forced)
+        for b, mode, ik in points:
+            out = L.nan_bf16(cfg.T, cfg.H)
+            L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws,
+                                    tuning=binding.make_tuning(b, mode, ik, debug_flags=pairs))
+            torch.cuda.synchronize()
+            assert torch.equal(out.view(torch.int16), base.view(torch.int16)), (pairs, b, mode, ik)
     L.check_device_status()
+    # in a CTA pair both CTAs pace their stores on the leader's MMA progress: with a gap after every store tile the
+    # hold counter (trace field 7) moves in leaders (even CTAs) and peers (odd CTAs) that drained a tile
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws,
+                            tuning=binding.make_tuning(1, 1, 4, debug_flags=8 | 1))
+    torch.cuda.synchronize()
+    tr = L.ctx.moe_get_ffn_trace()
+    drained = tr[1][:, 5] > 0
+    assert drained[0::2].any() and drained[1::2].any()
+    held = tr[1][:, 7] > 0
+    assert held[0::2][drained[0::2]].any(), "no leader CTA held a store"
+    assert held[1::2][drained[1::2]].any(), "no peer CTA held a store: the peer drains unpaced"
+    # a burst larger than one output tile (16 store tiles = two Linear-2 tiles) still inserts gaps: the burst spans tiles
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws,
+                            tuning=binding.make_tuning(16, 1, 4, debug_flags=16 | 1))
+    torch.cuda.synchronize()
+    tr = L.ctx.moe_get_ffn_trace()
+    assert (tr[1][:, 7] > 0).any(), "burst 16 never held a store"
+    L.check_device_status()
+
+
+def test_environment_override_of_the_default_tuning(monkeypatch):
+    """MOE_TUNING, read by moe_create, replaces the tuning of calls that pass none; an explicit tuning wins; a string
+    the parser rejects makes moe_create fail."""
+    cfg = gen.MoEConfig("env", T=2000, H=512, F=1024, E=6, k=2, seed=33, router="xWr")   # large enough for two launches
+    base_layer = Layer(cfg)
+    ws = torch.empty(base_layer.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    base = base_layer.nan_bf16(cfg.T, cfg.H)
+    # the built-in default runs the two GEMMs as two launches (7 kernels); the override asks for the interleaved order,
+    # which runs them as one launch (6 kernels)
+    base_layer.ctx.moe_fused_forward(base_layer.x, base_layer.d_logits, base_layer.w_gate, base_layer.w_up,
+                                     base_layer.w_down, base, ws, tuning=binding.make_tuning(debug_flags=16))
+    torch.cuda.synchronize()
+    assert base_layer.ctx.moe_last_launch_count() == 7
+    monkeypatch.setenv("MOE_TUNING", "schedule=1,lead=4,x.swap_prefetch=0")
+    L = Layer(cfg)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
+    torch.cuda.synchronize()
+    assert L.ctx.moe_last_launch_count() == 6, "the environment's schedule was not used"
+    assert torch.equal(out.view(torch.int16), base.view(torch.int16))
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws,
+                            tuning=binding.make_tuning(debug_flags=16))
+    torch.cuda.synchronize()
+    assert L.ctx.moe_last_launch_count() == 7, "an explicit tuning must win over the environment"
+    L.check_device_status()
+    monkeypatch.setenv("MOE_TUNING", "burst=3")
+    with pytest.raises(binding.MoeError) as ei:
+        binding.Context(cfg.T, cfg.H, cfg.F, cfg.E, cfg.k)
+    assert ei.value.code == 1
 
 
 @pytest.mark.parametrize("cfg", [SMALL[0], SMALL[1], SMALL[5], SMALL[7],

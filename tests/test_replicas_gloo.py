@@ -51,3 +51,15 @@ def test_single_rank_needs_no_process_group():
     x = np.arange(12, dtype=np.uint16).reshape(4, 3)
     assert replicas.rank_batch(x, 0) is x
     assert np.array_equal(replicas.rank_batch(x, 1), np.roll(x, 17, axis=0))
+
+
+def test_launcher_command_for_two_ranks():
+    cmd, env = replicas.launcher_command(2, "bench.py", ["--gpus", "2", "--steps", "5"], port=29511, python="python3")
+    assert cmd[:3] == ["python3", "-m", "torch.distributed.run"]
+    assert "--nnodes=1" in cmd and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29511"
+    assert cmd[-5:] == ["bench.py", "--gpus", "2", "--steps", "5"], "the script and its own arguments come last"
+    assert env == {"NCCL_DEBUG": "INFO"}
+    import pytest
+    with pytest.raises(ValueError):
+        replicas.launcher_command(1, "bench.py", [], port=1)

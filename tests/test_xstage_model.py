@@ -4,6 +4,7 @@ import math
 import os
 import random
 
+import numpy as np
 import pytest
 
 from oracle import xstage_oracle as xo
@@ -190,6 +191,46 @@ def test_calibrate_recovers_model_parameters_from_synthetic_rows():
     assert c["capacity"] <= Q + R * floor and Q - c["capacity"] < 3 * step
     flat = xstage.calibrate(periodic, [dict(volume=r["volume"], t_iss=floor) for r in isolated])
     assert flat["capacity"] is None and flat["knee_volume"] is None, "no knee, no capacity estimate"
+    # the oracle's own calibration is pinned by the same known parameters
+    t0, rate, cap, knee = xo.calibrate([(r["volume"], r["gap"], r["t_iss"], r["t_period"]) for r in periodic],
+                                       [(r["volume"], r["t_iss"]) for r in isolated])
+    assert t0 == pytest.approx(T0) and rate == pytest.approx(R)
+    assert cap <= Q + R * floor and Q - cap < 3 * step and knee == c["knee_volume"]
+
+
+def test_calibrate_matches_the_oracle_on_noisy_rows():
+    """The C routine against the oracle's calibration on random model parameters with measurement noise."""
+    rng = np.random.default_rng(11)
+    for case in range(40):
+        T0, R, Q = rng.uniform(200, 2000), rng.uniform(500, 5000), rng.uniform(2e6, 3e7)
+        floor_a, floor_b = rng.uniform(50, 400), rng.uniform(0, 2e-5)
+        V = 148 * int(rng.integers(4, 64)) * 1024
+        gaps = [0, 250, 500, 1000, 2000, 4000, 8000, 16000, 32000][: int(rng.integers(3, 10))]
+        periodic = []
+        for gap in gaps:
+            for _ in range(int(rng.integers(1, 3))):
+                tp, ti = xo.burst_gap(T0, R, V, gap)
+                periodic.append(dict(volume=V, gap=gap, t_iss=ti * rng.uniform(0.97, 1.03), t_period=tp * rng.uniform(0.97, 1.03)))
+        isolated = []
+        for b in (2048 * i for i in range(1, int(rng.integers(4, 90)))):
+            v = 148 * b
+            f = floor_a + floor_b * v
+            over = xo.pos(xo.isolated_occupancy(f, R, v) - Q)
+            isolated.append(dict(volume=v, t_iss=(f + over / R) * rng.uniform(0.98, 1.02)))
+        tol = float(rng.choice([0.05, 0.10, 0.25]))
+        c = xstage.calibrate(periodic, isolated, knee_tolerance=tol)
+        t0, rate, cap, knee = xo.calibrate([(r["volume"], r["gap"], r["t_iss"], r["t_period"]) for r in periodic],
+                                           [(r["volume"], r["t_iss"]) for r in isolated], knee_tolerance=tol)
+        assert c["t_iss0"] == pytest.approx(t0, rel=1e-12) and c["rate"] == pytest.approx(rate, rel=1e-12)
+        assert c["knee_volume"] == knee, case
+        if cap is None:
+            assert c["capacity"] is None
+        else:
+            assert c["capacity"] == pytest.approx(cap, rel=1e-9, abs=1e-6)
+    with pytest.raises(ValueError):
+        xstage.calibrate([], [])
+    only_large_gaps = xstage.calibrate([dict(volume=1e6, gap=100.0, t_iss=5.0, t_period=105.0)], [])
+    assert only_large_gaps["rate"] is None and only_large_gaps["t_iss0"] == 5.0
 
 
 @pytest.mark.gpu
