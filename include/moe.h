@@ -443,13 +443,15 @@ int32_t moe_last_launch_count(const moe_ctx* ctx);
 /*
  * Wait counters of the two grouped GEMMs (the instrumentation of Sec. 5.1 / App. A.2: per-tile store spans and
  * the MMA-side wait for a free accumulator, there read with clock64()).  When a call ran with
- * tuning->debug_flags bit 0 set, every CTA of Linear-1 and of Linear-2 recorded eight 64-bit counters, in SM
+ * tuning->debug_flags bit 0 set, every CTA of Linear-1 and of Linear-2 recorded twelve 64-bit counters, in SM
  * clocks: 0 producer loop span, 1 producer waited for a free shared-memory stage, 2 MMA warp waited for
  * operands, 3 MMA warp waited for a free accumulator (the epilogue's back-pressure, the paper's tmem_empty
  * wait), 4 epilogue waited for a finished accumulator, 5 epilogue drain-and-store span, 6 tiles processed
- * (a count), 7 epilogue held by the pacing gap.  This call synchronises `stream` and copies
- * counters_host[2][*num_ctas][8] (Linear-1 first) to HOST memory; capacity is in 64-bit elements and must be
- * at least 16 * (number of SMs).
+ * (a count), 7 epilogue held by the pacing gap, 8 tiles computed with swapped operands (a count), 9 the MMA
+ * warp's time in those tiles, 10 the part of it spent waiting for operands, 11 its time in the other tiles
+ * (8-11: single-CTA bf16/E4M3 kernel only, zero elsewhere).  This call synchronises `stream` and copies
+ * counters_host[2][*num_ctas][12] (Linear-1 first) to HOST memory; capacity is in 64-bit elements and must be
+ * at least 24 * (number of SMs).
  */
 moe_status moe_get_ffn_trace(moe_ctx* ctx, uint64_t* counters_host, int32_t capacity, int32_t* num_ctas,
                              void* stream);

@@ -33,7 +33,8 @@ EXPORTS = (
 )
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
-                "epilogue_wait_accumulator", "epilogue_store_span", "tiles", "epilogue_pacing_gap")
+                "epilogue_wait_accumulator", "epilogue_store_span", "tiles", "epilogue_pacing_gap",
+                "swapped_tiles", "swapped_tile_clocks", "swapped_wait_operands", "full_tile_clocks")
 
 KERNEL_NAMES = ("route_topk_hist", "route_scan", "route_scatter", "dispatch_rows", "expert_ffn_linear1",
                 "expert_ffn_linear2", "combine_rows")

@@ -1,8 +1,8 @@
 // Dispatch and combine: the two HBM-bound row movers of the layer.
 //
-// dispatch: token-centric.  A warp owns one token at a time, reads its row once with 16-byte loads and
-//           writes it to the k rows of the expert-contiguous buffer named by inv_perm.  Algorithmic
-//           traffic: 2H(T + R) bytes.
+// dispatch: token-centric.  A warp owns a (token, column block) item, reads that part of the token's row once
+//           with 16-byte loads and writes it to the k rows of the expert-contiguous buffer named by
+//           inv_perm.  Algorithmic traffic: 2H(T + R) bytes.
 // combine : a warp owns a (token, column block) item, gathers the k expert rows named by inv_perm,
 //           accumulates w[t,j] * y in fp32 in ascending j and writes bf16.  No atomics, fixed order.
 //           Algorithmic traffic: 2H(R + T) + 8R bytes.
@@ -13,37 +13,6 @@
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kVecPerLane = 4;                       // 16-byte vectors a lane keeps in flight
-constexpr int kVecPerPass = 32 * kVecPerLane;        // vectors a warp moves per pass (2 KiB)
-
-__global__ void __launch_bounds__(kThreads)
-dispatch_rows(const uint4* __restrict__ x, const int32_t* __restrict__ inv_perm, uint4* __restrict__ x_perm,
-              int T, int k, int vec_per_row) {
-  const int lane = threadIdx.x & 31;
-  const int warps_total = gridDim.x * (kThreads / 32);
-  const int gwarp = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-  for (int t = gwarp; t < T; t += warps_total) {
-    const int my_row = (lane < k) ? inv_perm[static_cast<size_t>(t) * k + lane] : 0;
-    const uint4* src = x + static_cast<size_t>(t) * vec_per_row;
-    for (int v0 = 0; v0 < vec_per_row; v0 += kVecPerPass) {
-      uint4 buf[kVecPerLane];
-#pragma unroll
-      for (int u = 0; u < kVecPerLane; ++u) {
-        const int v = v0 + u * 32 + lane;
-        if (v < vec_per_row) buf[u] = __ldg(src + v);
-      }
-      for (int j = 0; j < k; ++j) {
-        const int row = __shfl_sync(0xFFFFFFFFu, my_row, j);
-        uint4* dst = x_perm + static_cast<size_t>(row) * vec_per_row;
-#pragma unroll
-        for (int u = 0; u < kVecPerLane; ++u) {
-          const int v = v0 + u * 32 + lane;
-          if (v < vec_per_row) dst[v] = buf[u];
-        }
-      }
-    }
-  }
-}
 
 // 16-byte load of data read once: through the read-only path, not kept in L1
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
@@ -52,6 +21,39 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(p));
   return v;
+}
+
+// One item = one token x (32 * V) 16-byte vectors of its row: read once, written to the k rows inv_perm names.
+// Items rather than whole tokens per warp keep enough independent loads in flight for rows of several KiB.
+template <int V>
+__global__ void __launch_bounds__(kThreads)
+dispatch_rows(const uint4* __restrict__ x, const int32_t* __restrict__ inv_perm, uint4* __restrict__ x_perm,
+              int T, int k, int vec_per_row, int blocks_per_row) {
+  const int lane = threadIdx.x & 31;
+  const long long warps_total = static_cast<long long>(gridDim.x) * (kThreads / 32);
+  const long long gwarp = static_cast<long long>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
+  const long long items = static_cast<long long>(T) * blocks_per_row;
+  for (long long item = gwarp; item < items; item += warps_total) {
+    const int t = static_cast<int>(item / blocks_per_row);
+    const int v0 = static_cast<int>(item % blocks_per_row) * (32 * V);
+    const int my_row = (lane < k) ? __ldg(inv_perm + static_cast<size_t>(t) * k + lane) : 0;
+    const uint4* src = x + static_cast<size_t>(t) * vec_per_row;
+    uint4 buf[V];
+#pragma unroll
+    for (int u = 0; u < V; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < vec_per_row) buf[u] = ld_stream(src + v);
+    }
+    for (int j = 0; j < k; ++j) {
+      const int row = __shfl_sync(0xFFFFFFFFu, my_row, j);
+      uint4* dst = x_perm + static_cast<size_t>(row) * vec_per_row;
+#pragma unroll
+      for (int u = 0; u < V; ++u) {
+        const int v = v0 + u * 32 + lane;
+        if (v < vec_per_row) dst[v] = buf[u];
+      }
+    }
+  }
 }
 
 __device__ __forceinline__ void fma8(float (&acc)[8], float w, const uint4& v) {
@@ -67,8 +69,8 @@ __device__ __forceinline__ void fma8(float (&acc)[8], float w, const uint4& v) {
 // One item = one token x (32 * V) 16-byte vectors of its row.  The k expert rows are fetched in batches of kCombBatch
 // rows: all loads of a batch (kCombBatch * V per lane) are issued before the first of its FMAs, which then run in
 // ascending j, so the memory system sees the whole batch at once while the summation order stays the contract's.
-// What bounds the kernel is the bytes an SM keeps in flight (resident warps x loads per lane x 16 bytes), so V and
-// the batch are chosen per k: few rows per token -> more vectors per lane.
+// What bounds the kernel is the bytes an SM keeps in flight (resident warps x loads per lane x 16 bytes); V and the
+// batch are template parameters because registers decide how many warps are resident (the launcher picks them).
 template <int V, int kCombBatch>
 __global__ void __launch_bounds__(kThreads)
 combine_rows(const uint4* __restrict__ y_perm, const int32_t* __restrict__ inv_perm,
@@ -138,12 +140,19 @@ cudaError_t launch_dispatch(moe_ctx* ctx, const void* x, const int32_t* inv_perm
                             cudaStream_t stream) {
   const moe_shape& s = ctx->shape;
   const int vec_per_row = s.H / 8;
+  int V = moe_knob_value(ctx, "dispatch_vec", 0);
+  if (V != 1 && V != 2 && V != 4) V = 4;
+  while (V > 1 && vec_per_row < 32 * V) V >>= 1;
+  const int blocks_per_row = (vec_per_row + 32 * V - 1) / (32 * V);
+  const long long items = static_cast<long long>(s.T) * blocks_per_row;
   const int warps_per_block = kThreads / 32;
-  int blocks = (s.T + warps_per_block - 1) / warps_per_block;
-  const int cap = ctx->num_sms * 8;
-  if (blocks > cap) blocks = cap;
-  dispatch_rows<<<blocks, kThreads, 0, stream>>>(static_cast<const uint4*>(x), inv_perm,
-                                                 static_cast<uint4*>(x_perm), s.T, s.k, vec_per_row);
+  long long blocks = (items + warps_per_block - 1) / warps_per_block;
+  const long long cap = static_cast<long long>(ctx->num_sms) * moe_knob_value(ctx, "dispatch_ctas_per_sm", 16);
+  if (blocks > cap && cap > 0) blocks = cap;
+  auto kernel = V == 4 ? dispatch_rows<4> : V == 2 ? dispatch_rows<2> : dispatch_rows<1>;
+  kernel<<<static_cast<int>(blocks), kThreads, 0, stream>>>(static_cast<const uint4*>(x), inv_perm,
+                                                            static_cast<uint4*>(x_perm), s.T, s.k, vec_per_row,
+                                                            blocks_per_row);
   moe_mark(ctx, 4, stream);
   ctx->last_launches += 1;
   return cudaGetLastError();
@@ -153,9 +162,11 @@ cudaError_t launch_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_
                            void* out, cudaStream_t stream) {
   const moe_shape& s = ctx->shape;
   const int vec_per_row = s.H / 8;
-  // loads a lane keeps in flight = batch x V: about 8, split by k (the batch never exceeds the rows of a token)
-  int batch = s.k >= 8 ? 8 : s.k >= 4 ? 4 : s.k >= 2 ? 2 : 1;
-  int V = 8 / batch > 4 ? 4 : 8 / batch;
+  // Measured on the Mixtral-like (k = 2) and DeepSeek-V3-like (k = 8) movers: four vectors per lane, rows taken one at
+  // a time (72 registers, three resident CTAs per SM), beats every variant that batches rows or narrows the item; only
+  // batches of a few dozen tokens prefer one vector per lane with the rows batched (more warps, fewer bytes each).
+  int batch = 1, V = 4;
+  if (s.T < 2 * ctx->num_sms) { V = 1; batch = s.k >= 4 ? 4 : s.k >= 2 ? 2 : 1; }
   while (V > 1 && vec_per_row < 32 * V) V >>= 1;
   const int kv = moe_knob_value(ctx, "combine_vec", 0), kb = moe_knob_value(ctx, "combine_batch", 0);
   if (kv == 1 || kv == 2 || kv == 4) V = kv;

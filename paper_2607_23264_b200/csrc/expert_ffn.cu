@@ -71,6 +71,7 @@ struct SharedTail {
   volatile int mma_idle;            // 1 while the MMA warp waits for an accumulator or has finished
   int32_t hot_prefix[kMaxExperts + 1];    // exclusive prefix of 128-row blocks over hot experts (cold count 0)
   int32_t cold_prefix[kMaxExperts + 1];   // the same over cold experts
+  int32_t offs[kMaxExperts + 1];          // the expert row offsets, copied once: tile decoding reads no global memory
 };
 
 constexpr size_t kSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStages) * kStageBytes + sizeof(SharedTail);
@@ -106,8 +107,7 @@ struct FfnParams {
   int lead_D;               // Algorithm 1: minimum row lead of Linear-1 over Linear-2 (>= 1)
   int fp8;                  // operands are E4M3 bytes (128 per swizzle row) instead of bf16 (64 per row)
   int k_elems;              // K elements per pipeline stage: 64 (bf16) or 128 (E4M3)
-  int small_a;              // swapped-operand tiles load only their own (padded) rows of A, in 16-row boxes
-  int swap_prefetch;        // swapped-operand tiles ask L2 for their weight boxes this many K blocks ahead (0 = off)
+  int swap_rows;            // row blocks with at most this many rows run with swapped operands
   int withhold_ready;       // host-requested failure drill: Linear-1 never publishes its rows (one-launch runs)
   long long wait_budget;    // clocks a cross-CTA wait may last before it gives up
   int kernel_id;
@@ -139,13 +139,13 @@ __device__ __forceinline__ Tile make_tile(int phase, int e, int m_blk, int n_blk
   const PhaseDesc& d = p.ph[phase];
   Tile t;
   t.phase = phase;
-  t.row0 = p.offsets[e] + m_blk * BM;
-  t.row_end = p.offsets[e + 1];
+  t.row0 = st->offs[e] + m_blk * BM;
+  t.row_end = st->offs[e + 1];
   t.n0 = n_blk * d.out_cols_per_tile;
   t.w_row0 = e * d.N + t.n0;
   t.block = st->hot_prefix[e] + st->cold_prefix[e] + m_blk;
   const int rows = min(t.row_end - t.row0, BM);                   // rows of this block: a whole small expert, or the
-  t.n_pad = rows <= kSwapRows ? ((rows + 15) & ~15) : 0;          // short last block of a larger one: swapped operands
+  t.n_pad = rows <= p.swap_rows ? ((rows + 15) & ~15) : 0;          // short last block of a larger one: swapped operands
   return t;
 }
 
@@ -393,8 +393,7 @@ template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wg,
                   const __grid_constant__ CUtensorMap tm_wu, const __grid_constant__ CUtensorMap tm_h,
-                  const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_x16,
-                  const __grid_constant__ CUtensorMap tm_h16, const FfnParams p) {
+                  const __grid_constant__ CUtensorMap tm_wd, const FfnParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -428,10 +427,15 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   if (warp == 0) {
     // exclusive prefixes of ceil(count/128) over experts (hot and cold apart), 32 experts per step
     int32_t run_hot = 0, run_cold = 0;
+    if (lane == 0) st->offs[0] = p.offsets[0];
     for (int base = 0; base < p.E; base += 32) {
       const int e = base + lane;
       int32_t v = 0;
-      if (e < p.E) v = (p.offsets[e + 1] - p.offsets[e] + BM - 1) / BM;
+      if (e < p.E) {
+        const int32_t lo = p.offsets[e], hi = p.offsets[e + 1];
+        st->offs[e + 1] = hi;
+        v = (hi - lo + BM - 1) / BM;
+      }
       int32_t hot = v >= kHotBlocks ? v : 0;
       int32_t cold = v - hot;
 #pragma unroll
@@ -453,8 +457,6 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       ptx::prefetch_tensormap(&tm_wu);
       ptx::prefetch_tensormap(&tm_h);
       ptx::prefetch_tensormap(&tm_wd);
-      ptx::prefetch_tensormap(&tm_x16);
-      ptx::prefetch_tensormap(&tm_h16);
     }
   }
   if (warp == 1) {
@@ -484,6 +486,11 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       InterleaveCursor cursor{static_cast<int>(blockIdx.x), static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)};
       int n_drawn = 0;
       const long long t_begin = clock64();
+      // Schedule 0 draws positions from a global counter.  The round trip of that atomic would sit between two tiles
+      // with nothing new in flight, so the position of the following tile is requested a few K blocks before the
+      // current tile's loads end (kDrawAhead) and is only looked at when that tile begins.
+      constexpr int kDrawAhead = 8;
+      int pos_next = p.schedule == 0 ? atomicAdd(&p.sched[0], 1) : 0;
       while (ok) {
         if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_empty[slot]), ring_phase ^ 1u, abort_flag)) {
           report_timeout(p, 5);
@@ -491,10 +498,11 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         }
         // ---- next tile of this CTA
         int code = -1;
+        bool drawn_next = false;
         if (p.schedule == 1) {
           code = cursor.draw(tiles1, tiles2, p.ph[0].n_blocks, p.ph[1].n_blocks, p.lead_D);
         } else {
-          const int pos = atomicAdd(&p.sched[0], 1);
+          const int pos = pos_next;
           if (pos < tiles1) code = pos;
           else if (pos < tiles1 + tiles2) code = (1 << kPhaseShift) | (pos - tiles1);
         }
@@ -518,22 +526,10 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           }
           ptx::fence_proxy_async_all();   // h was written through the generic proxy, TMA reads through the async one
         }
-        // A tile with swapped operands holds n_pad <= 64 rows: it loads them as n_pad/16 boxes of 16 rows (the same
-        // swizzled layout as the first rows of a 128-row box) instead of 128 rows that are mostly other experts'.
-        const bool small_a = t.n_pad != 0 && p.small_a != 0;
-        const CUtensorMap* ma16 = t.phase == 0 ? &tm_x16 : &tm_h16;
-        const uint32_t stage_tx = small_a ? static_cast<uint32_t>(t.n_pad * 128 + 2 * kBHalfBytes) : kStageBytes;
-        // Such a tile only streams weights it uses once, and what limits it is the bytes one CTA keeps in flight: ask
-        // L2 for the weight boxes a few K blocks ahead of the ring.
-        const int ahead = t.n_pad != 0 ? p.swap_prefetch : 0;
-        for (int kb = 0; kb < ahead && kb < d.k_blocks; ++kb) {
-          ptx::tma_prefetch_l2_2d(mb0, kb * p.k_elems, t.w_row0);
-          ptx::tma_prefetch_l2_2d(mb1, kb * p.k_elems, t.w_row0 + d.b1_row_shift);
-        }
         for (int kb = 0; kb < d.k_blocks; ++kb) {
-          if (kb + ahead < d.k_blocks && ahead > 0) {
-            ptx::tma_prefetch_l2_2d(mb0, (kb + ahead) * p.k_elems, t.w_row0);
-            ptx::tma_prefetch_l2_2d(mb1, (kb + ahead) * p.k_elems, t.w_row0 + d.b1_row_shift);
+          if (p.schedule == 0 && !drawn_next && kb + kDrawAhead >= d.k_blocks) {
+            pos_next = atomicAdd(&p.sched[0], 1);
+            drawn_next = true;
           }
           if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, &w_empty)) {
             report_timeout(p, 1);
@@ -542,13 +538,8 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           }
           const uint32_t full = ptx::smem_u32(&st->full[stage]);
           const uint32_t sa = stage_u32 + stage * kStageBytes;
-          ptx::mbar_expect_tx(full, stage_tx);
-          if (small_a) {
-            for (int r16 = 0; r16 < t.n_pad; r16 += 16)
-              ptx::tma_load_2d(sa + r16 * 128, ma16, full, kb * p.k_elems, t.row0 + r16);
-          } else {
-            ptx::tma_load_2d(sa, ma, full, kb * p.k_elems, t.row0);
-          }
+          ptx::mbar_expect_tx(full, kStageBytes);
+          ptx::tma_load_2d(sa, ma, full, kb * p.k_elems, t.row0);
           ptx::tma_load_2d(sa + kABytes, mb0, full, kb * p.k_elems, t.w_row0);
           ptx::tma_load_2d(sa + kABytes + kBHalfBytes, mb1, full, kb * p.k_elems, t.w_row0 + d.b1_row_shift);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -571,8 +562,8 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       int slot = 0;
       uint32_t ring_phase = 0;
       bool ok = true;
-      long long w_full = 0, w_tmem = 0;
-      unsigned long long n_tiles = 0;
+      long long w_full = 0, w_tmem = 0, t_swapped = 0, w_swapped = 0, t_full_tiles = 0;
+      unsigned long long n_tiles = 0, n_swapped = 0;
       while (ok) {
         st->mma_idle = 1;
         if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
@@ -593,6 +584,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         st->mma_idle = 0;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN_ACC);
+        const long long t_tile = clock64(), w_full_before = w_full;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), phase, abort_flag, &w_full)) {
             report_timeout(p, 3);
@@ -638,12 +630,23 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
         ++n_tiles;
+        if (n_pad != 0) {
+          ++n_swapped;
+          t_swapped += clock64() - t_tile;
+          w_swapped += w_full - w_full_before;
+        } else {
+          t_full_tiles += clock64() - t_tile;
+        }
       }
       st->mma_idle = 1;
       if (p.trace) {
         p.trace[blockIdx.x * kMoeTraceFields + 2] = static_cast<unsigned long long>(w_full);
         p.trace[blockIdx.x * kMoeTraceFields + 3] = static_cast<unsigned long long>(w_tmem);
         p.trace[blockIdx.x * kMoeTraceFields + 6] = n_tiles;
+        p.trace[blockIdx.x * kMoeTraceFields + 8] = n_swapped;
+        p.trace[blockIdx.x * kMoeTraceFields + 9] = static_cast<unsigned long long>(t_swapped);
+        p.trace[blockIdx.x * kMoeTraceFields + 10] = static_cast<unsigned long long>(w_swapped);
+        p.trace[blockIdx.x * kMoeTraceFields + 11] = static_cast<unsigned long long>(t_full_tiles);
       }
     }
     __syncwarp();
@@ -754,6 +757,7 @@ struct PairTail {
   volatile uint32_t mma_progress;
   volatile int mma_idle;
   int32_t pair_prefix[kMaxExperts + 1];   // exclusive prefix of 256-row blocks per expert
+  int32_t offs[kMaxExperts + 1];          // the expert row offsets, copied once
 };
 constexpr size_t kPairSmemBytes = 1024 + static_cast<size_t>(kPairStages) * kPairStageBytes + sizeof(PairTail);
 
@@ -767,8 +771,8 @@ __device__ __forceinline__ Tile decode_pair_tile(int tile, int phase, uint32_t r
   const int pair_row = local - n_blk * pb;
   Tile t;
   t.phase = phase;
-  t.row0 = p.offsets[e] + pair_row * 2 * BM + static_cast<int>(rank) * BM;   // this CTA's 128 rows
-  t.row_end = p.offsets[e + 1];
+  t.row0 = st->offs[e] + pair_row * 2 * BM + static_cast<int>(rank) * BM;   // this CTA's 128 rows
+  t.row_end = st->offs[e + 1];
   t.n0 = n_blk * d.out_cols_per_tile;
   t.w_row0 = e * d.N + t.n0;
   t.block = 0;
@@ -814,7 +818,12 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     for (int base = 0; base < p.E; base += 32) {
       const int e = base + lane;
       int32_t v = 0;
-      if (e < p.E) v = (p.offsets[e + 1] - p.offsets[e] + 2 * BM - 1) / (2 * BM);
+      if (e < p.E) {
+        const int32_t lo = p.offsets[e], hi = p.offsets[e + 1];
+        st->offs[e + 1] = hi;
+        if (e == 0) st->offs[0] = lo;
+        v = (hi - lo + 2 * BM - 1) / (2 * BM);
+      }
       int32_t incl = v;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
@@ -1166,12 +1175,12 @@ cudaError_t launch_pair(moe_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b
 }  // namespace
 
 struct FfnMaps {
-  CUtensorMap x, wg, wu, h, wd, x16, h16;   // copies: the kernels take them by value
+  CUtensorMap x, wg, wu, h, wd;   // copies: the kernels take them by value
 };
 
 static void launch_single(int grid, const FfnMaps& m, const FfnParams& p, cudaStream_t stream) {
-  if (p.fp8) expert_ffn_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, m.x16, m.h16, p);
-  else expert_ffn_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, m.x16, m.h16, p);
+  if (p.fp8) expert_ffn_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, p);
+  else expert_ffn_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, p);
 }
 
 // Everything one expert-FFN call needs on the host side; fp8 selects E4M3 operands with epilogue scales.
@@ -1203,8 +1212,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     const uint64_t EF = static_cast<uint64_t>(s.E) * s.F, EH = static_cast<uint64_t>(s.E) * s.H;
     const bool ok = tensor_map_2d(ctx, c.a1, R, s.H, eb, 128, &m.x) && tensor_map_2d(ctx, c.w_gate, EF, s.H, eb, 128, &m.wg) &&
                     tensor_map_2d(ctx, c.w_up, EF, s.H, eb, 128, &m.wu) && tensor_map_2d(ctx, c.a2, R, s.F, eb, 128, &m.h) &&
-                    tensor_map_2d(ctx, c.w_down, EH, s.F, eb, 128, &m.wd) && tensor_map_2d(ctx, c.a1, R, s.H, eb, 16, &m.x16) &&
-                    tensor_map_2d(ctx, c.a2, R, s.F, eb, 16, &m.h16);
+                    tensor_map_2d(ctx, c.w_down, EH, s.F, eb, 128, &m.wd);
     if (!ok) return MOE_ERR_CUDA;
   }
 
@@ -1224,9 +1232,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   p.schedule = tn.schedule;
   p.fp8 = c.fp8;
   p.k_elems = k_elems;
-  p.small_a = moe_knob_value(ctx, "small_a", 1);
-  p.swap_prefetch = moe_knob_value(ctx, "swap_prefetch", 0);
-  if (p.swap_prefetch < 0 || p.swap_prefetch > 64) return MOE_ERR_INVALID_ARG;
+  p.swap_rows = moe_knob_value(ctx, "swap_rows", kSwapRows);
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
   // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
   p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);

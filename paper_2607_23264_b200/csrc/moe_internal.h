@@ -13,8 +13,10 @@ constexpr int kMoeKernels = 7;
 // Wait counters one CTA of a grouped GEMM records when tracing is on (SM clocks unless noted):
 // 0 producer loop span, 1 producer waited for a free stage, 2 MMA waited for data, 3 MMA waited for a free
 // accumulator (the epilogue's back-pressure), 4 epilogue waited for an accumulator, 5 epilogue drain+store span,
-// 6 tiles processed (count), 7 epilogue held by the pacing gap.
-constexpr int kMoeTraceFields = 8;
+// 6 tiles processed (count), 7 epilogue held by the pacing gap; and, by the MMA warp, per tile class: 8 tiles computed
+// with swapped operands (count), 9 their time from the first operand wait to the last MMA issued, 10 the part of it
+// spent waiting for operands, 11 the time of the other (full 128-row) tiles.
+constexpr int kMoeTraceFields = 12;
 // Tile codes (phase << 30 | index in the phase's tile list, -1 = end) a CTA logs when tracing a one-launch run.
 constexpr int kMoeOrderLogCap = 512;
 

@@ -57,7 +57,7 @@ class MxLayer:
 def out_from_gpu_codes(ws, lay, tokens, cfg, ids, w, inv_perm, oracle_weights, rows_of_tokens=None):
     """The oracle's Linear-2 and combine run on the GPU's own h codes (read from the fused call's workspace) for the
     given tokens: isolates the arithmetic after h from quantisation decisions that a last-bit difference in h flips."""
-    R, F, H, k = tokens * cfg.k if isinstance(tokens, int) else None, cfg.F, cfg.H, cfg.k
+    F, H, k = cfg.F, cfg.H, cfg.k
     toks = np.arange(tokens) if isinstance(tokens, int) else np.asarray(tokens)
     n_rows = int(inv_perm.size)
     hq = ws[lay["hq"]:lay["hq"] + n_rows * F].view(n_rows, F)
@@ -68,10 +68,13 @@ def out_from_gpu_codes(ws, lay, tokens, cfg, ids, w, inv_perm, oracle_weights, r
     w8 = sfh[:, rows_dev].cpu().numpy().view(np.uint8).reshape(F // 128, len(toks) * k, 4)
     scales = np.ascontiguousarray(w8.transpose(1, 0, 2)).reshape(len(toks), k, F // 32)
     ref = np.zeros((len(toks), H))
+    w_down = {}                                   # expert -> dequantised W_down [H, F], widened once
     for i, t in enumerate(toks):
         for j in range(k):
-            dq, ds = oracle_weights(int(ids[t, j]))[2]
-            ref[i] += w[t, j] * mx.gemm(codes[i, j:j + 1], scales[i, j:j + 1], dq, ds)[0]
+            e = int(ids[t, j])
+            if e not in w_down:
+                w_down[e] = mx.dequantize_rows(*oracle_weights(e)[2])
+            ref[i] += w[t, j] * (mx.dequantize_rows(codes[i, j:j + 1], scales[i, j:j + 1]) @ w_down[e].T)[0]
     return ref
 
 
