@@ -33,6 +33,8 @@
 // Layers whose experts hold many rows run the CTA-pair variant further down (256-row tiles, cta_group::2).
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "ffn_math.cuh"
 #include "moe_internal.h"
 #include "ptx_sm100.cuh"
@@ -47,6 +49,12 @@ constexpr int kStages = 4;
 constexpr int kABytes = BM * BK * 2;          // 16 KiB
 constexpr int kBHalfBytes = 128 * BK * 2;     // 16 KiB: one 128-row weight box
 constexpr int kStageBytes = kABytes + 2 * kBHalfBytes;   // 48 KiB
+// Wide mode (launches with many-row experts, see below): a stage holds a second 128-row A box, and three such stages
+// take the room of the four.
+constexpr int kWideStages = 3;
+constexpr int kWideStageBytes = 2 * kABytes + 2 * kBHalfBytes;   // 64 KiB
+static_assert(kWideStages * kWideStageBytes <= kStages * kStageBytes, "the wide ring must fit in the ring's shared memory");
+constexpr int kWideFlag = 1 << 16;   // in the per-tile word next to the tile code: a 256-row tile on both accumulators
 constexpr int kThreads = 192;
 constexpr int kMaxExperts = 1024;
 constexpr int kTmemCols = 512;
@@ -64,12 +72,14 @@ struct SharedTail {
   uint64_t ring_full[kRing];
   uint64_t ring_empty[kRing];
   int32_t ring_tile[kRing];
-  int32_t ring_npad[kRing];         // 0, or the padded row count of a tile computed with swapped operands
+  int32_t ring_kind[kRing];         // 0, the padded row count of a tile computed with swapped operands, or kWideFlag
   uint32_t tmem_base;
   volatile int abort_flag;
   volatile uint32_t mma_progress;   // K-blocks issued so far by the MMA warp (pacing clock)
   volatile int mma_idle;            // 1 while the MMA warp waits for an accumulator or has finished
-  int32_t hot_prefix[kMaxExperts + 1];    // exclusive prefix of 128-row blocks over hot experts (cold count 0)
+  int wide;                         // this launch cuts many-row experts into 256-row blocks (wide mode)
+  int32_t hot_prefix[kMaxExperts + 1];    // exclusive prefix of row blocks over hot experts (cold count 0): 128-row
+                                          // blocks, or 256-row blocks in wide mode
   int32_t cold_prefix[kMaxExperts + 1];   // the same over cold experts
   int32_t offs[kMaxExperts + 1];          // the expert row offsets, copied once: tile decoding reads no global memory
 };
@@ -108,6 +118,7 @@ struct FfnParams {
   int fp8;                  // operands are E4M3 bytes (128 per swizzle row) instead of bf16 (64 per row)
   int k_elems;              // K elements per pipeline stage: 64 (bf16) or 128 (E4M3)
   int swap_rows;            // row blocks with at most this many rows run with swapped operands
+  int wide_allowed;         // the launch may use wide mode (two-launch Expert-Wave runs)
   int withhold_ready;       // host-requested failure drill: Linear-1 never publishes its rows (one-launch runs)
   long long wait_budget;    // clocks a cross-CTA wait may last before it gives up
   int kernel_id;
@@ -121,6 +132,7 @@ struct Tile {
   int w_row0;    // first row of the weight box in the [E*N, K] weight matrix
   int block;     // global index of the 128-row block (ready counter)
   int n_pad;     // 0 for a 128-row tile; else operands are swapped and this is the row count padded to 16
+  int wide;      // 1: the tile covers rows row0 .. row0 + 255 on both accumulators (rows row0 + 128.. on the second)
 };
 
 // Largest e with prefix(e) <= q, prefix non-decreasing with prefix(0) = 0 and q < prefix(E).
@@ -134,18 +146,21 @@ __device__ __forceinline__ int find_expert(F prefix, int q, int E) {
   return lo;
 }
 
-__device__ __forceinline__ Tile make_tile(int phase, int e, int m_blk, int n_blk, const SharedTail* st,
+// m_blk counts the expert's row blocks in the unit of its class: 256 rows for a hot expert in wide mode, else 128.
+__device__ __forceinline__ Tile make_tile(int phase, int e, int m_blk, int n_blk, bool hot, const SharedTail* st,
                                           const FfnParams& p) {
   const PhaseDesc& d = p.ph[phase];
+  const int unit = (hot && st->wide) ? 2 * BM : BM;
   Tile t;
   t.phase = phase;
-  t.row0 = st->offs[e] + m_blk * BM;
+  t.row0 = st->offs[e] + m_blk * unit;
   t.row_end = st->offs[e + 1];
   t.n0 = n_blk * d.out_cols_per_tile;
   t.w_row0 = e * d.N + t.n0;
   t.block = st->hot_prefix[e] + st->cold_prefix[e] + m_blk;
-  const int rows = min(t.row_end - t.row0, BM);                   // rows of this block: a whole small expert, or the
-  t.n_pad = rows <= p.swap_rows ? ((rows + 15) & ~15) : 0;          // short last block of a larger one: swapped operands
+  const int rows = min(t.row_end - t.row0, unit);                 // rows of this block: a whole small expert, or the
+  t.wide = rows > BM ? 1 : 0;                                     // (short) last block of a larger one
+  t.n_pad = rows <= p.swap_rows ? ((rows + 15) & ~15) : 0;        // few rows: swapped operands
   return t;
 }
 
@@ -162,7 +177,7 @@ __device__ __forceinline__ Tile decode_tile(int code, const SharedTail* st, cons
     const int row = idx / nb;
     const int n_blk = idx - row * nb;
     const int e = find_expert([&](int i) { return st->hot_prefix[i] + st->cold_prefix[i]; }, row, p.E);
-    return make_tile(phase, e, row - (st->hot_prefix[e] + st->cold_prefix[e]), n_blk, st, p);
+    return make_tile(phase, e, row - (st->hot_prefix[e] + st->cold_prefix[e]), n_blk, false, st, p);   // never wide
   }
   const long long hot_tiles = static_cast<long long>(st->hot_prefix[p.E]) * nb;
   const long long cold_tiles = static_cast<long long>(st->cold_prefix[p.E]) * nb;
@@ -175,7 +190,7 @@ __device__ __forceinline__ Tile decode_tile(int code, const SharedTail* st, cons
   const int mb = prefix[e + 1] - prefix[e];
   const int local = tile - nb * prefix[e];
   const int n_blk = local / mb;
-  return make_tile(phase, e, local - n_blk * mb, n_blk, st, p);
+  return make_tile(phase, e, local - n_blk * mb, n_blk, !is_cold, st, p);
 }
 
 // Schedule 1 (the paper's Algorithm 1): a CTA owns every stride-th tile of each GEMM's row-major tile list and keeps
@@ -389,6 +404,29 @@ __device__ __forceinline__ void drain_swapped(const Tile& t, const FfnParams& p,
   }
 }
 
+// The eight MMAs of one K block of a swapped-operand tile: weight box 0 into columns 0.., weight box 1 into columns
+// 128.., N = kRows (the tile's rows padded to 16).  kRows is a template parameter because the instruction descriptor
+// must be a compile-time constant: with the descriptor in an ordinary register each of these short instructions took
+// about 100 clocks to issue, twice what the tensor pipe needs for them (measured with a stand-alone loop: 58 against
+// 95 to 190 clocks per instruction).
+template <bool kFp8, int kRows>
+__device__ __forceinline__ void issue_swapped(uint32_t d_tmem, uint64_t w0_desc, uint64_t w1_desc, uint64_t rows_desc,
+                                              uint32_t accumulate_first) {
+  constexpr uint32_t idesc = kFp8 ? ptx::idesc_e4m3_f32(BM, kRows) : ptx::idesc_bf16_f32(BM, kRows);
+#pragma unroll
+  for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
+    const uint64_t adv = static_cast<uint64_t>(2 * k4);
+    const uint32_t accum = k4 != 0 ? 1u : accumulate_first;
+    if constexpr (kFp8) {
+      ptx::tc_mma_e4m3(d_tmem, w0_desc + adv, rows_desc + adv, idesc, accum);
+      ptx::tc_mma_e4m3(d_tmem + 128u, w1_desc + adv, rows_desc + adv, idesc, accum);
+    } else {
+      ptx::tc_mma_bf16(d_tmem, w0_desc + adv, rows_desc + adv, idesc, accum);
+      ptx::tc_mma_bf16(d_tmem + 128u, w1_desc + adv, rows_desc + adv, idesc, accum);
+    }
+  }
+}
+
 template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wg,
@@ -425,19 +463,38 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     ptx::fence_proxy_async_smem();
   }
   if (warp == 0) {
-    // exclusive prefixes of ceil(count/128) over experts (hot and cold apart), 32 experts per step
+    // Wide mode is chosen per launch, by every CTA alike, from the expert row counts.  An expert with several 128-row
+    // blocks is then cut into 256-row blocks, each one tile on both accumulators: its two halves
+    // share the weight boxes of a stage, a third less to bring into shared memory per flop, which is what holds
+    // these tiles back when the weights of many experts stream through L2 at once.
+    // The price is one stage of the ring (three stages of 64 KiB), which the one-block tiles of small experts feel
+    // (they stream weights and live on the bytes in flight), so wide mode needs them to be few: at most a fifth of
+    // the launch's tiles.
+    int hot_wide_blocks = 0, cold_blocks = 0;
+    for (int base = 0; base < p.E; base += 32) {
+      const int e = base + lane;
+      const int rows = e < p.E ? p.offsets[e + 1] - p.offsets[e] : 0;
+      if (rows > BM * (kHotBlocks - 1)) hot_wide_blocks += (rows + 2 * BM - 1) / (2 * BM);
+      else if (rows > 0) cold_blocks += 1;
+    }
+    hot_wide_blocks = __reduce_add_sync(0xFFFFFFFFu, hot_wide_blocks);
+    cold_blocks = __reduce_add_sync(0xFFFFFFFFu, cold_blocks);
+    const bool wide_mode = p.wide_allowed != 0 && hot_wide_blocks > 0 && (4 * cold_blocks <= hot_wide_blocks || p.wide_allowed == 2);
+    if (lane == 0) st->wide = wide_mode ? 1 : 0;
+    // exclusive prefixes of the row-block counts over experts (hot and cold apart), 32 experts per step
     int32_t run_hot = 0, run_cold = 0;
     if (lane == 0) st->offs[0] = p.offsets[0];
     for (int base = 0; base < p.E; base += 32) {
       const int e = base + lane;
-      int32_t v = 0;
+      int32_t v = 0, rows = 0;
       if (e < p.E) {
         const int32_t lo = p.offsets[e], hi = p.offsets[e + 1];
         st->offs[e + 1] = hi;
-        v = (hi - lo + BM - 1) / BM;
+        rows = hi - lo;
+        v = (rows + BM - 1) / BM;
       }
-      int32_t hot = v >= kHotBlocks ? v : 0;
-      int32_t cold = v - hot;
+      int32_t hot = v >= kHotBlocks ? (wide_mode ? (rows + 2 * BM - 1) / (2 * BM) : v) : 0;
+      int32_t cold = v >= kHotBlocks ? 0 : v;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
         const int32_t oh = __shfl_up_sync(0xFFFFFFFFu, hot, off);
@@ -468,6 +525,11 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   ptx::tc_fence_after_sync();
 
   const uint32_t tmem_base = st->tmem_base;
+  // ring geometry of this launch: [A][B0][B1] x 4 stages, or in wide mode [A][A'][B0][B1] x 3 stages
+  const bool wide_mode = st->wide != 0;
+  const int n_stages = wide_mode ? kWideStages : kStages;
+  const uint32_t stage_bytes = wide_mode ? kWideStageBytes : kStageBytes;
+  const uint32_t b_off = wide_mode ? 2 * kABytes : kABytes;       // offset of the first weight box inside a stage
   const int total_blocks = st->hot_prefix[p.E] + st->cold_prefix[p.E];
   const int tiles1 = p.phase_lo == 0 ? total_blocks * p.ph[0].n_blocks : 0;   // Linear-1 tiles of this launch
   const int tiles2 = p.phase_hi == 2 ? total_blocks * p.ph[1].n_blocks : 0;   // Linear-2 tiles of this launch
@@ -510,7 +572,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         Tile t{};
         if (code >= 0) t = decode_tile(code, st, p);
         st->ring_tile[slot] = code;
-        st->ring_npad[slot] = t.n_pad;
+        st->ring_kind[slot] = t.wide ? kWideFlag : t.n_pad;
         ptx::mbar_arrive(ptx::smem_u32(&st->ring_full[slot]));
         if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
         if (code < 0) break;
@@ -537,12 +599,13 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             break;
           }
           const uint32_t full = ptx::smem_u32(&st->full[stage]);
-          const uint32_t sa = stage_u32 + stage * kStageBytes;
-          ptx::mbar_expect_tx(full, kStageBytes);
+          const uint32_t sa = stage_u32 + stage * stage_bytes;
+          ptx::mbar_expect_tx(full, t.wide ? kWideStageBytes : kStageBytes);
           ptx::tma_load_2d(sa, ma, full, kb * p.k_elems, t.row0);
-          ptx::tma_load_2d(sa + kABytes, mb0, full, kb * p.k_elems, t.w_row0);
-          ptx::tma_load_2d(sa + kABytes + kBHalfBytes, mb1, full, kb * p.k_elems, t.w_row0 + d.b1_row_shift);
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (t.wide) ptx::tma_load_2d(sa + kABytes, ma, full, kb * p.k_elems, t.row0 + BM);
+          ptx::tma_load_2d(sa + b_off, mb0, full, kb * p.k_elems, t.w_row0);
+          ptx::tma_load_2d(sa + b_off + kBHalfBytes, mb1, full, kb * p.k_elems, t.w_row0 + d.b1_row_shift);
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
         }
       }
       if (p.trace) {
@@ -553,17 +616,122 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = kFp8 ? ptx::idesc_e4m3_f32(BM, BN_ACC) : ptx::idesc_bf16_f32(BM, BN_ACC);
       int stage = 0;
       uint32_t phase = 0;
-      int acc = 0;
-      uint32_t acc_phase = 0;
+      int acc = 0;                    // accumulator of the next one-accumulator tile
+      uint32_t acc_uses[2] = {0, 0};  // tiles that have used each accumulator so far (the barriers' phases)
       uint32_t progress = 0;
       int slot = 0;
       uint32_t ring_phase = 0;
       bool ok = true;
       long long w_full = 0, w_tmem = 0, t_swapped = 0, w_swapped = 0, t_full_tiles = 0;
       unsigned long long n_tiles = 0, n_swapped = 0;
+
+      // One K block: wait for the stage, issue its MMAs, release the stage.  `issue` gets the stage's address.
+      auto k_block = [&](auto&& issue) -> bool {
+        if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), phase, abort_flag, &w_full)) {
+          report_timeout(p, 3);
+          return false;
+        }
+        ptx::tc_fence_after_sync();
+        issue(stage_u32 + stage * stage_bytes);
+        ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // stage is free once these MMAs have read it
+        st->mma_progress = ++progress;
+        if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+        return true;
+      };
+      // The K loop of one tile, one instantiation per tile kind: a run-time branch between the MMAs of a K block costs
+      // 100 to 200 clocks per block (measured with a stand-alone issue loop: a never-taken branch around four dependent
+      // N = 16 instructions takes them from 65 to 115 clocks each), which is nothing next to four 128-clock instructions
+      // but doubles the time of a swapped-operand tile.  kKind: 0 = 128 rows on accumulator `acc`; -1 = 256 rows on
+      // both accumulators; otherwise the padded row count of a swapped-operand tile.
+      auto run_tile = [&](auto kind_tag, int k_blocks, uint32_t d_tmem) -> bool {
+        constexpr int kKind = decltype(kind_tag)::value;
+        constexpr uint32_t idesc = kFp8 ? ptx::idesc_e4m3_f32(BM, BN_ACC) : ptx::idesc_bf16_f32(BM, BN_ACC);
+        auto mma = [](uint32_t d, uint64_t a, uint64_t b, uint32_t accumulate) {
+          if constexpr (kFp8) ptx::tc_mma_e4m3(d, a, b, idesc, accumulate);
+          else ptx::tc_mma_bf16(d, a, b, idesc, accumulate);
+        };
+        if constexpr (kKind == 0) {
+          for (int kb = 0; kb < k_blocks; ++kb) {
+            const uint32_t later = kb != 0 ? 1u : 0u;
+            if (!k_block([&](uint32_t sa) {
+                  const uint64_t a_desc = ptx::smem_desc_sw128(sa), b_desc = ptx::smem_desc_sw128(sa + b_off);
+                  // +32 bytes along K inside the swizzle row = +2 in the descriptor's 16-byte address units
+                  // (16 bf16 or 32 E4M3 elements per instruction: 32 bytes either way)
+#pragma unroll
+                  for (int k4 = 0; k4 < BK / UMMA_K; ++k4) mma(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, k4 != 0 ? 1u : later);
+                }))
+              return false;
+          }
+        } else if constexpr (kKind == -1) {
+          // rows 0..127 into accumulator 0, rows 128..255 (the second A box) into accumulator 1, same weight boxes.
+          // The first K block is peeled: accumulator 1 may still be draining (the previous tile's epilogue) while
+          // the first MMAs into accumulator 0 run.
+          auto half = [&](uint32_t sa, uint32_t a_off, uint32_t d, uint32_t later) {
+            const uint64_t a_desc = ptx::smem_desc_sw128(sa + a_off), b_desc = ptx::smem_desc_sw128(sa + b_off);
+#pragma unroll
+            for (int k4 = 0; k4 < BK / UMMA_K; ++k4) mma(d, a_desc + 2 * k4, b_desc + 2 * k4, k4 != 0 ? 1u : later);
+          };
+          bool acc1_ok = true;
+          if (!k_block([&](uint32_t sa) {
+                half(sa, 0, tmem_base, 0u);
+                st->mma_idle = 1;   // (a paced epilogue must not hold its stores for an MMA warp that waits for it)
+                acc1_ok = ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[1]), (acc_uses[1] & 1u) ^ 1u, abort_flag, &w_tmem);
+                st->mma_idle = 0;
+                ptx::tc_fence_after_sync();
+                if (acc1_ok) half(sa, kABytes, tmem_base + BN_ACC, 0u);
+              }))
+            return false;
+          if (!acc1_ok) {
+            report_timeout(p, 2);
+            return false;
+          }
+          for (int kb = 1; kb < k_blocks; ++kb) {
+            if (!k_block([&](uint32_t sa) {
+                  half(sa, 0, tmem_base, 1u);
+                  half(sa, kABytes, tmem_base + BN_ACC, 1u);
+                }))
+              return false;
+          }
+        } else {
+          // swapped operands: each 128-row weight box is the M side, the expert's rows (the A box) the N side; the
+          // first weight box accumulates into columns 0.., the second into columns 128..
+          auto issue = [&](uint32_t sa, uint32_t later) {
+            issue_swapped<kFp8, kKind>(d_tmem, ptx::smem_desc_sw128(sa + b_off),
+                                       ptx::smem_desc_sw128(sa + b_off + kBHalfBytes), ptx::smem_desc_sw128(sa), later);
+          };
+          // Two K blocks per wait: the sixteen short MMAs of two stages are issued without a branch between them (the
+          // bubble a branch opens in the issue stream costs as much as three of these instructions; with one wait per
+          // two blocks the stand-alone loop goes from 723 to 588 clocks per block).
+          int kb = 0;
+          for (; n_stages == kStages && kb + 2 <= k_blocks; kb += 2) {   // (the three-stage ring cannot spare two stages)
+            const int s0 = stage, s1 = stage + 1 == n_stages ? 0 : stage + 1;
+            const uint32_t ph1 = s1 == 0 ? phase ^ 1u : phase;
+            const uint32_t bar0 = ptx::smem_u32(&st->full[s0]), bar1 = ptx::smem_u32(&st->full[s1]);
+            if (!(ptx::mbar_try_wait(bar0, phase) & ptx::mbar_try_wait(bar1, ph1))) {
+              if (!ptx::mbar_wait_timed(bar0, phase, abort_flag, &w_full) || !ptx::mbar_wait_timed(bar1, ph1, abort_flag, &w_full)) {
+                report_timeout(p, 3);
+                return false;
+              }
+            }
+            ptx::tc_fence_after_sync();
+            issue(stage_u32 + s0 * stage_bytes, kb != 0 ? 1u : 0u);
+            ptx::tc_commit(ptx::smem_u32(&st->empty[s0]));
+            issue(stage_u32 + s1 * stage_bytes, 1u);
+            ptx::tc_commit(ptx::smem_u32(&st->empty[s1]));
+            progress += 2;
+            st->mma_progress = progress;
+            stage = s1 + 1 == n_stages ? 0 : s1 + 1;
+            phase = stage == 0 ? ph1 ^ 1u : ph1;
+          }
+          for (; kb < k_blocks; ++kb) {
+            if (!k_block([&](uint32_t sa) { issue(sa, kb != 0 ? 1u : 0u); })) return false;
+          }
+        }
+        return true;
+      };
+
       while (ok) {
         st->mma_idle = 1;
         if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
@@ -571,13 +739,17 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           break;
         }
         const int code = st->ring_tile[slot];
-        const int n_pad = st->ring_npad[slot];
+        const int kind = st->ring_kind[slot];
         ptx::mbar_arrive(ptx::smem_u32(&st->ring_empty[slot]));
         if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
         if (code < 0) break;
+        const bool wide = kind == kWideFlag;
+        const int n_pad = wide ? 0 : kind;
         const int k_blocks = p.ph[code >> kPhaseShift].k_blocks;
-        const uint32_t idesc_swap = kFp8 ? ptx::idesc_e4m3_f32(BM, n_pad) : ptx::idesc_bf16_f32(BM, n_pad);
-        if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, &w_tmem)) {
+        // a wide tile takes both accumulators, first rows on accumulator 0; the tile after it starts on 0 again,
+        // the one the epilogue hands back first
+        if (wide) acc = 0;
+        if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[acc]), (acc_uses[acc] & 1u) ^ 1u, abort_flag, &w_tmem)) {
           report_timeout(p, 2);
           break;
         }
@@ -585,50 +757,33 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN_ACC);
         const long long t_tile = clock64(), w_full_before = w_full;
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), phase, abort_flag, &w_full)) {
-            report_timeout(p, 3);
-            ok = false;
-            break;
+        if (wide) {
+          ok = run_tile(std::integral_constant<int, -1>{}, k_blocks, d_tmem);
+        } else {
+          switch (n_pad >> 4) {
+            case 0: ok = run_tile(std::integral_constant<int, 0>{}, k_blocks, d_tmem); break;
+            case 1: ok = run_tile(std::integral_constant<int, 16>{}, k_blocks, d_tmem); break;
+            case 2: ok = run_tile(std::integral_constant<int, 32>{}, k_blocks, d_tmem); break;
+            case 3: ok = run_tile(std::integral_constant<int, 48>{}, k_blocks, d_tmem); break;
+            case 4: ok = run_tile(std::integral_constant<int, 64>{}, k_blocks, d_tmem); break;
+            case 5: ok = run_tile(std::integral_constant<int, 80>{}, k_blocks, d_tmem); break;
+            case 6: ok = run_tile(std::integral_constant<int, 96>{}, k_blocks, d_tmem); break;
+            case 7: ok = run_tile(std::integral_constant<int, 112>{}, k_blocks, d_tmem); break;
+            default: ok = run_tile(std::integral_constant<int, 128>{}, k_blocks, d_tmem); break;
           }
-          ptx::tc_fence_after_sync();
-          const uint32_t sa = stage_u32 + stage * kStageBytes;
-          const uint64_t a_desc = ptx::smem_desc_sw128(sa);
-          const uint64_t b_desc = ptx::smem_desc_sw128(sa + kABytes);
-          if (n_pad == 0) {
-#pragma unroll
-            for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
-              // +32 bytes along K inside the swizzle row = +2 in the descriptor's 16-byte address units
-              // (16 bf16 or 32 E4M3 elements per instruction: 32 bytes either way)
-              const uint64_t adv = static_cast<uint64_t>(2 * k4);
-              if constexpr (kFp8) ptx::tc_mma_e4m3(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
-              else ptx::tc_mma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, (kb | k4) != 0 ? 1u : 0u);
-            }
-          } else {
-            // swapped operands: each 128-row weight box is the M side, the expert's rows (first box) the N side;
-            // the first weight box accumulates into columns 0.., the second into columns 128..
-            const uint64_t w1_desc = ptx::smem_desc_sw128(sa + kABytes + kBHalfBytes);
-#pragma unroll
-            for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
-              const uint64_t adv = static_cast<uint64_t>(2 * k4);
-              const uint32_t accum = (kb | k4) != 0 ? 1u : 0u;
-              if constexpr (kFp8) {
-                ptx::tc_mma_e4m3(d_tmem, b_desc + adv, a_desc + adv, idesc_swap, accum);
-                ptx::tc_mma_e4m3(d_tmem + 128u, w1_desc + adv, a_desc + adv, idesc_swap, accum);
-              } else {
-                ptx::tc_mma_bf16(d_tmem, b_desc + adv, a_desc + adv, idesc_swap, accum);
-                ptx::tc_mma_bf16(d_tmem + 128u, w1_desc + adv, a_desc + adv, idesc_swap, accum);
-              }
-            }
-          }
-          ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // stage is free once these MMAs have read it
-          st->mma_progress = ++progress;
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        ptx::tc_commit(ptx::smem_u32(&st->tmem_full[acc]));    // accumulator complete
-        acc ^= 1;
-        if (acc == 0) acc_phase ^= 1u;
+        if (wide) {
+          ptx::tc_commit(ptx::smem_u32(&st->tmem_full[0]));    // both accumulators complete
+          ptx::tc_commit(ptx::smem_u32(&st->tmem_full[1]));
+          ++acc_uses[0];
+          ++acc_uses[1];
+          acc = 0;
+        } else {
+          ptx::tc_commit(ptx::smem_u32(&st->tmem_full[acc]));  // accumulator complete
+          ++acc_uses[acc];
+          acc ^= 1;
+        }
         ++n_tiles;
         if (n_pad != 0) {
           ++n_swapped;
@@ -654,13 +809,14 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     // ------------------------------------------------------------------ epilogue (4 warps = 128 rows)
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const int r_in_tile = quarter * 32 + lane;
-    int acc = 0;
-    uint32_t acc_phase = 0;
+    int acc = 0;                    // accumulator of the next one-accumulator tile (the MMA warp counts the same way)
+    uint32_t acc_uses[2] = {0, 0};
     int slot = 0;
     uint32_t ring_phase = 0;
     long long w_acc = 0, busy = 0;
     Pacer pacer{ptx::smem_u32(const_cast<uint32_t*>(&st->mma_progress)), ptx::smem_u32(const_cast<int*>(&st->mma_idle)), 0, 0u, 0};
-    while (true) {
+    bool ok = true;
+    while (ok) {
       if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
         if (lane == 0) report_timeout(p, 7);
         break;
@@ -670,37 +826,45 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&st->ring_empty[slot]));
       if (++slot == kRing) { slot = 0; ring_phase ^= 1u; }
       if (code < 0) break;
-      const Tile t = decode_tile(code, st, p);
-      if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, &w_acc)) {
-        if (lane == 0) report_timeout(p, 4);
-        break;
+      Tile t = decode_tile(code, st, p);
+      // a wide tile is drained as two 128-row parts, accumulator 0 then accumulator 1
+      const int parts = t.wide ? 2 : 1;
+      if (t.wide) acc = 0;
+      for (int part = 0; part < parts; ++part) {
+        if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_full[acc]), acc_uses[acc] & 1u, abort_flag, &w_acc)) {
+          if (lane == 0) report_timeout(p, 4);
+          ok = false;
+          break;
+        }
+        ptx::tc_fence_after_sync();
+        const long long t_store = clock64();
+        const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                static_cast<uint32_t>(acc * BN_ACC);
+        if (t.n_pad != 0) {
+          if (t.phase == 0) drain_swapped<true, kFp8>(t, p, t_addr, r_in_tile);
+          else drain_swapped<false, kFp8>(t, p, t_addr, r_in_tile);
+        } else if (t.phase == 0) {
+          drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
+        } else {
+          drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
+        }
+        ptx::tc_fence_before_sync();
+        if (chained && t.phase == 0) {
+          // publish this warp's 32 rows x 128 columns of h to the Linear-2 tiles of the block
+          __threadfence();
+          ptx::fence_proxy_async_all();
+        }
+        __syncwarp();
+        if (lane == 0) {
+          ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
+          if (chained && t.phase == 0 && !p.withhold_ready) atomicAdd(&p.ready[t.block], 1);
+        }
+        busy += clock64() - t_store;
+        ++acc_uses[acc];
+        acc ^= 1;
+        t.row0 += BM;               // the second part of a wide tile
       }
-      ptx::tc_fence_after_sync();
-      const long long t_store = clock64();
-      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                              static_cast<uint32_t>(acc * BN_ACC);
-      if (t.n_pad != 0) {
-        if (t.phase == 0) drain_swapped<true, kFp8>(t, p, t_addr, r_in_tile);
-        else drain_swapped<false, kFp8>(t, p, t_addr, r_in_tile);
-      } else if (t.phase == 0) {
-        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
-      } else {
-        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
-      }
-      ptx::tc_fence_before_sync();
-      if (chained && t.phase == 0) {
-        // publish this warp's 32 rows x 128 columns of h to the Linear-2 tiles of the block
-        __threadfence();
-        ptx::fence_proxy_async_all();
-      }
-      __syncwarp();
-      if (lane == 0) {
-        ptx::mbar_arrive(ptx::smem_u32(&st->tmem_empty[acc]));
-        if (chained && t.phase == 0 && !p.withhold_ready) atomicAdd(&p.ready[t.block], 1);
-      }
-      busy += clock64() - t_store;
-      acc ^= 1;
-      if (acc == 0) acc_phase ^= 1u;
+      if (t.wide) acc = 0;
     }
     if (p.trace && warp == 2 && lane == 0) {
       p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
@@ -1267,6 +1431,8 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     ctx->last_launches += 1;
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
   }
+  // two separate launches: many-row experts may run as 256-row tiles (decided in the kernel from the row counts)
+  p.wide_allowed = moe_knob_value(ctx, "wide_tiles", 1);   // 0 never, 1 by the kernel's rule, 2 whenever an expert has several blocks
   if (!second_phase_only) {
     p.phase_lo = 0;
     p.phase_hi = 1;
