@@ -624,6 +624,16 @@ def main():
         dist.destroy_process_group()
 
 
+def preheat(step, seconds):
+    """Back-to-back untimed steps for `seconds`, until the power cap has settled the clocks."""
+    import torch
+    t0 = time.time()
+    while time.time() - t0 < seconds:
+        for _ in range(10):
+            step()
+        torch.cuda.synchronize()
+
+
 def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
     """The FP8 (E4M3, W8A8) variant: same layer, same algorithmic flops, experts in E4M3 with row scales."""
     import torch
@@ -641,17 +651,18 @@ def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
     tn = binding.make_tuning(args.burst, args.mode, args.ik, debug_flags={"auto": 0, "on": 8, "off": 16}[args.pairs])
     step = lambda: ctx.moe_fused_forward_fp8(x, d_logits, *wq, out, ws, tuning=tn)
     sampler = ClockSampler(torch.cuda.current_device())
+    burst_ms = timed(step, args.steps, args.warmup) / args.steps
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
-    ms = timed(step, args.steps, args.warmup) / args.steps
-    clocks = sampler.stop() if rank == 0 else None
+    preheat(step, args.heat_seconds)
+    ms = timed(step, args.steps, 0) / args.steps
     ctx.moe_set_kernel_timing(True)
     per = []
     for _ in range(args.steps):
         step()
         per.append(ctx.moe_get_kernel_times())
     ctx.moe_set_kernel_timing(False)
+    clocks = sampler.stop() if rank == 0 else None
     km = [float(np.mean([p[i] for p in per])) for i in range(len(binding.KERNEL_NAMES))]
     waits = None
     if args.trace:
@@ -682,6 +693,7 @@ def run_fp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
     line = {
         "metric": "fused MoE fwd tokens/s", "variant": "fp8 (E4M3 W8A8, per-row scales)", "value": cfg.T * world / (ms * 1e-3),
         "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "burst_ms_per_step": burst_ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3", "data": "synthetic",
         "config": workload_config(cfg, world), "tflops": tflops, "frac_fp8_peak": tflops / world / peak,
         "kernels_ms": {"routing": km[0] + km[1] + km[2], "quantize_x+dispatch": km[3], "linear1": km[4],
@@ -710,17 +722,18 @@ def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
     ws = torch.empty(ctx.workspace_layout_mx()["total"], dtype=torch.uint8, device=dev)
     step = lambda: ctx.moe_fused_forward_mx(x, d_logits, *wq, out, ws)
     sampler = ClockSampler(torch.cuda.current_device())
+    burst_ms = timed(step, args.steps, args.warmup) / args.steps
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
-    ms = timed(step, args.steps, args.warmup) / args.steps
-    clocks = sampler.stop() if rank == 0 else None
+    preheat(step, args.heat_seconds)
+    ms = timed(step, args.steps, 0) / args.steps
     ctx.moe_set_kernel_timing(True)
     per = []
     for _ in range(args.steps):
         step()
         per.append(ctx.moe_get_kernel_times())
     ctx.moe_set_kernel_timing(False)
+    clocks = sampler.stop() if rank == 0 else None
     km = [float(np.mean([p[i] for p in per])) for i in range(len(binding.KERNEL_NAMES))]
     # the GEMMs' own wait counters (recorded while per-kernel timing is on), averaged over CTAs, as shares of the span
     tr = ctx.moe_get_ffn_trace().astype(np.float64)
@@ -746,6 +759,7 @@ def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         "metric": "fused MoE fwd tokens/s", "variant": "mxfp8 (E4M3 elements, E8M0 scale per 32 along K)",
         "value": cfg.T * world / (ms * 1e-3),
         "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "burst_ms_per_step": burst_ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "mxfp8_e4m3", "data": "synthetic",
         "config": workload_config(cfg, world), "tflops": tflops, "frac_fp8_peak": tflops / world / peak,
         "kernels_ms": {"routing": km[0] + km[1] + km[2], "quantize_x+dispatch": km[3], "linear1+quantize_h": km[4],

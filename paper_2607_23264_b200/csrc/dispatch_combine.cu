@@ -175,7 +175,7 @@ cudaError_t launch_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_
   const long long items = static_cast<long long>(s.T) * blocks_per_row;
   const int warps_per_block = kThreads / 32;
   long long blocks = (items + warps_per_block - 1) / warps_per_block;
-  const long long cap = static_cast<long long>(ctx->num_sms) * moe_knob_value(ctx, "combine_ctas_per_sm", 6);
+  const long long cap = static_cast<long long>(ctx->num_sms) * moe_knob_value(ctx, "combine_ctas_per_sm", 3);
   if (blocks > cap && cap > 0) blocks = cap;
   using kernel_t = void (*)(const uint4*, const int32_t*, const float*, uint4*, int, int, int, int);
   static const kernel_t table[3][4] = {

@@ -86,6 +86,23 @@ def test_c2_mixtral_like_sampled():
     assert c.min() > 0.8 * cfg.R / cfg.E and c.max() < 1.2 * cfg.R / cfg.E, "near-uniform expert loads"
 
 
+def test_c2_layer_at_2048_tokens_runs_256_row_tiles():
+    """The Mixtral-like layer at a serving batch of 2048 tokens: about 512 rows per expert, too few for CTA pairs, so
+    the single-CTA kernel runs it and cuts every expert into 256-row tiles on both accumulators (the rows sampled in
+    every 128-row block fall into both halves of every such tile)."""
+    import dataclasses
+    cfg = dataclasses.replace(gen.CONFIGS["C2"], name="C2@T=2048", T=2048)
+    L, plan = run_sampled(cfg, n_random=16)
+    c = plan["counts"]
+    assert c.min() > 256 and c.max() < 1024, "several 128-row blocks per expert, fewer than the CTA-pair threshold"
+    L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, L.nan_bf16(cfg.T, cfg.H),
+                            torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV),
+                            tuning=binding.make_tuning(debug_flags=1))
+    tr = L.ctx.moe_get_ffn_trace()
+    wide_blocks = int(((c + 255) // 256).sum())
+    assert tr[0, :, 6].sum() == wide_blocks * (cfg.F // 128), "Linear-1 ran one tile per 256-row block and column tile"
+
+
 def test_c3_deepseek_like_sampled():
     cfg = gen.CONFIGS["C3"]
     _, plan = run_sampled(cfg, n_random=16)
