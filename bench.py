@@ -86,7 +86,7 @@ class ClockSampler:
                 self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, power, reasons = [], [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for line in self.tmp.read().splitlines():
             parts = [p.strip() for p in line.split(",")]
@@ -95,6 +95,7 @@ class ClockSampler:
             try:
                 sm.append(float(parts[0]))
                 mx.append(float(parts[1]))
+                power.append(float(parts[2]))
             except ValueError:
                 continue
             for name, val in zip(names, parts[3:7]):
@@ -104,7 +105,8 @@ class ClockSampler:
         os.unlink(self.tmp.name)
         busy = [v for v in sm if v > 0]
         return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm),
+                "power_w_median": statistics.median(power) if power else None, "power_w_max": max(power) if power else None}
 
 
 def oracle_threads() -> int:

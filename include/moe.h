@@ -34,8 +34,9 @@ typedef enum {
   MOE_ERR_INVALID_ARG = 1,         /* null pointer, misaligned pointer, wrong device, bad tuning value */
   MOE_ERR_UNSUPPORTED_SHAPE = 2,   /* H or F not a multiple of 64, k or E out of range, T < 0 */
   MOE_ERR_WORKSPACE_TOO_SMALL = 3,
-  MOE_ERR_BAD_ROUTING = 4,         /* device status only: an expert id given to moe_plan_routing_from_topk is
-                                      outside [0, E) */
+  MOE_ERR_BAD_ROUTING = 4,         /* device status: an expert id given to moe_plan_routing_from_topk is outside
+                                      [0, E); returned by a call only from the debug check of the logits
+                                      (MOE_TUNING entry x.check_logits=1: non-finite logits, tested on the host) */
   MOE_ERR_CUDA = 5,                /* a CUDA runtime or driver call failed */
   MOE_ERR_TIMEOUT = 6,             /* device status only: a bounded on-device wait expired */
   MOE_ERR_UNSUPPORTED = 7,         /* ep_size != 1, unknown schedule */
@@ -152,7 +153,10 @@ moe_status moe_get_workspace_layout(const moe_shape* shape, moe_workspace_layout
  * slots s' < s with the same expert).  perm[row] = s, inv_perm[s] = row.
  *   logits [T,E] fp32 (finite)  ->  topk_ids [T,k] int32, topk_w [T,k] fp32, counts [E] int32,
  *   offsets [E+1] int32, perm [R] int32, inv_perm [R] int32.
- * T == 0 writes zero counts/offsets and launches nothing else.
+ * T == 0 writes zero counts/offsets and launches nothing else.  Infinite or NaN logits violate the contract and are
+ * not tested on the device; a context created with the MOE_TUNING entry x.check_logits=1 (a debug aid: it copies the
+ * logits to the host and synchronises the stream in every call that takes logits) returns MOE_ERR_BAD_ROUTING for them
+ * before anything is launched.
  */
 moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids, float* topk_w,
                             int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,

@@ -79,6 +79,31 @@ moe_status parse_tuning_text(const char* text, moe_tuning* t, int* named_field, 
   return *named_field ? check_tuning(t) : MOE_OK;
 }
 
+// Debug aid (development knob x.check_logits=1): copy the logits to the host, wait, and refuse non-finite values,
+// which the top-k contract excludes and the kernels do not test.  Synchronises the stream; not for timed runs.
+moe_status check_logits_on_host(const moe_ctx* ctx, const float* logits, cudaStream_t cs) {
+  if (moe_knob_value(ctx, "check_logits", 0) == 0) return MOE_OK;
+  const size_t n = static_cast<size_t>(ctx->shape.T) * ctx->shape.E;
+  float* host = static_cast<float*>(std::malloc(n * sizeof(float)));
+  if (!host) return MOE_ERR_CUDA;
+  moe_status st = MOE_OK;
+  if (cudaMemcpyAsync(host, logits, n * sizeof(float), cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaStreamSynchronize(cs) != cudaSuccess) {
+    st = MOE_ERR_CUDA;
+  } else {
+    for (size_t i = 0; i < n; ++i) {
+      uint32_t bits;
+      std::memcpy(&bits, host + i, 4);
+      if ((bits & 0x7F800000u) == 0x7F800000u) {   // exponent all ones: infinity or NaN
+        st = MOE_ERR_BAD_ROUTING;
+        break;
+      }
+    }
+  }
+  std::free(host);
+  return st;
+}
+
 moe_status check_ctx(const moe_ctx* ctx) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   int dev = -1;
@@ -295,6 +320,8 @@ moe_status moe_plan_routing(moe_ctx* ctx, const float* logits, int32_t* topk_ids
   if (!aligned16(logits) || !aligned16(topk_ids) || !aligned16(topk_w) || !aligned16(counts) ||
       !aligned16(offsets) || !aligned16(perm) || !aligned16(inv_perm))
     return MOE_ERR_INVALID_ARG;
+  st = check_logits_on_host(ctx, logits, cs);
+  if (st != MOE_OK) return st;
   return moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) == cudaSuccess
              ? MOE_OK
              : MOE_ERR_CUDA;
@@ -395,6 +422,8 @@ moe_status moe_fused_forward(moe_ctx* ctx, const void* x, const float* logits, c
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
   begin_call(ctx, 0, stream);
+  st = check_logits_on_host(ctx, logits, cs);
+  if (st != MOE_OK) return st;
   if (moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
     return MOE_ERR_CUDA;
   if (moe::launch_dispatch(ctx, x, inv_perm, x_perm, cs) != cudaSuccess) return MOE_ERR_CUDA;
@@ -611,6 +640,8 @@ moe_status moe_fused_forward_fp8(moe_ctx* ctx, const void* x, const float* logit
   int32_t* inv_perm = reinterpret_cast<int32_t*>(ws + L.inv_perm);
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   begin_call(ctx, 0, stream);
+  st = check_logits_on_host(ctx, logits, cs);
+  if (st != MOE_OK) return st;
   if (moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
     return MOE_ERR_CUDA;
   if (moe::launch_quantize_rows(ctx, x, s.T, s.H, ws + L.xq, reinterpret_cast<float*>(ws + L.sx), cs) != cudaSuccess)
@@ -752,6 +783,8 @@ moe_status moe_fused_forward_mx(moe_ctx* ctx, const void* x, const float* logits
   uint32_t* sfx_perm = reinterpret_cast<uint32_t*>(ws + L.sfx_perm);
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   begin_call(ctx, 0, stream);
+  st = check_logits_on_host(ctx, logits, cs);
+  if (st != MOE_OK) return st;
   if (moe::launch_plan_routing(ctx, logits, topk_ids, topk_w, counts, offsets, perm, inv_perm, cs) != cudaSuccess)
     return MOE_ERR_CUDA;
   if (moe::launch_quantize_rows_mx(ctx, x, s.T, s.H, ws + L.xq, sfx, cs) != cudaSuccess) return MOE_ERR_CUDA;

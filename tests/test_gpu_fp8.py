@@ -14,6 +14,9 @@ CASES = [
     gen.MoEConfig("f8_small", T=300, H=256, F=384, E=5, k=2, seed=91, router="xWr"),
     gen.MoEConfig("f8_skew", T=700, H=128, F=256, E=24, k=4, seed=92, router="xWr_zipf"),
     gen.MoEConfig("f8_dense", T=2600, H=384, F=512, E=2, k=2, seed=93, router="xWr"),      # CTA-pair kernel
+    # about 1000 rows per expert in two launches: below the CTA-pair threshold, so 256-row tiles on both accumulators,
+    # with a short swapped-operand or 128-row tile at the end of each expert
+    gen.MoEConfig("f8_wide", T=3000, H=512, F=1024, E=6, k=2, seed=94, router="xWr"),
 ]
 
 

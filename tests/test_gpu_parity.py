@@ -254,6 +254,33 @@ def test_environment_override_of_the_default_tuning(monkeypatch):
     assert ei.value.code == 1
 
 
+def test_debug_check_refuses_non_finite_logits(monkeypatch):
+    """Non-finite logits violate the routing contract and are not tested on the device; the debug entry
+    x.check_logits=1 of MOE_TUNING tests them on the host and returns MOE_ERR_BAD_ROUTING before any launch."""
+    cfg = gen.MoEConfig("nan", T=96, H=128, F=128, E=8, k=2, seed=35, router="xWr")
+    monkeypatch.setenv("MOE_TUNING", "x.check_logits=1")
+    L = Layer(cfg)
+    L.plan()                                         # finite logits pass
+    assert_plan_matches(L, oracle_for(L))
+    for bad in (float("nan"), float("inf"), float("-inf")):
+        logits = L.d_logits.clone()
+        logits[17, 3] = bad
+        with pytest.raises(binding.MoeError) as ei:
+            L.ctx.moe_plan_routing(logits, L.topk_ids, L.topk_w, L.counts, L.offsets, L.perm, L.inv_perm)
+        assert ei.value.code == 4
+        ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+        with pytest.raises(binding.MoeError) as ei:
+            L.ctx.moe_fused_forward(L.x, logits, L.w_gate, L.w_up, L.w_down, L.nan_bf16(cfg.T, cfg.H), ws)
+        assert ei.value.code == 4
+        assert L.ctx.moe_last_launch_count() == 0
+    monkeypatch.delenv("MOE_TUNING")
+    L2 = Layer(cfg)                                  # without the entry nothing is tested (and nothing synchronises)
+    logits = L2.d_logits.clone()
+    logits[0, 0] = float("inf")
+    L2.ctx.moe_plan_routing(logits, L2.topk_ids, L2.topk_w, L2.counts, L2.offsets, L2.perm, L2.inv_perm)
+    torch.cuda.synchronize()
+
+
 @pytest.mark.parametrize("cfg", [SMALL[0], SMALL[1], SMALL[5], SMALL[7],
                                  gen.MoEConfig("waves", T=1500, H=512, F=512, E=6, k=2, seed=51, router="xWr")],
                          ids=lambda c: c.name)
