@@ -1246,7 +1246,8 @@ bool tensor_map_2d(moe_ctx* ctx, const void* base, uint64_t rows, uint64_t cols,
                                                                : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
                                        const_cast<void*>(base), dims, strides, box, elem,
                                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                                       static_cast<CUtensorMapL2promotion>(moe_knob_value(ctx, "l2_promo", 3)),
+                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     m.base = nullptr;
     m.rows = 0;

@@ -45,23 +45,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 
-// The same test, but the hardware may keep the thread suspended for up to `hint_ns` before it answers: a warp that
-// waits this way leaves its scheduler's issue slots to the other warps (the MMA-issuing warp shares one with an
-// epilogue warp).
-__device__ __forceinline__ uint32_t mbar_try_wait_suspended(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(hint_ns)
-      : "memory");
-  return ok;
-}
-
 // Clock budget of one wait (about two seconds at 2 GHz): far above any legitimate wait in these kernels.
 constexpr long long kWaitClockBudget = 4000000000LL;
 
@@ -80,32 +63,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
-}
-
-// Bounded wait for roles that can afford a late wake-up (the epilogue warps, the tile ring): polls through the
-// suspending form and sleeps between polls, so that the waiting warp does not compete for issue slots.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait_suspended(bar, parity, 2000u)) return true;
-    __nanosleep(100);
-    if ((it & 0x3Fu) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitClockBudget) {
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait_relaxed_timed(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                                        long long* waited) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  const bool ok = mbar_wait_relaxed(bar, parity, abort_flag);
-  *waited += clock64() - t0;
-  return ok;
 }
 
 // Same, adding the clocks spent waiting (zero when the phase had already completed) to *waited.
