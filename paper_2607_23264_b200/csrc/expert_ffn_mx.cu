@@ -79,6 +79,7 @@ struct MxTail {
   uint32_t tmem_base;
   int abort_flag;
   int32_t blk_prefix[1025];   // exclusive prefix of ceil(count / 128) over experts
+  int32_t offs[1025];         // the expert row offsets, copied once: tile decoding reads no global memory
 };
 
 __device__ __forceinline__ void mx_timeout(const MxParams& p, int role) {
@@ -100,8 +101,8 @@ __device__ __forceinline__ MxTile decode_tile(int t, const MxTail* st, const MxP
   const int local = t - st->blk_prefix[e] * p.n_blocks;
   const int nb = local / blocks_e, mb = local - nb * blocks_e;
   MxTile tile;
-  tile.row0 = p.offsets[e] + mb * BM;
-  tile.row_end = p.offsets[e + 1];
+  tile.row0 = st->offs[e] + mb * BM;
+  tile.row_end = st->offs[e + 1];
   tile.n0 = nb * (kGated ? BNH : BN);
   tile.w_row0 = e * p.N + tile.n0;
   return tile;
@@ -139,7 +140,13 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     int32_t run = 0;
     for (int b0 = 0; b0 < p.E; b0 += 32) {
       const int e = b0 + lane;
-      int32_t v = e < p.E ? (p.offsets[e + 1] - p.offsets[e] + BM - 1) / BM : 0;
+      int32_t v = 0;
+      if (e < p.E) {
+        const int32_t lo = p.offsets[e], hi = p.offsets[e + 1];
+        st->offs[e + 1] = hi;
+        if (e == 0) st->offs[0] = lo;
+        v = (hi - lo + BM - 1) / BM;
+      }
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
         const int32_t o = __shfl_up_sync(0xFFFFFFFFu, v, off);
