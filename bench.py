@@ -204,6 +204,9 @@ def main():
                     help="run the burst/gap store microbenchmark on local HBM, print the rows and the calibration, exit")
     ap.add_argument("--trace", action="store_true",
                     help="add the grouped GEMMs' per-CTA wait counters (one extra traced step) to the JSON line")
+    ap.add_argument("--zero-operands", choices=["none", "weights", "all"], default="none",
+                    help="power diagnostic, not a benchmark: the same launches, bytes and instructions with the expert "
+                         "weights (and x) set to zero, which the 1 kW cap does not throttle")
     ap.add_argument("--profile", action="store_true",
                     help="profiler run: warm-up and timed steps only (no per-kernel pass, end-to-end or CPU legs)")
     args = ap.parse_args()
@@ -286,6 +289,12 @@ def main():
 
     gen.for_each_expert(cfg, sink)
     x = to_dev(x_bits)
+    if args.zero_operands != "none":
+        want_cpu = False
+        for w in (w_gate, w_up, w_down):
+            w.zero_()
+        if args.zero_operands == "all":
+            x.zero_()     # the logits stay the seeded ones: same routing, same tiles
     d_logits = torch.from_numpy(logits).to(dev)
     ctx = binding.Context(cfg.T, cfg.H, cfg.F, cfg.E, cfg.k, device=local_rank)
     ws = torch.empty(ctx.workspace_bytes(), dtype=torch.uint8, device=dev)
@@ -566,7 +575,9 @@ def main():
     line = {
         "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic" if args.zero_operands == "none" else
+                f"synthetic routing, ZERO {args.zero_operands} operands: power diagnostic, not a benchmark figure",
         "config": workload_config(cfg, world),
         "tflops": tflops, "frac_bf16_peak": tflops / world / peak_tf, "frac_bf16_peak_of": "bf16_tflops_sustained",
         "burst_ms_per_step": burst_ms_per_step, "burst_value": cfg.T * world / (burst_ms_per_step * 1e-3),
