@@ -266,7 +266,8 @@ def main():
     if args.router:
         run_router(args, cfg, binding, local_rank, dev)
         return
-    replicas.init_process_group(world, "nccl", torch.device(dev))
+    # started by a launcher (WORLD_SIZE set): join the group even as the only rank, so N = 1 takes the N-rank path
+    replicas.init_process_group(world, "nccl", torch.device(dev), force="WORLD_SIZE" in os.environ)
 
     # every rank gets its own batch (the seeded batch, rows rotated by rank); expert weights are replicated
     x_bits = replicas.rank_batch(gen.make_x(cfg), rank)
@@ -371,7 +372,7 @@ def main():
         if rank == 0:
             print(json.dumps({"profile_run": True, "ms_per_step": burst_total_ms / args.steps,
                               "config": workload_config(cfg, world)}), flush=True)
-        if world > 1:
+        if dist.is_initialized():
             dist.destroy_process_group()
         return
     burst_kernel_ms = kernel_pass(args.steps)
@@ -497,7 +498,7 @@ def main():
     d2h = out_host.numel() * 2
 
     if rank != 0:
-        if world > 1:
+        if dist.is_initialized():
             dist.destroy_process_group()
         return
 
@@ -633,7 +634,7 @@ def main():
     else:
         line["cpu_baseline"] = None
     print(json.dumps(line), flush=True)
-    if world > 1:
+    if dist.is_initialized():
         dist.destroy_process_group()
 
 

@@ -15,10 +15,13 @@ def rank_batch(x_bits: np.ndarray, rank: int) -> np.ndarray:
     return x_bits if rank == 0 else np.roll(x_bits, rank * 17, axis=0)
 
 
-def init_process_group(world: int, backend: str, device=None):
-    """Join the job's process group (rendezvous from the MASTER_* / RANK / WORLD_SIZE environment)."""
+def init_process_group(world: int, backend: str, device=None, force: bool = False):
+    """Join the job's process group (rendezvous from the MASTER_* / RANK / WORLD_SIZE environment).
+
+    A single process needs no group; `force` joins one all the same (a launcher started this process as the only
+    rank), so that a one-rank run takes the same path as an N-rank run."""
     import torch.distributed as dist
-    if world <= 1:
+    if world <= 1 and not force:
         return False
     if backend == "nccl":
         dist.init_process_group("nccl", device_id=device)
@@ -27,9 +30,14 @@ def init_process_group(world: int, backend: str, device=None):
     return True
 
 
+def _in_group() -> bool:
+    import torch.distributed as dist
+    return dist.is_available() and dist.is_initialized()
+
+
 def barrier(world: int):
     import torch.distributed as dist
-    if world > 1:
+    if world > 1 or _in_group():
         dist.barrier()
 
 
@@ -37,7 +45,7 @@ def max_over_ranks(value: float, world: int, device="cpu") -> float:
     """Slowest rank's figure (e.g. the device time of the timed region)."""
     import torch
     import torch.distributed as dist
-    if world <= 1:
+    if world <= 1 and not _in_group():
         return float(value)
     t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)

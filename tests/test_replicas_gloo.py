@@ -2,6 +2,8 @@
 import os
 import socket
 
+import pytest
+
 import numpy as np
 import torch.multiprocessing as mp
 
@@ -63,3 +65,42 @@ def test_launcher_command_for_two_ranks():
     import pytest
     with pytest.raises(ValueError):
         replicas.launcher_command(1, "bench.py", [], port=1)
+
+
+def test_forced_one_rank_group_takes_the_group_path():
+    """A process started by a launcher joins the group even as the only rank (gloo here, NCCL in bench.py)."""
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    p = ctx.Process(target=_forced_worker, args=(_free_port(), q))
+    p.start()
+    assert q.get(timeout=120) == (True, 7.25)
+    p.join(timeout=60)
+    assert p.exitcode == 0
+
+
+def _forced_worker(port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK="0", WORLD_SIZE="1")
+    import torch.distributed as dist
+    joined = replicas.init_process_group(1, "gloo", force=True)
+    replicas.barrier(1)
+    q.put((joined and dist.is_initialized(), replicas.max_over_ranks(7.25, 1)))
+    dist.destroy_process_group()
+
+
+@pytest.mark.gpu
+def test_bench_under_the_launcher_with_one_rank_joins_an_nccl_group():
+    """bench.py started by torch.distributed.run as the only rank: NCCL group, barrier and max-over-ranks reduction on the
+    GPU, the path every rank of an N-GPU run takes (N > 1 needs more GPUs than this test has)."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=1", "--master-addr", "127.0.0.1",
+           "--master-port", str(_free_port()), os.path.join(root, "bench.py"), "--gpus", "1", "--config", "C1",
+           "--steps", "5", "--warmup", "3", "--no-cpu-baseline", "--heat-seconds", "0.2"]
+    env = dict(os.environ, NCCL_DEBUG="INFO")
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=600, cwd=root, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["n_gpus"] == 1 and line["value"] > 0 and line["gpu_launches"] > 0
+    assert "NCCL INFO" in (r.stdout + r.stderr), "the NCCL group was not joined"
