@@ -62,7 +62,7 @@ class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-             "clocks_event_reasons.sw_power_cap")
+             "clocks_event_reasons.sw_power_cap,temperature.gpu")
 
     def __init__(self, index: int):
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
@@ -86,7 +86,7 @@ class ClockSampler:
                 self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, mx, power, reasons = [], [], [], set()
+        sm, mx, power, temp, reasons = [], [], [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for line in self.tmp.read().splitlines():
             parts = [p.strip() for p in line.split(",")]
@@ -98,6 +98,10 @@ class ClockSampler:
                 power.append(float(parts[2]))
             except ValueError:
                 continue
+            try:
+                temp.append(float(parts[7]))      # context: a hotter die leaks more and holds a lower clock at the cap
+            except (ValueError, IndexError):
+                pass
             for name, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
@@ -106,7 +110,8 @@ class ClockSampler:
         busy = [v for v in sm if v > 0]
         return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": sorted(reasons), "samples": len(sm),
-                "power_w_median": statistics.median(power) if power else None, "power_w_max": max(power) if power else None}
+                "power_w_median": statistics.median(power) if power else None, "power_w_max": max(power) if power else None,
+                "temp_c_median": statistics.median(temp) if temp else None}
 
 
 def oracle_threads() -> int:
@@ -339,15 +344,19 @@ def main():
     #   steady: args.steps steps back to back, bracketed by a barrier and a synchronize on both sides, one event
     #           between consecutive steps: ms_per_step = the whole region / steps (this is the line's value), and
     #           the median of the per-step times is reported beside it;
-    #   kernel passes after the burst and after the steady region: the same steps with the library's per-kernel
-    #           events read after every step.
+    #   the per-kernel times of the burst and of the steady region come from those very steps: the library records
+    #           its events inside them and keeps the last 32 calls' events, which are read after the region.
     for _ in range(args.warmup):
         step()
     barrier()
     sampler = ClockSampler(local_rank)
 
     def region(steps):
+        """steps back-to-back steps between two barriers.  The library records its per-kernel events inside the same
+        steps (a ring of the last 32 calls' events, read after the region: no host synchronisation in between), so the
+        kernel times are those of the timed steps themselves and sum to no more than the step."""
         marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        ctx.moe_set_kernel_timing(events_inside)
         barrier()
         marks[0].record(stream)
         for i in range(steps):
@@ -355,18 +364,30 @@ def main():
             marks[i + 1].record(stream)
         barrier()
         total = replicas.max_over_ranks(marks[0].elapsed_time(marks[-1]), world, dev)
-        return total, [marks[i].elapsed_time(marks[i + 1]) for i in range(steps)]
+        if events_inside:
+            per = [ctx.moe_get_kernel_times_back(b) for b in range(min(steps, binding.TIMING_SLOTS))]
+            ctx.moe_set_kernel_timing(False)
+        else:       # launch-bound layer: a pass of its own, the events read after every step
+            ctx.moe_set_kernel_timing(True)
+            per = []
+            for _ in range(steps):
+                step()
+                per.append(ctx.moe_get_kernel_times())
+            ctx.moe_set_kernel_timing(False)
+        kernels = [float(np.mean([s[i] for s in per])) for i in range(len(binding.KERNEL_NAMES))]
+        return total, [marks[i].elapsed_time(marks[i + 1]) for i in range(steps)], kernels
 
-    def kernel_pass(steps):
-        ctx.moe_set_kernel_timing(True)
-        per = []
-        for _ in range(steps):
-            step()
-            per.append(ctx.moe_get_kernel_times())
-        ctx.moe_set_kernel_timing(False)
-        return [float(np.mean([s[i] for s in per])) for i in range(len(binding.KERNEL_NAMES))]
+    # Eight event records per step cost a launch-bound layer a third of its step (65 against 44 us on the tiny
+    # layer), so for steps under half a millisecond the per-kernel times come from a separate pass instead.
+    probe = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    probe[0].record(stream)
+    for _ in range(3):
+        step()
+    probe[1].record(stream)
+    torch.cuda.synchronize()
+    events_inside = probe[0].elapsed_time(probe[1]) / 3 >= 0.5
 
-    burst_total_ms, _ = region(args.steps)
+    burst_total_ms, _, burst_kernel_ms = region(args.steps)
     launches = ctx.moe_last_launch_count() * args.steps
     if args.profile:
         if rank == 0:
@@ -375,7 +396,6 @@ def main():
         if dist.is_initialized():
             dist.destroy_process_group()
         return
-    burst_kernel_ms = kernel_pass(args.steps)
     if rank == 0:
         sampler.start()
     heat_t0, heat_steps = time.time(), 0
@@ -384,8 +404,7 @@ def main():
             step()
         heat_steps += 10
         torch.cuda.synchronize()
-    total_ms, step_times = region(args.steps)
-    kernel_ms = kernel_pass(args.steps)
+    total_ms, step_times, kernel_ms = region(args.steps)
     # SM clock of the steady region from the kernel itself: the Linear-1 producer's clock64 span over the kernel's
     # CUDA-event time, in one traced step taken while the GPU is still in that state (read, never set)
     ctx.moe_set_kernel_timing(True)
@@ -586,6 +605,8 @@ def main():
         "timed_region": f"{args.steps} back-to-back steps after {heat_steps} untimed pre-heating steps "
                         f"({args.heat_seconds:.1f} s); burst_* = {args.steps} steps right after the warm-up",
         "kernels_ms": dict(zip(binding.KERNEL_NAMES, kernel_ms)),
+        "kernels_ms_source": ("the timed steady steps themselves (library events inside the region)" if events_inside
+                              else "a separate pass after the region (launch-bound layer)"),
         "burst_kernels_ms": dict(zip(binding.KERNEL_NAMES, burst_kernel_ms)),
         "linear2_tflops": l2_tf, "linear1_gbs": l1_gbs, "linear2_gbs": l2_gbs, "dispatch_gbs": disp_gbs, "combine_gbs": comb_gbs,
         "dispatch_frac_hbm": disp_gbs / float(peaks["hbm_gbs"]), "combine_frac_hbm": comb_gbs / float(peaks["hbm_gbs"]),

@@ -492,9 +492,14 @@ moe_status moe_probe_mma_cycles_kind(moe_ctx* ctx, int32_t kind, int32_t M, int3
  * moe_get_kernel_times waits for the last call's events and writes the seven device durations in
  * milliseconds, in launch order {top-k + histogram, scan, scatter, dispatch, Linear-1, Linear-2, combine},
  * to the HOST array ms_host[n], n == 7; kernels the last call did not launch read -1.
+ * The events of the last 32 timed calls are kept (a ring, one slot per call), so a run of back-to-back calls can be
+ * timed per kernel without a host synchronisation between them: moe_get_kernel_times_back reads the call that
+ * was `calls_back` timed calls before the last one (0 = the last; 0 <= calls_back < 32, else MOE_ERR_INVALID_ARG;
+ * a slot no call has used since timing was enabled reads -1 throughout).  Enabling or disabling clears the ring.
  */
 moe_status moe_set_kernel_timing(moe_ctx* ctx, int32_t enable);
 moe_status moe_get_kernel_times(moe_ctx* ctx, float* ms_host, int32_t n);
+moe_status moe_get_kernel_times_back(moe_ctx* ctx, int32_t calls_back, float* ms_host, int32_t n);
 
 #ifdef __cplusplus
 }

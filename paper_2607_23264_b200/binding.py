@@ -29,8 +29,10 @@ EXPORTS = (
     "moe_set_active_tokens", "moe_plan_routing_from_topk", "moe_router_weight_bytes", "moe_router_scratch_bytes",
     "moe_router_prepare", "moe_route_tokens", "moe_fused_forward_routed", "moe_quantize_rows_mx", "moe_dispatch_mx",
     "moe_expert_ffn_mx", "moe_get_workspace_layout_mx", "moe_fused_forward_mx", "moe_probe_mma_cycles_kind",
-    "moe_parse_tuning",
+    "moe_parse_tuning", "moe_get_kernel_times_back",
 )
+
+TIMING_SLOTS = 32     # timed calls whose per-kernel events the library keeps (moe_get_kernel_times_back)
 
 TRACE_FIELDS = ("producer_span", "producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator",
                 "epilogue_wait_accumulator", "epilogue_store_span", "tiles", "epilogue_pacing_gap",
@@ -138,6 +140,7 @@ def load_library() -> C.CDLL:
     lib.moe_last_launch_count.restype = C.c_int32
     lib.moe_set_kernel_timing.argtypes = [vp, C.c_int32]
     lib.moe_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32]
+    lib.moe_get_kernel_times_back.argtypes = [vp, C.c_int32, C.POINTER(C.c_float), C.c_int32]
     lib.moe_probe_mma_cycles.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_double), vp]
     lib.moe_probe_mma_cycles_kind.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_double), vp]
     lib.moe_get_ffn_order.argtypes = [vp, C.POINTER(C.c_int32), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
@@ -453,4 +456,10 @@ class Context:
     def moe_get_kernel_times(self) -> list:
         ms = (C.c_float * len(KERNEL_NAMES))()
         _check(self._lib.moe_get_kernel_times(self._handle, ms, len(KERNEL_NAMES)), "moe_get_kernel_times")
+        return list(ms)
+
+    def moe_get_kernel_times_back(self, calls_back: int) -> list:
+        ms = (C.c_float * len(KERNEL_NAMES))()
+        _check(self._lib.moe_get_kernel_times_back(self._handle, calls_back, ms, len(KERNEL_NAMES)),
+               "moe_get_kernel_times_back")
         return list(ms)

@@ -115,7 +115,10 @@ moe_status check_ctx(const moe_ctx* ctx) {
 // precedes the call's first kernel.
 inline void begin_call(moe_ctx* ctx, int first_mark, void* stream) {
   ctx->last_launches = 0;
-  ctx->ev_recorded = 0;
+  if (ctx->timing) {                      // a timed call takes the next slot of the event ring
+    ctx->ev_slot = (ctx->ev_slot + 1) % kMoeTimingSlots;
+    ctx->ev_recorded[ctx->ev_slot] = 0;
+  }
   moe_mark(ctx, first_mark, static_cast<cudaStream_t>(stream));
 }
 
@@ -257,7 +260,8 @@ moe_status moe_create(moe_ctx** out_ctx, const moe_shape* shape, int device) {
   ok = ok && moe::prepare_expert_ffn(ctx) == cudaSuccess;
   ok = ok && moe::prepare_router(ctx) == cudaSuccess;
   ok = ok && moe::prepare_expert_ffn_mx(ctx) == cudaSuccess;
-  for (int i = 0; ok && i <= kMoeKernels; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
+  for (int sl = 0; ok && sl < kMoeTimingSlots; ++sl)
+    for (int i = 0; ok && i <= kMoeKernels; ++i) ok = cudaEventCreate(&ctx->ev[sl][i]) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) == cudaSuccess;
   for (int i = 0; ok && i < 2; ++i) {
@@ -290,8 +294,9 @@ void moe_destroy(moe_ctx* ctx) {
   if (ctx->d_ready) cudaFree(ctx->d_ready);
   if (ctx->d_order) cudaFree(ctx->d_order);
   if (ctx->d_router_done) cudaFree(ctx->d_router_done);
-  for (int i = 0; i <= kMoeKernels; ++i)
-    if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
+  for (int sl = 0; sl < kMoeTimingSlots; ++sl)
+    for (int i = 0; i <= kMoeKernels; ++i)
+      if (ctx->ev[sl][i]) cudaEventDestroy(ctx->ev[sl][i]);
   for (int i = 0; i < 2; ++i) {
     if (ctx->ev_h2d[i]) cudaEventDestroy(ctx->ev_h2d[i]);
     if (ctx->ev_compute[i]) cudaEventDestroy(ctx->ev_compute[i]);
@@ -940,22 +945,27 @@ moe_status moe_get_ffn_order(moe_ctx* ctx, int32_t* codes_host, int32_t capacity
 moe_status moe_set_kernel_timing(moe_ctx* ctx, int32_t enable) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   ctx->timing = enable ? 1 : 0;
-  ctx->ev_recorded = 0;
+  for (int sl = 0; sl < kMoeTimingSlots; ++sl) ctx->ev_recorded[sl] = 0;
+  return MOE_OK;
+}
+
+moe_status moe_get_kernel_times_back(moe_ctx* ctx, int32_t calls_back, float* ms_host, int32_t n) {
+  moe_status st = check_ctx(ctx);
+  if (st != MOE_OK) return st;
+  if (!ms_host || n != kMoeKernels || calls_back < 0 || calls_back >= kMoeTimingSlots) return MOE_ERR_INVALID_ARG;
+  const int sl = ((ctx->ev_slot - calls_back) % kMoeTimingSlots + kMoeTimingSlots) % kMoeTimingSlots;
+  for (int i = 0; i < kMoeKernels; ++i) {
+    ms_host[i] = -1.f;
+    const uint32_t need = (1u << i) | (1u << (i + 1));
+    if ((ctx->ev_recorded[sl] & need) != need) continue;
+    if (cudaEventSynchronize(ctx->ev[sl][i + 1]) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms_host[i], ctx->ev[sl][i], ctx->ev[sl][i + 1]) != cudaSuccess) return MOE_ERR_CUDA;
+  }
   return MOE_OK;
 }
 
 moe_status moe_get_kernel_times(moe_ctx* ctx, float* ms_host, int32_t n) {
-  moe_status st = check_ctx(ctx);
-  if (st != MOE_OK) return st;
-  if (!ms_host || n != kMoeKernels) return MOE_ERR_INVALID_ARG;
-  for (int i = 0; i < kMoeKernels; ++i) {
-    ms_host[i] = -1.f;
-    const uint32_t need = (1u << i) | (1u << (i + 1));
-    if ((ctx->ev_recorded & need) != need) continue;
-    if (cudaEventSynchronize(ctx->ev[i + 1]) != cudaSuccess) return MOE_ERR_CUDA;
-    if (cudaEventElapsedTime(&ms_host[i], ctx->ev[i], ctx->ev[i + 1]) != cudaSuccess) return MOE_ERR_CUDA;
-  }
-  return MOE_OK;
+  return moe_get_kernel_times_back(ctx, 0, ms_host, n);
 }
 
 }  // extern "C"

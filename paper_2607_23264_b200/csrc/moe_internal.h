@@ -10,6 +10,7 @@
 constexpr int kRouteThreads = 256;
 // Kernels of one forward, in launch order: top-k+histogram, scan, scatter, dispatch, Linear-1, Linear-2, combine.
 constexpr int kMoeKernels = 7;
+constexpr int kMoeTimingSlots = 32;   // calls whose per-kernel events are kept (a ring: one slot per timed call)
 // Wait counters one CTA of a grouped GEMM records when tracing is on (SM clocks unless noted):
 // 0 producer loop span, 1 producer waited for a free stage, 2 MMA waited for data, 3 MMA waited for a free
 // accumulator (the epilogue's back-pressure), 4 epilogue waited for an accumulator, 5 epilogue drain+store span,
@@ -72,8 +73,9 @@ struct moe_ctx {
   int pipe_slot;
   // Optional per-kernel timing: event i is recorded after kernel i (event 0 before the first kernel).
   int timing;
-  uint32_t ev_recorded;          // bit i set when ev[i] was recorded by the last call
-  cudaEvent_t ev[kMoeKernels + 1];
+  int ev_slot;                                  // slot of the last timed call
+  uint32_t ev_recorded[kMoeTimingSlots];        // bit i set when ev[slot][i] was recorded by that slot's call
+  cudaEvent_t ev[kMoeTimingSlots][kMoeKernels + 1];
 };
 
 // Value of the development knob "x.<name>" from MOE_TUNING, or dflt.
@@ -95,7 +97,8 @@ inline moe_tuning moe_effective_tuning(const moe_ctx* ctx, const moe_tuning* giv
 
 // Record timing mark i on the stream when per-kernel timing is enabled.
 inline void moe_mark(moe_ctx* ctx, int i, cudaStream_t stream) {
-  if (ctx->timing && cudaEventRecord(ctx->ev[i], stream) == cudaSuccess) ctx->ev_recorded |= 1u << i;
+  if (ctx->timing && cudaEventRecord(ctx->ev[ctx->ev_slot][i], stream) == cudaSuccess)
+    ctx->ev_recorded[ctx->ev_slot] |= 1u << i;
 }
 
 // Launchers (each returns the cudaError_t of its launches).  `stream` is the caller's stream.

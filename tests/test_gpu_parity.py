@@ -385,6 +385,40 @@ def test_host_side_errors_are_synchronous():
     L.check_device_status()
 
 
+def test_kernel_times_of_back_to_back_calls():
+    """The library keeps the per-kernel events of the last 32 timed calls, so a run of calls is timed per kernel without a
+    host synchronisation in between; each call's kernel times sum to no more than the time between the calls' ends."""
+    cfg = gen.MoEConfig("ring", T=2000, H=512, F=512, E=6, k=2, seed=62, router="xWr")
+    L = Layer(cfg)
+    ws = torch.empty(L.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    out = L.nan_bf16(cfg.T, cfg.H)
+    step = lambda: L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
+    for _ in range(3):
+        step()
+    n = 5
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    L.ctx.moe_set_kernel_timing(True)
+    assert all(v == -1 for v in L.ctx.moe_get_kernel_times_back(0)), "enabling clears the ring"
+    marks[0].record()
+    for i in range(n):
+        step()
+        marks[i + 1].record()
+    torch.cuda.synchronize()
+    per = [L.ctx.moe_get_kernel_times_back(b) for b in range(n)]      # per[0] = the last call
+    assert all(len(ms) == 7 and all(v > 0 for v in ms) for ms in per)
+    for b in range(n):
+        step_ms = marks[n - 1 - b].elapsed_time(marks[n - b])
+        assert sum(per[b]) <= step_ms * 1.02 + 0.01, (b, per[b], step_ms)
+    assert per[0] == L.ctx.moe_get_kernel_times()
+    assert all(v == -1 for v in L.ctx.moe_get_kernel_times_back(n)), "a slot no call has used reads -1"
+    for bad in (-1, binding.TIMING_SLOTS):
+        with pytest.raises(binding.MoeError) as ei:
+            L.ctx.moe_get_kernel_times_back(bad)
+        assert ei.value.code == 1
+    L.ctx.moe_set_kernel_timing(False)
+    L.check_device_status()
+
+
 def test_ffn_trace_and_kernel_times():
     """Measurement aids: per-kernel event times and the per-CTA wait counters of the grouped GEMMs."""
     cfg = gen.MoEConfig("traced", T=4000, H=512, F=384, E=6, k=2, seed=61, router="xWr")   # two launches
