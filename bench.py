@@ -186,6 +186,8 @@ def main():
     ap.add_argument("--cpu-baseline-tokens", type=int, default=128,
                     help="tokens of the cpu_baseline leg (the same sample size as a step of the reference arm)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-local-peak", action="store_true",
+                    help="skip the context measurement of the library bf16 GEMM on this GPU (after all timed regions)")
     ap.add_argument("--heat-seconds", type=float, default=2.0,
                     help="back-to-back untimed steps before the timed region, until the power cap has settled the clocks")
     ap.add_argument("--burst", type=int, default=1)
@@ -516,6 +518,34 @@ def main():
     h2d = x_host.numel() * 2 + logits_host.numel() * 4
     d2h = out_host.numel() * 2
 
+    # Context, after every timed region and on nothing the layer uses: the library bf16 GEMM of the measured-peaks file
+    # (8192^3, back to back for 2 s after 1 s of the same) on the GPU at hand.  GPUs of one pool hold different clocks
+    # at the same 1 kW cap; this says how the GPU of this run compares with the one the peaks were taken on.  The
+    # roofline's `peak` stays the file's figure.
+    local_peak = None
+    if rank == 0 and world == 1 and not args.no_local_peak and not args.profile:
+        n = 8192
+        ga = torch.randn((n, n), device=dev, dtype=torch.float32).to(torch.bfloat16)
+        gb = torch.randn((n, n), device=dev, dtype=torch.float32).to(torch.bfloat16)
+        gc = torch.empty((n, n), device=dev, dtype=torch.bfloat16)
+        t_heat = time.time()
+        while time.time() - t_heat < 1.0:
+            for _ in range(20):
+                torch.matmul(ga, gb, out=gc)
+            torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        count, t_run = 0, time.time()
+        g0.record(stream)
+        while time.time() - t_run < 2.0:
+            for _ in range(20):
+                torch.matmul(ga, gb, out=gc)
+            count += 20
+            torch.cuda.synchronize()
+        g1.record(stream)
+        torch.cuda.synchronize()
+        local_peak = 2.0 * n ** 3 * count / (g0.elapsed_time(g1) * 1e-3) / 1e12
+        del ga, gb, gc
+
     if rank != 0:
         if dist.is_initialized():
             dist.destroy_process_group()
@@ -591,6 +621,12 @@ def main():
     if roofline["bound"] == "tensor" and peak_mhz > 0 and clocks and clocks.get("sm_mhz_kernel"):
         roofline["peak_sm_mhz"] = peak_mhz
         roofline["frac_at_equal_clock"] = roofline["frac"] * peak_mhz / clocks["sm_mhz_kernel"]
+    if local_peak is not None:
+        roofline["local_library_gemm"] = {
+            "bf16_tflops_sustained_this_gpu": local_peak,
+            "how": "torch.matmul bf16 8192^3 back to back for 2 s after 1 s of the same, after all timed regions",
+            "of_measured_peaks_file": local_peak / float(peaks.get("bf16_tflops_sustained") or float("nan")),
+            **({"frac_of_this_gpu": roofline["achieved"] / local_peak} if roofline["bound"] == "tensor" else {})}
     burst_ms_per_step = burst_total_ms / args.steps
     line = {
         "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,

@@ -315,7 +315,10 @@ def test_schedules_are_bitwise_identical(cfg):
 
 
 @pytest.mark.parametrize("cfg", [SMALL[1], SMALL[3], SMALL[5], SMALL[7],
-                                 gen.MoEConfig("pairs", T=3000, H=512, F=640, E=3, k=2, seed=81, router="xWr")],
+                                 gen.MoEConfig("pairs", T=3000, H=512, F=640, E=3, k=2, seed=81, router="xWr"),
+                                 gen.MoEConfig("pair_tails", T=1500, H=1024, F=512, E=4, k=2, seed=82, router="xWr"),
+                                 gen.MoEConfig("pair_tails_skew", T=2200, H=512, F=256, E=8, k=2, seed=83,
+                                               router="xWr_zipf")],
                          ids=lambda c: c.name)
 def test_cta_pair_kernel_matches_single_cta_kernel(cfg):
     """The cta_group::2 variant (256-row tiles over a cluster of two CTAs), forced on, gives the same bits as the
