@@ -205,6 +205,10 @@ def main():
                     help="time the FP8 (E4M3, W8A8) variant of the layer instead (weights quantised on the GPU first)")
     ap.add_argument("--mxfp8", action="store_true",
                     help="the block-scaled FP8 variant of the experts (E4M3 elements, E8M0 scale per 32 elements along K)")
+    ap.add_argument("--library-gemms", action="store_true",
+                    help="context, not the product: the layer's two grouped GEMMs as one library bf16 GEMM call per "
+                         "expert (torch.matmul on the seeded routing's row ranges; no SiLU, no routing, no movers), "
+                         "pre-heated, on this GPU")
     ap.add_argument("--router", action="store_true",
                     help="time the router front end (logits + top-k in one kernel, then the plan) on --config's shape")
     ap.add_argument("--xstage-probe", action="store_true",
@@ -272,6 +276,9 @@ def main():
         return
     if args.router:
         run_router(args, cfg, binding, local_rank, dev)
+        return
+    if args.library_gemms:
+        run_library_gemms(args, cfg, dev, local_rank)
         return
     # started by a launcher (WORLD_SIZE set): join the group even as the only rank, so N = 1 takes the N-rank path
     replicas.init_process_group(world, "nccl", torch.device(dev), force="WORLD_SIZE" in os.environ)
@@ -841,6 +848,71 @@ def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
         "gpu_launches": ctx.moe_last_launch_count() * args.steps, "clocks": clocks, "gemm_waits": waits,
     }
     print(json.dumps(line), flush=True)
+
+
+def run_library_gemms(args, cfg, dev, local_rank):
+    """What the two grouped GEMMs cost as library calls on this GPU: one torch.matmul per non-empty expert and weight
+    matrix over that expert's rows of the seeded routing.  Random operands of the layer's distributions (timing does
+    not depend on the values beyond their statistics); no SiLU*mul, routing, dispatch or combine.  Context for the
+    bench line of the same workload: both sit under the same 1 kW cap on the same GPU."""
+    import torch
+    from oracle import moe_oracle as orc      # host-side routing of the seeded logits: counts only, outside any timing
+    x_bits = gen.make_x(cfg)
+    ids, _ = orc.topk_route(gen.make_logits(cfg, x_bits), cfg.k)
+    counts = np.bincount(ids.ravel(), minlength=cfg.E)
+    offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    R, H, F = cfg.R, cfg.H, cfg.F
+    gsd = torch.Generator(device=dev).manual_seed(cfg.seed)
+    rnd = lambda shape, std: (torch.randn(shape, generator=gsd, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
+    live = [e for e in range(cfg.E) if counts[e] > 0]
+    xp, hp = rnd((R, H), 1.0), rnd((R, F), 0.5)
+    wg = {e: rnd((F, H), H ** -0.5) for e in live}
+    wu = {e: rnd((F, H), H ** -0.5) for e in live}
+    wd = {e: rnd((H, F), F ** -0.5) for e in live}
+    g, u = torch.empty((R, F), dtype=torch.bfloat16, device=dev), torch.empty((R, F), dtype=torch.bfloat16, device=dev)
+    y = torch.empty((R, H), dtype=torch.bfloat16, device=dev)
+
+    def linear1():
+        for e in live:
+            lo, hi = int(offs[e]), int(offs[e + 1])
+            torch.matmul(xp[lo:hi], wg[e].t(), out=g[lo:hi])
+            torch.matmul(xp[lo:hi], wu[e].t(), out=u[lo:hi])
+
+    def linear2():
+        for e in live:
+            lo, hi = int(offs[e]), int(offs[e + 1])
+            torch.matmul(hp[lo:hi], wd[e].t(), out=y[lo:hi])
+
+    def sustained(fn):
+        t0 = time.time()
+        while time.time() - t0 < max(args.heat_seconds, 1.0):
+            fn()
+            torch.cuda.synchronize()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n, t0 = 0, time.time()
+        e0.record()
+        while time.time() - t0 < 2.0:
+            for _ in range(5):
+                fn()
+            n += 5
+            torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n, sampler.stop()
+
+    ms1, _ = sustained(linear1)
+    ms2, _ = sustained(linear2)
+    ms12, clocks = sustained(lambda: (linear1(), linear2()))
+    print(json.dumps({
+        "library_gemms": "torch.matmul bf16, one call per non-empty expert and weight matrix, rows of the seeded routing",
+        "config": workload_config(cfg, 1), "nonempty_experts": len(live),
+        "linear1_ms": ms1, "linear2_ms": ms2, "both_ms": ms12,
+        "linear1_tflops": 4.0 * R * H * F / (ms1 * 1e-3) / 1e12, "linear2_tflops": 2.0 * R * H * F / (ms2 * 1e-3) / 1e12,
+        "both_tflops": 6.0 * R * H * F / (ms12 * 1e-3) / 1e12, "clocks": clocks,
+        "note": "GEMMs only (no SiLU*mul, routing, dispatch, combine); context for the bench line, not a product path"}),
+        flush=True)
 
 
 def run_router(args, cfg, binding, local_rank, dev):
