@@ -856,12 +856,16 @@ def run_library_gemms(args, cfg, dev, local_rank):
     not depend on the values beyond their statistics); no SiLU*mul, routing, dispatch or combine.  Context for the
     bench line of the same workload: both sit under the same 1 kW cap on the same GPU."""
     import torch
-    from oracle import moe_oracle as orc      # host-side routing of the seeded logits: counts only, outside any timing
-    x_bits = gen.make_x(cfg)
-    ids, _ = orc.topk_route(gen.make_logits(cfg, x_bits), cfg.k)
-    counts = np.bincount(ids.ravel(), minlength=cfg.E)
-    offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    from paper_2607_23264_b200 import binding
     R, H, F = cfg.R, cfg.H, cfg.F
+    x_bits = gen.make_x(cfg)
+    d_logits = torch.from_numpy(gen.make_logits(cfg, x_bits)).to(dev)
+    ctx = binding.Context(cfg.T, H, F, cfg.E, cfg.k, device=local_rank)      # the library's own routing plan: row ranges
+    i32 = lambda n: torch.empty(n, dtype=torch.int32, device=dev)
+    d_counts, d_offs = i32(cfg.E), i32(cfg.E + 1)
+    ctx.moe_plan_routing(d_logits, i32(R), torch.empty(R, dtype=torch.float32, device=dev), d_counts, d_offs, i32(R), i32(R))
+    torch.cuda.synchronize()
+    counts, offs = d_counts.cpu().numpy(), d_offs.cpu().numpy().astype(np.int64)
     gsd = torch.Generator(device=dev).manual_seed(cfg.seed)
     rnd = lambda shape, std: (torch.randn(shape, generator=gsd, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
     live = [e for e in range(cfg.E) if counts[e] > 0]
