@@ -584,7 +584,8 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         const PhaseDesc& d = p.ph[t.phase];
         // L2 priorities: the weights of an expert with a single row block are read by this tile alone (bit 0: they go
         // first); the rows of A are read once per column block (bit 1: they stay, Linear-2 only: bit 2)
-        const uint64_t pol_w = ((p.cache_hints & 1) && t.single) ? pol_first : pol_normal;
+        const uint64_t pol_w = ((p.cache_hints & 1) && t.single) ? pol_first
+                               : ((p.cache_hints & 32) && !t.single) ? pol_last : pol_normal;
         const uint64_t pol_a = ((p.cache_hints & 2) && (t.phase == 1 || !(p.cache_hints & 4))) ? pol_last : pol_normal;
         const CUtensorMap* ma = t.phase == 0 ? &tm_x : &tm_h;
         const CUtensorMap* mb0 = t.phase == 0 ? &tm_wg : &tm_wd;
@@ -1414,14 +1415,16 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   p.fp8 = c.fp8;
   p.k_elems = k_elems;
   p.swap_rows = moe_knob_value(ctx, "swap_rows", kSwapRows);
-  // L2 eviction priorities of the TMA loads (development knob cache_hints, a bit mask).  Default 3 = in the single-CTA
-  // kernel the weights of an expert with a single row block go first (bit 0: no other tile reads them, and on layers
-  // of many small experts they are nearly all of the traffic) and the rows of A stay (bit 1: every column block of
-  // the expert reads them again).  Measured in the power-capped steady state: -6 % on the decode-like layer, -3.7 %
-  // on the DeepSeek-V3-like one, nothing on the Mixtral-like layer at any batch size.  Bit 2 restricts bit 1 to
-  // Linear-2; bits 3 and 4 are the same two priorities in the CTA-pair kernel, where they do not pay (A rows: no
-  // change; weights first: 17 % slower, the row blocks that share a weight box do not run closely enough together).
-  p.cache_hints = moe_knob_value(ctx, "cache_hints", 3);
+  // L2 eviction priorities of the TMA loads (development knob cache_hints, a bit mask).  Default 35 = in the
+  // single-CTA kernel the weights of an expert with a single row block go first (bit 0: no other tile reads them, and
+  // on layers of many small experts they are nearly all of the traffic), the rows of A stay (bit 1: every column block
+  // of the expert reads them again) and so do the weights of experts with several row blocks (bit 5: each of those
+  // blocks reads them).  Measured in the power-capped steady state: bits 0 and 1 -6 % on the decode-like layer and
+  // -3.7 % on the DeepSeek-V3-like one; bit 5 another -1.2 % there and -1 to -2 % on the Mixtral-like layer at 1024 to
+  // 3072 tokens.  Bit 2 restricts bit 1 to Linear-2; bits 3 and 4 are the priorities of bits 1 and 0 in the CTA-pair
+  // kernel, where they do not pay (A rows: no change; weights first: 17 % slower, the row blocks that share a weight
+  // box do not run closely enough together).
+  p.cache_hints = moe_knob_value(ctx, "cache_hints", 35);
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
   // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
   p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);

@@ -65,10 +65,12 @@ struct MxParams {
   __nv_bfloat16* y;         // Linear-2 out: bf16 [R, N]
   int32_t* status;
   unsigned long long* trace;   // null, or [CTAs][kMoeTraceFields] wait counters (the fields of the bf16 kernel)
+  int cache_hints;          // L2 eviction priorities of the TMA loads: the bits of the bf16 kernel's knob (0, 1, 5)
 };
 
 struct MxTile {
   int row0, row_end, n0, w_row0;
+  int single;     // the expert has a single row block: no other tile reads these weight boxes
 };
 
 struct MxTail {
@@ -105,6 +107,7 @@ __device__ __forceinline__ MxTile decode_tile(int t, const MxTail* st, const MxP
   tile.row_end = st->offs[e + 1];
   tile.n0 = nb * (kGated ? BNH : BN);
   tile.w_row0 = e * p.N + tile.n0;
+  tile.single = blocks_e == 1 ? 1 : 0;
   return tile;
 }
 
@@ -182,8 +185,15 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       bool ok = true;
       long long w_empty = 0;
       const long long t_begin = clock64();
+      // L2 priorities as in the bf16 kernel: weights read by this tile alone go first, weights other row blocks read
+      // again and the rows of A (read again by every column block) stay
+      const uint64_t pol_first = ptx::l2_policy_evict_first(), pol_last = ptx::l2_policy_evict_last(),
+                     pol_normal = ptx::l2_policy_evict_normal();
+      const uint64_t pol_a = (p.cache_hints & 2) ? pol_last : pol_normal;
       for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
         const MxTile tile = decode_tile<kGated>(t, st, p);
+        const uint64_t pol_w = ((p.cache_hints & 1) && tile.single) ? pol_first
+                               : ((p.cache_hints & 32) && !tile.single) ? pol_last : pol_normal;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, &w_empty)) {
             mx_timeout(p, 1);
@@ -193,9 +203,9 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
           const uint32_t full = ptx::smem_u32(&st->full[stage]);
           const uint32_t sa = ring_u32 + stage * kOperandBytes;
           ptx::mbar_expect_tx(full, kOperandBytes);
-          ptx::tma_load_2d(sa, &tm_a, full, kb * BK, tile.row0);
-          ptx::tma_load_2d(sa + kABytes, &tm_b0, full, kb * BK, tile.w_row0);
-          ptx::tma_load_2d(sa + kABytes + kBBoxBytes, &tm_b1, full, kb * BK, tile.w_row0 + b1_shift);
+          ptx::tma_load_2d_hint(sa, &tm_a, full, kb * BK, tile.row0, pol_a);
+          ptx::tma_load_2d_hint(sa + kABytes, &tm_b0, full, kb * BK, tile.w_row0, pol_w);
+          ptx::tma_load_2d_hint(sa + kABytes + kBBoxBytes, &tm_b1, full, kb * BK, tile.w_row0 + b1_shift, pol_w);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -478,6 +488,7 @@ moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, cudaStre
   p1.h_dbg = a->h_fp32_debug;
   p1.status = ctx->d_status;
   p1.trace = ctx->timing ? ctx->d_trace : nullptr;   // per-kernel timing also turns the wait counters on
+  p1.cache_hints = moe_knob_value(ctx, "cache_hints", 35);
 
   MxParams p2{};
   p2.offsets = p1.offsets;
@@ -492,6 +503,7 @@ moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, cudaStre
   p2.sf_b1 = p2.sf_b0;
   p2.y = static_cast<__nv_bfloat16*>(a->y_perm);
   p2.status = ctx->d_status;
+  p2.cache_hints = p1.cache_hints;
   p2.trace = ctx->timing ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
 
   const int grid = ctx->num_sms;
