@@ -822,7 +822,10 @@ def run_mxfp8(args, cfg, ctx, binding, bufs, timed, rank, world, dev):
                         "mma_waits_operands": float((tr[gi, :, 2] / span).mean()),
                         "mma_waits_accumulator": float((tr[gi, :, 3] / span).mean()),
                         "producer_waits_stage": float((tr[gi, :, 1] / span).mean()),
-                        "epilogue_busy": float((tr[gi, :, 5] / span).mean())}
+                        "epilogue_busy": float((tr[gi, :, 5] / span).mean()),
+                        "swapped_tiles_per_cta": float(tr[gi, :, 8].mean()),
+                        "clocks_per_swapped_tile": float(tr[gi, :, 9].sum() / max(tr[gi, :, 8].sum(), 1.0)),
+                        "clocks_per_other_tile": float(tr[gi, :, 11].sum() / max((tr[gi, :, 6] - tr[gi, :, 8]).sum(), 1.0))}
     code, detail = ctx.moe_last_device_status()
     if code != 0:
         raise RuntimeError(f"device status {code} detail {detail:#x}")

@@ -22,6 +22,8 @@
 // Every wait is bounded; a wait that gives up is reported through the status word and the CTA unwinds.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "ffn_math.cuh"
 #include "moe_internal.h"
 #include "mx_quant.cuh"
@@ -47,6 +49,7 @@ constexpr uint32_t kTmemSfA = kAccBufs * BN;   // column of the A scales
 constexpr uint32_t kTmemSfB = kAccBufs * BN + 4;
 constexpr int kSfThreads = 128;
 constexpr int kKernelIdMx = 9;          // in the detail word of a time-out: 9 * 65536 + role
+constexpr int kMxSwapRows = 64;         // row blocks with at most this many rows run with swapped operands
 
 struct MxParams {
   const int32_t* offsets;   // [E+1]
@@ -66,11 +69,13 @@ struct MxParams {
   int32_t* status;
   unsigned long long* trace;   // null, or [CTAs][kMoeTraceFields] wait counters (the fields of the bf16 kernel)
   int cache_hints;          // L2 eviction priorities of the TMA loads: the bits of the bf16 kernel's knob (0, 1, 5)
+  int swap_rows;            // row blocks with at most this many rows run with swapped operands (at most 64)
 };
 
 struct MxTile {
   int row0, row_end, n0, w_row0;
   int single;     // the expert has a single row block: no other tile reads these weight boxes
+  int n_pad;      // 0, or the row count padded to 16 of a block of few rows, computed with swapped operands
 };
 
 struct MxTail {
@@ -108,6 +113,12 @@ __device__ __forceinline__ MxTile decode_tile(int t, const MxTail* st, const MxP
   tile.n0 = nb * (kGated ? BNH : BN);
   tile.w_row0 = e * p.N + tile.n0;
   tile.single = blocks_e == 1 ? 1 : 0;
+  const int rows = min(tile.row_end - tile.row0, BM);
+  // swapped operands for small experts only: in clocks such a tile is slower than a 128-row tile (eight short
+  // block-scaled MMAs per K block are bound by the issuing thread: 1060 against 810 clocks), what it saves is power,
+  // which pays where such tiles are most of the launch (decode-like batches) and not for the odd short last block of
+  // a many-row expert
+  tile.n_pad = (blocks_e == 1 && rows <= p.swap_rows) ? ((rows + 15) & ~15) : 0;
   return tile;
 }
 
@@ -223,47 +234,90 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      long long w_full = 0, w_tmem = 0;
-      unsigned long long n_tiles = 0;
+      long long w_full = 0, w_tmem = 0, t_swapped = 0, t_plain = 0;
+      unsigned long long n_tiles = 0, n_swapped = 0;
       for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+        const long long t_tile = clock64();
+        const int n_pad = decode_tile<kGated>(t, st, p).n_pad;    // (decoded while the epilogue still drains)
         if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, &w_tmem)) {
           mx_timeout(p, 2);
           break;
         }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), phase, abort_flag, &w_full)) {
-            mx_timeout(p, 3);
-            ok = false;
-            break;
+        // One K loop per tile kind (a run-time branch between the MMAs of a K block would cost the issuing thread
+        // 100-200 clocks per block): wait for the stage, copy its scales to tensor memory, issue, free the stage.
+        auto k_loop = [&](auto&& issue) -> bool {
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->full[stage]), phase, abort_flag, &w_full)) {
+              mx_timeout(p, 3);
+              return false;
+            }
+            ptx::tc_fence_after_sync();
+            const uint32_t sf = sf_u32 + stage * kSfBytes;
+            ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfA, sf);
+            ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB, sf + kSfABytes);
+            ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB + 4, sf + kSfABytes + 512);
+            issue(ring_u32 + stage * kOperandBytes, kb != 0 ? 1u : 0u);
+            ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // codes and scales are free once these are done
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
-          ptx::tc_fence_after_sync();
-          const uint32_t sa = ring_u32 + stage * kOperandBytes;
-          const uint32_t sf = sf_u32 + stage * kSfBytes;
-          ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfA, sf);
-          ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB, sf + kSfABytes);
-          ptx::tc_cp_32x128b_warpx4(tmem_base + kTmemSfB + 4, sf + kSfABytes + 512);
-          const uint64_t a_desc = ptx::smem_desc_sw128(sa);
-          const uint64_t b_desc = ptx::smem_desc_sw128(sa + kABytes);
+          return true;
+        };
+        // Swapped operands for a block of few rows: each 128-row weight box is the M side (its scales, the second and
+        // third 512-byte group of the stage, are the A scales), the block's rows padded to 16 the N side (their
+        // scales, the first group, the B scales); box 0 accumulates into columns 0.., box 1 into columns 128...
+        auto swapped = [&](auto rows_tag) -> bool {
+          constexpr int kRows = decltype(rows_tag)::value;
+          return k_loop([&](uint32_t sa, uint32_t later) {
+            const uint64_t r_desc = ptx::smem_desc_sw128(sa), w0_desc = ptx::smem_desc_sw128(sa + kABytes),
+                           w1_desc = ptx::smem_desc_sw128(sa + kABytes + kBBoxBytes);
 #pragma unroll
-          for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
-            const uint64_t adv = static_cast<uint64_t>(2 * k4);   // +32 bytes along K inside the swizzle row
-            ptx::tc_mma_mx(d_tmem, a_desc + adv, b_desc + adv, ptx::idesc_mx_e4m3(BM, BN, k4, k4),
-                           tmem_base + kTmemSfA, tmem_base + kTmemSfB, (kb | k4) != 0 ? 1u : 0u);
-          }
-          ptx::tc_commit(ptx::smem_u32(&st->empty[stage]));   // codes and scales are free once these are done
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
+              const uint64_t adv = static_cast<uint64_t>(2 * k4);
+              const uint32_t accum = k4 != 0 ? 1u : later;
+              ptx::tc_mma_mx(d_tmem, w0_desc + adv, r_desc + adv, ptx::idesc_mx_e4m3(BNH, kRows, k4, k4),
+                             tmem_base + kTmemSfB, tmem_base + kTmemSfA, accum);
+              ptx::tc_mma_mx(d_tmem + BNH, w1_desc + adv, r_desc + adv, ptx::idesc_mx_e4m3(BNH, kRows, k4, k4),
+                             tmem_base + kTmemSfB + 4, tmem_base + kTmemSfA, accum);
+            }
+          });
+        };
+        switch (n_pad >> 4) {
+          case 0:
+            ok = k_loop([&](uint32_t sa, uint32_t later) {
+              const uint64_t a_desc = ptx::smem_desc_sw128(sa), b_desc = ptx::smem_desc_sw128(sa + kABytes);
+#pragma unroll
+              for (int k4 = 0; k4 < BK / UMMA_K; ++k4) {
+                const uint64_t adv = static_cast<uint64_t>(2 * k4);   // +32 bytes along K inside the swizzle row
+                ptx::tc_mma_mx(d_tmem, a_desc + adv, b_desc + adv, ptx::idesc_mx_e4m3(BM, BN, k4, k4),
+                               tmem_base + kTmemSfA, tmem_base + kTmemSfB, k4 != 0 ? 1u : later);
+              }
+            });
+            break;
+          case 1: ok = swapped(std::integral_constant<int, 16>{}); break;
+          case 2: ok = swapped(std::integral_constant<int, 32>{}); break;
+          case 3: ok = swapped(std::integral_constant<int, 48>{}); break;
+          default: ok = swapped(std::integral_constant<int, 64>{}); break;
         }
         if (!ok) break;
         ptx::tc_commit(ptx::smem_u32(&st->tmem_full[acc]));
         if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
         ++n_tiles;
+        if (n_pad != 0) {
+          ++n_swapped;
+          t_swapped += clock64() - t_tile;
+        } else {
+          t_plain += clock64() - t_tile;
+        }
       }
       if (p.trace) {
         p.trace[blockIdx.x * kMoeTraceFields + 2] = static_cast<unsigned long long>(w_full);
         p.trace[blockIdx.x * kMoeTraceFields + 3] = static_cast<unsigned long long>(w_tmem);
         p.trace[blockIdx.x * kMoeTraceFields + 6] = n_tiles;
+        p.trace[blockIdx.x * kMoeTraceFields + 8] = n_swapped;
+        p.trace[blockIdx.x * kMoeTraceFields + 9] = static_cast<unsigned long long>(t_swapped);
+        p.trace[blockIdx.x * kMoeTraceFields + 11] = static_cast<unsigned long long>(t_plain);
       }
     }
     __syncwarp();
@@ -291,7 +345,48 @@ expert_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(empty_bar);
       };
-      if constexpr (kGated) {
+      if (tile.n_pad != 0) {
+        // Swapped operands: this thread's lane is output column n0 + f (and n0 + 128 + f for Linear-2's second weight
+        // box), accumulator column j is row row0 + j.  Few rows: the first four warps drain them all, the other four
+        // only hand the accumulator back.  In Linear-1 the 32 lanes of a warp hold one 32-element block of h of a row,
+        // so the block's maximum is a warp reduction and every lane converts and stores its own code byte: the same
+        // bits as the per-thread quantisation of the 128-row tiles (maximum and conversion do not depend on order).
+        if (half == 1) {
+          release();
+        } else {
+          const int f = quarter * 32 + lane;
+          const int col_a = tile.n0 + f, col_b = col_a + BNH;
+#pragma unroll 1
+          for (int j0 = 0; j0 < tile.n_pad; j0 += 16) {
+            uint32_t va[16], vb[16];
+            ptx::tmem_ld_32x16(t_addr + j0, va);
+            ptx::tmem_ld_32x16(t_addr + BNH + j0, vb);
+            ptx::tmem_ld_wait();
+            if (j0 + 16 >= tile.n_pad) release();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int r = tile.row0 + j0 + i;
+              if (r >= tile.row_end) continue;          // (the same for every lane of the warp)
+              const float a = __uint_as_float(va[i]), b = __uint_as_float(vb[i]);
+              if constexpr (kGated) {
+                const float hv = silu_mul(a, b);
+                const uint32_t amax_bits = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(fabsf(hv)));
+                const uint32_t byte = mx::scale_byte(__uint_as_float(amax_bits));
+                const unsigned char code = static_cast<unsigned char>(
+                    __nv_cvt_float_to_fp8(hv * mx::inverse_scale(byte), __NV_SATFINITE, __NV_E4M3));
+                if (col_a < p.N) {                      // N is a multiple of 32: a warp's block is inside or outside
+                  reinterpret_cast<unsigned char*>(p.hq)[static_cast<size_t>(r) * p.N + col_a] = code;
+                  if (lane == 0) p.sf_h[mx::scale_byte_index(p.a_rows, r, col_a >> 5)] = static_cast<unsigned char>(byte);
+                  if (p.h_dbg != nullptr) p.h_dbg[static_cast<size_t>(r) * p.N + col_a] = hv;
+                }
+              } else {
+                if (col_a < p.N) p.y[static_cast<size_t>(r) * p.N + col_a] = __float2bfloat16_rn(a);
+                if (col_b < p.N) p.y[static_cast<size_t>(r) * p.N + col_b] = __float2bfloat16_rn(b);
+              }
+            }
+          }
+        }
+      } else if constexpr (kGated) {
         // this warp's blocks of 32 h columns (N is a multiple of 32: blocks are whole); the accumulator is handed
         // back right after the warp's last load from tensor memory, before that block is processed and stored
         const int jb = half * (BNH / 64);
@@ -489,6 +584,8 @@ moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, cudaStre
   p1.status = ctx->d_status;
   p1.trace = ctx->timing ? ctx->d_trace : nullptr;   // per-kernel timing also turns the wait counters on
   p1.cache_hints = moe_knob_value(ctx, "cache_hints", 35);
+  p1.swap_rows = moe_knob_value(ctx, "mx_swap_rows", kMxSwapRows);
+  if (p1.swap_rows < 0 || p1.swap_rows > kMxSwapRows) p1.swap_rows = kMxSwapRows;
 
   MxParams p2{};
   p2.offsets = p1.offsets;
@@ -504,6 +601,7 @@ moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, cudaStre
   p2.y = static_cast<__nv_bfloat16*>(a->y_perm);
   p2.status = ctx->d_status;
   p2.cache_hints = p1.cache_hints;
+  p2.swap_rows = p1.swap_rows;
   p2.trace = ctx->timing ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
 
   const int grid = ctx->num_sms;
