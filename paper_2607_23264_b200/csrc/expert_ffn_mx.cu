@@ -19,6 +19,10 @@
 // stored in the 512-byte layout tcgen05.cp expects, then a proxy fence and an arrival on the stage's full barrier),
 // warp 1 = MMA issuer (per stage: three tcgen05.cp of scales into tensor memory, then four MMAs picking scale byte
 // 0..3), warps 2-5 and 10-13 = epilogue.  Four stages of 49.5 KB.
+// An expert of at most 64 rows is computed with swapped operands (weight box = M side, its rows padded to 16 = N
+// side, the scale groups change roles with them): fewer multiply-adds on padding rows, which under the power cap is
+// worth more than the clocks the extra instructions cost.  TMA loads carry L2 eviction priorities: weights only this
+// tile reads go first, rows of A and weights other row blocks read again stay.
 // Every wait is bounded; a wait that gives up is reported through the status word and the CTA unwinds.
 #include <cuda_bf16.h>
 
