@@ -471,8 +471,10 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     // share the weight boxes of a stage, a third less to bring into shared memory per flop, which is what holds
     // these tiles back when the weights of many experts stream through L2 at once.
     // The price is one stage of the ring (three stages of 64 KiB), which the one-block tiles of small experts feel
-    // (they stream weights and live on the bytes in flight), so wide mode needs them to be few: at most a fifth of
-    // the launch's tiles.
+    // (they stream weights and live on the bytes in flight), so wide mode needs enough many-row work to pay for
+    // it: at least three 256-row blocks for every four single-block experts.  (Measured in steady state on the
+    // DeepSeek-V3-like layer at 1024 to 16384 tokens, where that ratio runs from 0.31 to 3.4: +3 %, -0.7 %, -3.1 %,
+    // -5.2 %, -6.3 % with wide mode; the crossover lies near 0.5.)
     int hot_wide_blocks = 0, cold_blocks = 0;
     for (int base = 0; base < p.E; base += 32) {
       const int e = base + lane;
@@ -482,7 +484,10 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     }
     hot_wide_blocks = __reduce_add_sync(0xFFFFFFFFu, hot_wide_blocks);
     cold_blocks = __reduce_add_sync(0xFFFFFFFFu, cold_blocks);
-    const bool wide_mode = p.wide_allowed != 0 && hot_wide_blocks > 0 && (4 * cold_blocks <= hot_wide_blocks || p.wide_allowed == 2);
+    // (E4M3 operands: the weight-streaming tiles are a larger share of the time there, and on the same layer wide mode
+    // costs 2 % at 4096 tokens; they keep the stricter rule of four 256-row blocks per single-block expert.)
+    const bool enough_hot = p.fp8 ? 4 * cold_blocks <= hot_wide_blocks : 3 * cold_blocks <= 4 * hot_wide_blocks;
+    const bool wide_mode = p.wide_allowed != 0 && hot_wide_blocks > 0 && (enough_hot || p.wide_allowed == 2);
     if (lane == 0) st->wide = wide_mode ? 1 : 0;
     // exclusive prefixes of the row-block counts over experts (hot and cold apart), 32 experts per step
     int32_t run_hot = 0, run_cold = 0;
