@@ -32,16 +32,17 @@ from paper_2607_23264_b200 import inputs as gen  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-def dram_traffic_per_expert(kernel: str):
-    """ncu DRAM bytes (read + write) of one Linear-1 launch, per non-empty expert, for `kernel`, from the committed
-    summary of the capture (a table row per kernel: name | case | experts | dram read bytes | dram write bytes).
-    None when the summary or the row is missing."""
+def dram_traffic_per_expert(kernel: str, H: int, F: int):
+    """ncu DRAM bytes (read + write) of one Linear-1 launch, per non-empty expert, for `kernel` on experts of shape
+    H x F, from the committed summary of the captures (a table row per kernel and expert shape: name | case |
+    experts | dram read bytes | dram write bytes; the case names its "H=..., F=...").  None when the summary or the
+    row is missing."""
     path = os.path.join(ROOT, "profiles", "linear1_dram_traffic.md")
     try:
         with open(path) as fh:
             for line in fh:
                 cells = [c.strip() for c in line.strip().strip("|").split("|")]
-                if len(cells) >= 5 and cells[0].strip("`") == kernel:
+                if len(cells) >= 5 and cells[0].strip("`") == kernel and f"H={H}, F={F}" in cells[1]:
                     experts, rd, wr = int(cells[2]), int(cells[3].replace(",", "")), int(cells[4].replace(",", ""))
                     return (rd + wr) / experts
     except (OSError, ValueError):
@@ -588,11 +589,11 @@ def main():
         l1_bytes, l2_bytes = l1_bytes + l2_bytes, 0
     l1_gbs = l1_bytes / (kernel_ms[4] * 1e-3) / 1e9
     l2_gbs = 0.0 if one_launch else l2_bytes / (kernel_ms[5] * 1e-3) / 1e9
-    pair_kernel = not one_launch and (args.pairs == "on" or (args.pairs == "auto" and cfg.R // cfg.E >= 1024))
+    pair_kernel = not one_launch and args.pairs == "on"      # "auto": the library's default, the single-CTA kernel
     kernel_symbol = "expert_ffn_pair_kernel<false>" if pair_kernel else "expert_ffn_kernel<false>"
     gemm_name = (kernel_symbol + " (Linear-1 + SiLU*mul + Linear-2, one launch)" if one_launch
                  else kernel_symbol + ", Linear-1 + SiLU*mul launch")
-    per_expert = None if one_launch else dram_traffic_per_expert(kernel_symbol)
+    per_expert = None if one_launch else dram_traffic_per_expert(kernel_symbol, cfg.H, cfg.F)
     traffic = None if per_expert is None else per_expert * nonempty
     # the roofline that binds Linear-1: tensor time at the measured GEMM peak vs HBM time at the measured copy rate
     t_tensor = l1_flops / (peak_tf_burst * 1e12)

@@ -80,9 +80,11 @@ typedef struct {
                                       tiles fit in about one wave of CTAs always do); bit 2: failure drill, requested
                                       by the host: runs as one launch in which Linear-1 never publishes its rows, so
                                       every Linear-2 wait expires (after about 0.1 s), the kernel unwinds and the
-                                      status word reads MOE_ERR_TIMEOUT; outputs are then undefined; bit 3: always use
-                                      the CTA-pair kernel for two-launch runs, bit 4: never use it (by default it
-                                      runs when the layer averages at least 1024 rows per expert); other bits 0 */
+                                      status word reads MOE_ERR_TIMEOUT; outputs are then undefined; bit 3: use the
+                                      CTA-pair kernel (clusters of two CTAs on 256-row tiles) for two-launch runs; by
+                                      default every layer runs the single-CTA kernel, which cuts many-row experts
+                                      into 256-row tiles on its two accumulators; bit 4: accepted, no effect (it
+                                      used to switch the pair kernel off); other bits 0 */
 } moe_tuning;
 
 /*

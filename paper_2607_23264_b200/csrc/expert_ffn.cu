@@ -30,7 +30,7 @@
 // side and the expert's rows, padded to a multiple of 16, its N side.  A tcgen05.mma costs 128 clocks at N = 256 but
 // 46 at N <= 32, so the two instructions per K step (one per weight box) take 92 clocks instead of 128; the
 // shared-memory stage is the same three boxes, only the MMA issue and the epilogue (lane = output column) differ.
-// Layers whose experts hold many rows run the CTA-pair variant further down (256-row tiles, cta_group::2).
+// A CTA-pair variant (256-row tiles over a cluster of two CTAs, cta_group::2) follows further down; it runs on request.
 #include <cuda_bf16.h>
 
 #include <type_traits>
@@ -916,7 +916,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 
 
 // ------------------------------------------------------------------------------------------------------------
-// CTA-pair variant for layers whose experts hold many rows: a cluster of two CTAs computes a 256-row x 256-column
+// CTA-pair variant (on request: debug_flags bit 3) for layers whose experts hold many rows: a cluster of two CTAs computes a 256-row x 256-column
 // tile with tcgen05.mma.cta_group::2.  Each CTA loads its own 128 rows of A and one 128-row weight box (for
 // Linear-1 the leader holds the gate box, its peer the up box), so a stage is 32 KiB per CTA instead of 48 and
 // six stages fit; the leader's MMA thread issues for both, reading the peer's operands from the peer's shared
@@ -1445,10 +1445,12 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   const long long max_blocks = static_cast<long long>(R / 128) + s.E;
   const bool tiny = max_blocks * (p.ph[0].n_blocks + p.ph[1].n_blocks) <= 2LL * grid;
   const bool one_launch = !split && (tn.schedule == 1 || (tn.debug_flags & 6) != 0 || tiny);
-  // CTA pairs (256-row tiles) pay off when experts hold many rows; single-block experts would waste the peer.
-  const bool dense = R / static_cast<uint64_t>(s.E) >= 1024;
-  const bool pairs = !one_launch && ctx->max_pairs > 0 &&
-                     ((tn.debug_flags & 8) != 0 || (dense && (tn.debug_flags & 16) == 0));
+  // The CTA-pair kernel runs on request only.  It used to be the default for layers averaging 1024 rows per expert or
+  // more; since the TMA loads carry L2 eviction priorities the single-CTA kernel with 256-row tiles is the faster one
+  // there as well (Mixtral-like layer, steady state: -1.6 to -4 % at 8192 tokens, -6 % at 4096, -9 % at 16384; burst
+  // equal): it computes an expert's remainder rows as a 128-row or swapped-operand tile instead of a whole 256-row
+  // tile, draws tiles dynamically instead of in rounds, and holds a higher SM clock under the power cap.
+  const bool pairs = !one_launch && ctx->max_pairs > 0 && (tn.debug_flags & 8) != 0;
   unsigned long long* trace2 = trace ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
 
   if (one_launch) {
