@@ -1467,8 +1467,15 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
   }
   // two separate launches: many-row experts may run as 256-row tiles (decided in the kernel from the row counts)
-  p.wide_allowed = moe_knob_value(ctx, "wide_tiles", 1);   // 0 never, 1 by the kernel's rule, 2 whenever an expert has several blocks
+  const int wide_knob = moe_knob_value(ctx, "wide_tiles", 1);   // 0 never, 1 by the kernel's rule, 2 whenever an expert has several blocks
+  // Which GEMMs may use them (bit 0 Linear-1, bit 1 Linear-2).  A 256-row tile holds both accumulators, so the next
+  // tile waits for the drain of the first; with E4M3 operands the mainloop is half as long and that wait weighs twice
+  // as much in Linear-1 (gated epilogue): there 256-row tiles pay in Linear-2 only (Mixtral-like layer, per-row FP8,
+  // steady state: 3.07 against 3.18-3.24 ms with both, 3.22-3.23 with Linear-1 only); bf16 gains from both (4.85-4.89
+  // against 5.05-5.13 ms with either one alone).
+  const int wide_phases = moe_knob_value(ctx, "wide_phases", c.fp8 ? 2 : 3);
   if (!second_phase_only) {
+    p.wide_allowed = (wide_phases & 1) ? wide_knob : 0;
     p.phase_lo = 0;
     p.phase_hi = 1;
     p.sched = ctx->d_sched;
@@ -1483,6 +1490,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     ctx->last_launches += 1;
   }
   if (!first_phase_only) {
+    p.wide_allowed = (wide_phases & 2) ? wide_knob : 0;
     p.phase_lo = 1;
     p.phase_hi = 2;
     p.sched = ctx->d_sched + 2;
