@@ -1050,8 +1050,8 @@ def run_sweep(args, cfg, ctx, binding, bufs, timed, rank):
     The GPU is first brought to its steady power-capped state (about 1.5 s of steps); every point is then
     timed in two passes (forward and reverse order) so that clock drift shows up as spread, not as a trend.
     Per point: median/min ms per step, TFLOP/s, algorithmic HBM GB/s, per-kernel times, and from one traced step
-    the share of each GEMM's span its tensor pipe was busy (MMA instructions issued x the 128 clocks the pipe needs
-    for one, over the CTA's span), the Linear-2 per-tile epilogue store span, pacing hold and MMA wait for a free
+    the share of each GEMM's span its tensor pipe did useful work (the GEMM's multiply-adds over the 4096 per clock
+    and SM the pipe can do, over the launch's mean CTA span), the Linear-2 per-tile epilogue store span, pacing hold and MMA wait for a free
     accumulator (SM clocks), and how many CTAs held stores at all."""
     import torch
     x, d_logits, w_gate, w_up, w_down, out, ws = bufs
@@ -1088,7 +1088,10 @@ def run_sweep(args, cfg, ctx, binding, bufs, timed, rank):
                 for gi in (0, 1):
                     issuing = tr[gi][:, 6] > 0           # CTAs whose MMA warp issued (in a CTA pair: the leader)
                     span = np.maximum(tr[gi][issuing, 0], 1.0)
-                    pipe.append(float((tr[gi][issuing, 6] * k_blocks[gi] * 4 * 128 / span).mean()) if issuing.any() else 0.0)
+                    # useful multiply-adds of the GEMM over what the launch's SMs could issue in its span (an SM's tensor
+                    # pipe does 128 x 256 x 16 bf16 multiply-adds in 128 clocks = 4096 per clock); padded rows not counted
+                    macs = (2 if gi == 0 else 1) * cfg.R * cfg.H * cfg.F
+                    pipe.append(float(macs / (tr[gi].shape[0] * 4096.0 * span.mean())) if issuing.any() else 0.0)
                 l2 = tr[1].mean(axis=0)
                 tiles = max(tr[1][:, 6].sum() / max((tr[1][:, 5] > 0).sum(), 1), 1.0)   # tiles per draining CTA
                 extra[pt] = {"linear1_ms": km[4], "linear2_ms": km[5], "identical_bits": bool(torch.equal(bits, base)),
