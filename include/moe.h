@@ -455,7 +455,8 @@ int32_t moe_last_launch_count(const moe_ctx* ctx);
  * wait), 4 epilogue waited for a finished accumulator, 5 epilogue drain-and-store span, 6 tiles processed
  * (a count), 7 epilogue held by the pacing gap, 8 tiles computed with swapped operands (a count), 9 the MMA
  * warp's time in those tiles, 10 the part of it spent waiting for operands, 11 its time in the other tiles
- * (8-11: single-CTA bf16/E4M3 kernel only, zero elsewhere).  This call synchronises `stream` and copies
+ * (8-11: the single-CTA bf16/E4M3 kernel; the block-scaled FP8 kernel, whose counters moe_expert_ffn_mx records
+ * while per-kernel timing is enabled, writes 8, 9 and 11; zero in the CTA-pair kernel).  This call synchronises `stream` and copies
  * counters_host[2][*num_ctas][12] (Linear-1 first) to HOST memory; capacity is in 64-bit elements and must be
  * at least 24 * (number of SMs).
  */
