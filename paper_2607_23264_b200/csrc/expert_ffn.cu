@@ -1057,11 +1057,12 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       bool ok = true;
       long long w_empty = 0;
       const long long t_begin = clock64();
-      // L2 priorities (bits of cache_hints): 8 = the rows of A stay (they are read once per column block),
-      // 16 = the weight boxes go first (the row blocks that read a box run at about the same time)
+      // L2 priorities (bits of cache_hints): 8 = the rows of A stay (they are read once per column block), 64 = the
+      // weight boxes stay (every row block of the expert reads them), 16 = the weight boxes go first
       const uint64_t pol_a = ((p.cache_hints & 8) && (phase == 1 || !(p.cache_hints & 4))) ? ptx::l2_policy_evict_last()
                                                                                           : ptx::l2_policy_evict_normal();
-      const uint64_t pol_w = (p.cache_hints & 16) ? ptx::l2_policy_evict_first() : ptx::l2_policy_evict_normal();
+      const uint64_t pol_w = (p.cache_hints & 16) ? ptx::l2_policy_evict_first()
+                             : (p.cache_hints & 64) ? ptx::l2_policy_evict_last() : ptx::l2_policy_evict_normal();
       for (int tile = pair; ok && tile < total_tiles; tile += pairs) {
         const Tile t = decode_pair_tile(tile, phase, rank, st, p);
         for (int kb = 0; kb < d.k_blocks; ++kb) {
@@ -1442,10 +1443,10 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   // of the expert reads them again) and so do the weights of experts with several row blocks (bit 5: each of those
   // blocks reads them).  Measured in the power-capped steady state: bits 0 and 1 -6 % on the decode-like layer and
   // -3.7 % on the DeepSeek-V3-like one; bit 5 another -1.2 % there and -1 to -2 % on the Mixtral-like layer at 1024 to
-  // 3072 tokens.  Bit 2 restricts bit 1 to Linear-2; bits 3 and 4 are the priorities of bits 1 and 0 in the CTA-pair
-  // kernel, where they do not pay (A rows: no change; weights first: 17 % slower, the row blocks that share a weight
-  // box do not run closely enough together).
-  p.cache_hints = moe_knob_value(ctx, "cache_hints", 35);
+  // 3072 tokens.  Bit 2 restricts bit 1 to Linear-2.  In the CTA-pair kernel bit 3 = rows of A stay, bit 6 = weights
+  // stay (together -3 % on the Mixtral-like layer, both on by default), bit 4 = weights go first (17 % slower: the row
+  // blocks that share a weight box do not run closely enough together).
+  p.cache_hints = moe_knob_value(ctx, "cache_hints", 35 | 8 | 64);
   // Swapped-operand tiles of at most 16 rows (most tiles of a decode-like batch) load those rows as one 16-row box
   // instead of a 128-row box of mostly other experts' rows: a third less to move per K block; -1 % on the decode-like
   // layer, -0.4 % on the DeepSeek-V3-like one in steady state (larger row counts, several boxes per K block: no gain).

@@ -587,7 +587,7 @@ moe_status launch_expert_ffn_mx(moe_ctx* ctx, const moe_mx_ffn_args* a, cudaStre
   p1.h_dbg = a->h_fp32_debug;
   p1.status = ctx->d_status;
   p1.trace = ctx->timing ? ctx->d_trace : nullptr;   // per-kernel timing also turns the wait counters on
-  p1.cache_hints = moe_knob_value(ctx, "cache_hints", 35);
+  p1.cache_hints = moe_knob_value(ctx, "cache_hints", 35 | 8 | 64);   // (this kernel reads bits 0, 1 and 5)
   p1.swap_rows = moe_knob_value(ctx, "mx_swap_rows", kMxSwapRows);
   if (p1.swap_rows < 0 || p1.swap_rows > kMxSwapRows) p1.swap_rows = kMxSwapRows;
 
