@@ -254,6 +254,32 @@ def test_environment_override_of_the_default_tuning(monkeypatch):
     assert ei.value.code == 1
 
 
+def test_development_knobs_do_not_change_values(monkeypatch):
+    """The development knobs of MOE_TUNING choose between ways of computing the same tiles (256-row tiles on or off or
+    in one GEMM only, swapped operands up to 128 rows, 16-row boxes of A for larger tiles, L2 priorities off, the
+    CTA-pair kernel): every setting gives the bits of the default, on a layer of many-row experts and on a skewed one."""
+    settings = ("x.wide_tiles=0", "x.wide_tiles=2", "x.wide_phases=1", "x.wide_phases=2", "x.small_a=64,x.swap_rows=128",
+                "x.small_a=0,x.swap_rows=16", "x.cache_hints=0", "flags=8")
+    for cfg in (gen.MoEConfig("knobs_dense", T=2000, H=512, F=1024, E=6, k=2, seed=91, router="xWr"),
+                gen.MoEConfig("knobs_skew", T=1500, H=512, F=512, E=24, k=4, seed=92, router="xWr_zipf")):
+        monkeypatch.delenv("MOE_TUNING", raising=False)
+        base_layer = Layer(cfg)
+        ws = torch.empty(base_layer.ctx.workspace_bytes(), dtype=torch.uint8, device=DEV)
+        base = base_layer.nan_bf16(cfg.T, cfg.H)
+        base_layer.ctx.moe_fused_forward(base_layer.x, base_layer.d_logits, base_layer.w_gate, base_layer.w_up,
+                                         base_layer.w_down, base, ws)
+        torch.cuda.synchronize()
+        assert_out_close(dev_bf16_to_f64(base), oracle_for(base_layer)["out"], f"out[{cfg.name}]")
+        for setting in settings:
+            monkeypatch.setenv("MOE_TUNING", setting)
+            L = Layer(cfg)
+            out = L.nan_bf16(cfg.T, cfg.H)
+            L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws)
+            torch.cuda.synchronize()
+            L.check_device_status()
+            assert torch.equal(out.view(torch.int16), base.view(torch.int16)), (cfg.name, setting)
+
+
 def test_debug_check_refuses_non_finite_logits(monkeypatch):
     """Non-finite logits violate the routing contract and are not tested on the device; the debug entry
     x.check_logits=1 of MOE_TUNING tests them on the host and returns MOE_ERR_BAD_ROUTING before any launch."""
