@@ -103,7 +103,12 @@ def test_quantize_rows_mx_bits(rows, cols):
     (129, 256, 640, 16, 4, "xWr_zipf"), # skewed: empty experts, experts of one row
     (5, 384, 256, 6, 6, "xWr"),         # k = E, five rows per expert
 ])
-def test_expert_ffn_mx_parity(T, H, F, E, k, router):
+@pytest.mark.parametrize("swapped", [True, False], ids=["swapped_small_experts", "128_row_tiles_only"])
+def test_expert_ffn_mx_parity(T, H, F, E, k, router, swapped, monkeypatch):
+    """Experts of at most 64 rows run with swapped operands by default (h quantised with a warp-wide block maximum);
+    the development knob switches that off, and both ways must give the oracle's codes and values."""
+    if not swapped:
+        monkeypatch.setenv("MOE_TUNING", "x.mx_swap_rows=0")
     cfg = small_cfg(T, H, F, E, k, seed=T + H, router=router)
     M = MxLayer(cfg)
     L, ctx = M.L, M.L.ctx
