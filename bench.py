@@ -530,7 +530,7 @@ def main():
     # (8192^3, back to back for 2 s after 1 s of the same) on the GPU at hand.  GPUs of one pool hold different clocks
     # at the same 1 kW cap; this says how the GPU of this run compares with the one the peaks were taken on.  The
     # roofline's `peak` stays the file's figure.
-    local_peak = None
+    local_peak, library_grouped_ms = None, None
     if rank == 0 and world == 1 and not args.no_local_peak and not args.profile:
         n = 8192
         ga = torch.randn((n, n), device=dev, dtype=torch.float32).to(torch.bfloat16)
@@ -553,6 +553,40 @@ def main():
         torch.cuda.synchronize()
         local_peak = 2.0 * n ** 3 * count / (g0.elapsed_time(g1) * 1e-3) / 1e12
         del ga, gb, gc
+        # and the layer's own two grouped GEMMs as library calls, one per expert and weight matrix, on the very tensors
+        # of the last step (x_perm, h and the expert row ranges in the workspace; no SiLU*mul): layers of few experts only
+        if cfg.E <= 16:
+            lay = ctx.workspace_layout()
+            offs = ws[lay["offsets"]:lay["offsets"] + 4 * (cfg.E + 1)].view(torch.int32).cpu().numpy().astype(np.int64)
+            xp = ws[lay["x_perm"]:lay["x_perm"] + cfg.R * cfg.H * 2].view(torch.bfloat16).view(cfg.R, cfg.H)
+            hp = ws[lay["h"]:lay["h"] + cfg.R * cfg.F * 2].view(torch.bfloat16).view(cfg.R, cfg.F)
+            lg = torch.empty((cfg.R, cfg.F), dtype=torch.bfloat16, device=dev)
+            lu = torch.empty((cfg.R, cfg.F), dtype=torch.bfloat16, device=dev)
+            ly = torch.empty((cfg.R, cfg.H), dtype=torch.bfloat16, device=dev)
+            spans = [(e, int(offs[e]), int(offs[e + 1])) for e in range(cfg.E) if offs[e + 1] > offs[e]]
+
+            def library_gemms():
+                for e, lo, hi in spans:
+                    torch.matmul(xp[lo:hi], w_gate[e].t(), out=lg[lo:hi])
+                    torch.matmul(xp[lo:hi], w_up[e].t(), out=lu[lo:hi])
+                for e, lo, hi in spans:
+                    torch.matmul(hp[lo:hi], w_down[e].t(), out=ly[lo:hi])
+
+            t_heat = time.time()
+            while time.time() - t_heat < 1.0:
+                library_gemms()
+                torch.cuda.synchronize()
+            count, t_run = 0, time.time()
+            g0.record(stream)
+            while time.time() - t_run < 1.5:
+                for _ in range(5):
+                    library_gemms()
+                count += 5
+                torch.cuda.synchronize()
+            g1.record(stream)
+            torch.cuda.synchronize()
+            library_grouped_ms = g0.elapsed_time(g1) / count
+            del lg, lu, ly
 
     if rank != 0:
         if dist.is_initialized():
@@ -634,7 +668,13 @@ def main():
             "bf16_tflops_sustained_this_gpu": local_peak,
             "how": "torch.matmul bf16 8192^3 back to back for 2 s after 1 s of the same, after all timed regions",
             "of_measured_peaks_file": local_peak / float(peaks.get("bf16_tflops_sustained") or float("nan")),
-            **({"frac_of_this_gpu": roofline["achieved"] / local_peak} if roofline["bound"] == "tensor" else {})}
+            **({"frac_of_this_gpu": roofline["achieved"] / local_peak} if roofline["bound"] == "tensor" else {}),
+            **({"grouped_gemms_as_library_calls_ms": library_grouped_ms,
+                "grouped_gemms_this_build_ms": kernel_ms[4] + kernel_ms[5],
+                "grouped_how": "torch.matmul per expert and weight matrix on the step's own x_perm, h and expert row "
+                               "ranges (no SiLU*mul), back to back for 1.5 s after 1 s of the same; this build's figure "
+                               "is its two GEMM kernels in the steady region"}
+               if library_grouped_ms is not None else {})}
     burst_ms_per_step = burst_total_ms / args.steps
     line = {
         "metric": "fused MoE fwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
