@@ -116,6 +116,17 @@ def test_fused_forward_fp8_parity(cfg):
     assert rel_fro(dev_bf16_to_f64(out), full["out"]) < 0.08
 
 
+def test_fused_forward_fp8_random_layers():
+    """The same checks on random layers: ragged and empty experts, one to thousands of rows per expert."""
+    rng = np.random.default_rng(8)
+    for trial in range(6):
+        E = int(rng.integers(1, 5)) if trial % 2 else int(rng.integers(5, 30))
+        cfg = gen.random_small_config(rng, T=int(rng.integers(1, 3000)), E=E, k=int(rng.integers(1, min(E, 8) + 1)),
+                                      H=128 * int(rng.integers(1, 5)), F=128 * int(rng.integers(1, 5)),
+                                      router="xWr_zipf" if trial % 3 == 0 else "xWr")
+        test_fused_forward_fp8_parity(cfg)
+
+
 def test_fp8_rejects_unsupported_requests():
     ctx = binding.Context(16, 192, 128, 2, 1)          # H not a multiple of 128
     with pytest.raises(binding.MoeError) as ei:

@@ -201,6 +201,17 @@ def test_fused_forward_mx_and_sampled_rows_at_full_k():
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
 
 
+def test_expert_ffn_mx_random_layers(monkeypatch):
+    """The same checks on random layers, with and without swapped-operand tiles for the small experts."""
+    rng = np.random.default_rng(14)
+    for trial in range(6):
+        E = int(rng.integers(1, 5)) if trial % 2 else int(rng.integers(5, 30))
+        k = int(rng.integers(1, min(E, 8) + 1))
+        monkeypatch.delenv("MOE_TUNING", raising=False)
+        test_expert_ffn_mx_parity(int(rng.integers(1, 2500)), 128 * int(rng.integers(1, 5)), 128 * int(rng.integers(1, 6)),
+                                  E, k, "xWr_zipf" if trial % 3 == 0 else "xWr", trial % 4 != 3, monkeypatch)
+
+
 def test_mx_rejects_shapes_it_cannot_tile():
     ctx = binding.Context(16, 192, 128, 2, 1)       # H is not a multiple of 128
     t = torch.zeros(64, dtype=torch.uint8, device=DEV)

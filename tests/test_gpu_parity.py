@@ -542,6 +542,38 @@ def test_random_small_layers_property():
         L.check_device_status()
 
 
+def test_random_mid_size_layers_property():
+    """Random layers of up to 5000 tokens on few or many experts: several hundred to a few thousand rows per expert
+    (256-row tiles on both accumulators, the merged order of many-row and few-row experts, swapped-operand remainders),
+    through the default path, the CTA-pair kernel, the interleaved schedule and a paced store; all bitwise equal."""
+    rng = np.random.default_rng(77)
+    for trial in range(10):
+        few = trial % 2 == 0
+        E = int(rng.integers(1, 5)) if few else int(rng.integers(5, 40))
+        cfg = gen.random_small_config(rng, T=int(rng.integers(1500, 5000)), E=E, k=int(rng.integers(1, min(E, 8) + 1)),
+                                      H=64 * int(rng.integers(1, 9)), F=64 * int(rng.integers(1, 9)),
+                                      router="xWr" if few else "xWr_zipf")
+        L = Layer(cfg)
+        ref = oracle_for(L)
+        lay = L.ctx.workspace_layout()
+        ws = torch.empty(lay["total"], dtype=torch.uint8, device=DEV)
+        outs = []
+        for tn in (None, binding.make_tuning(1, 0, 1, debug_flags=8),
+                   binding.make_tuning(1, 0, 1, schedule=1, dep_lead_D=1 + trial % 3),
+                   binding.make_tuning([2, 4, 8, 16][trial % 4], 1, [1, 2, 4][trial % 3])):
+            out = L.nan_bf16(cfg.T, cfg.H)
+            L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws, tuning=tn)
+            torch.cuda.synchronize()
+            outs.append(out)
+        what = f"trial {trial}: {cfg}"
+        perm = ws[lay["perm"]:lay["perm"] + 4 * cfg.R].view(torch.int32).cpu().numpy()
+        assert np.array_equal(perm, ref["perm"]), what
+        assert_out_close(dev_bf16_to_f64(outs[0]), ref["out"], what)
+        for o in outs[1:]:
+            assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16)), what
+        L.check_device_status()
+
+
 def test_smaller_batches_on_one_context():
     """A context created for T tokens serves any smaller batch (moe_set_active_tokens), with a workspace sized once."""
     cfg = gen.MoEConfig("varT", T=900, H=256, F=384, E=6, k=2, seed=101, router="xWr")
