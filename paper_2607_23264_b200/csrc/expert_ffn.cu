@@ -13,6 +13,10 @@
 // ring of tile codes.
 // Expert row ranges are ragged: a tile may cover rows of the next expert (or past R, zero-filled by
 // TMA); those rows are computed and discarded, stores are masked to the expert's own rows.
+// Stores: an epilogue warp whose 32 rows all belong to the expert packs 64 output columns at a time into a
+// swizzled 4 KiB box of shared memory and one lane hands the box to the TMA unit (whole 128-byte lines, no
+// load/store-unit work per row); a warp with rows of the next expert, a paced run and a launch whose Linear-2 tiles
+// wait for h store 16 bytes per lane and row from registers instead.  Both ways write the same values.
 //
 // Tile orders (moe_tuning.schedule):
 //   0  Expert-Wave: all Linear-1 tiles, then all Linear-2 tiles.  Inside a GEMM the order within an expert is
@@ -84,7 +88,21 @@ struct SharedTail {
   int32_t offs[kMaxExperts + 1];          // the expert row offsets, copied once: tile decoding reads no global memory
 };
 
-constexpr size_t kSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStages) * kStageBytes + sizeof(SharedTail);
+// Staging for the epilogue's bulk tensor stores: per epilogue warp one box of 32 rows x 64 bf16 columns (4 KiB, rows
+// of 128 bytes in the 128-byte swizzle), between the ring and the tail.
+constexpr int kStoreBoxCols = 64;
+constexpr int kStoreBoxBytes = 32 * kStoreBoxCols * 2;
+constexpr int kStoreStagingBytes = 4 * kStoreBoxBytes;
+constexpr size_t kSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStages) * kStageBytes + kStoreStagingBytes +
+                              sizeof(SharedTail);
+static_assert(kSmemBytes + 64 <= 227 * 1024, "ring + store staging + tail must fit in one CTA's shared memory");
+
+// How one epilogue warp stores: smem == 0 = 16-byte stores from registers (each lane its own row); else the warp
+// stages 32 rows x 64 columns there and one lane hands them to the TMA unit as whole 128-byte lines.
+struct StoreStage {
+  uint32_t smem;               // this warp's box (1024-byte aligned), or 0
+  const CUtensorMap* map;      // the [R, N] output in boxes of 32 rows x 64 columns, 128-byte swizzle
+};
 
 struct PhaseDesc {          // one of the two GEMMs
   int N;                    // output columns per row (F for Linear-1, H for Linear-2) = weight rows per expert
@@ -121,6 +139,7 @@ struct FfnParams {
   int wide_allowed;         // the launch may use wide mode (two-launch Expert-Wave runs)
   int cache_hints;          // L2 eviction priorities of the TMA loads, bit mask (see run_ffn)
   int small_a;              // swapped-operand tiles of at most this many padded rows load A in 16-row boxes (0: never)
+  int bulk_stores;          // single-CTA kernel: whole 32-row groups of a tile leave through shared memory and TMA stores
   int withhold_ready;       // host-requested failure drill: Linear-1 never publishes its rows (one-launch runs)
   long long wait_budget;    // clocks a cross-CTA wait may last before it gives up
   int kernel_id;
@@ -274,9 +293,13 @@ __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target,
 // : 256 plain columns, written as bf16 with 16-byte stores masked to the expert's rows and to N.
 template <bool kGated, bool kFp8>
 __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams& p, uint32_t t_addr, int row,
-                                                  Pacer& pacer, volatile int* aborting) {
+                                                  Pacer& pacer, volatile int* aborting, const StoreStage& ss) {
   const PhaseDesc& d = p.ph[kGated ? 0 : 1];
   const bool row_ok = row < t.row_end;
+  const int lane = threadIdx.x & 31;
+  // Bulk stores when all 32 rows of the warp belong to the expert (a box cannot be masked by rows) and the stores
+  // are not paced (a paced store tile is one 32-column chunk)
+  const bool bulk = ss.smem != 0 && p.mode == 0 && p.h_dbg == nullptr && row - lane + 32 <= t.row_end;
   __nv_bfloat16* out_row = d.out + static_cast<size_t>(row) * d.N + t.n0;
   constexpr int kChunks = kGated ? (128 / kChunkCols) : (BN_ACC / kChunkCols);
 #pragma unroll 1
@@ -331,7 +354,30 @@ __device__ __forceinline__ void drain_accumulator(const Tile& t, const FfnParams
       }
     }
     const int col0 = t.n0 + c * kChunkCols;
-    if (row_ok) {
+    if (bulk) {
+      if ((c & 1) == 0) {             // the box is free again once the TMA unit has read the previous one
+        if (lane == 0) ptx::bulk_wait_group_read_all();
+        __syncwarp();
+      }
+      const uint32_t row_smem = ss.smem + static_cast<uint32_t>(lane) * 128u;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t j = static_cast<uint32_t>((c & 1) * 4 + q);          // 16-byte piece of the 128-byte row
+        const uint32_t dst = row_smem + ((j ^ (static_cast<uint32_t>(lane) & 7u)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16(o[q * 8 + 0], o[q * 8 + 1])),
+                     "r"(pack_bf16(o[q * 8 + 2], o[q * 8 + 3])), "r"(pack_bf16(o[q * 8 + 4], o[q * 8 + 5])),
+                     "r"(pack_bf16(o[q * 8 + 6], o[q * 8 + 7]))
+                     : "memory");
+      }
+      if (c & 1) {
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && col0 - kChunkCols < d.N) {   // (a box that starts beyond N has nothing to write)
+          ptx::tma_store_2d(ss.map, ss.smem, col0 - kChunkCols, row);
+          ptx::bulk_commit_group();
+        }
+      }
+    } else if (row_ok) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         if (col0 + q * 8 < d.N) {     // N is a multiple of 8: a 16-byte vector is inside or outside
@@ -436,13 +482,16 @@ __global__ void __launch_bounds__(kThreads, 1)
 expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wg,
                   const __grid_constant__ CUtensorMap tm_wu, const __grid_constant__ CUtensorMap tm_h,
                   const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_x16,
-                  const __grid_constant__ CUtensorMap tm_h16, const FfnParams p) {   // tm_x16, tm_h16: 16-row boxes of A
+                  const __grid_constant__ CUtensorMap tm_h16, const __grid_constant__ CUtensorMap tm_h_out,
+                  const __grid_constant__ CUtensorMap tm_y_out, const FfnParams p) {
+  // tm_x16, tm_h16: 16-row boxes of A; tm_h_out, tm_y_out: the two outputs in boxes of 32 rows x 64 columns (stores)
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   unsigned char* stage_base = smem_raw + pad;                 // 1024-byte aligned: required by the swizzle
   const uint32_t stage_u32 = raw + pad;
-  SharedTail* st = reinterpret_cast<SharedTail*>(stage_base + static_cast<size_t>(kStages) * kStageBytes);
+  const uint32_t store_u32 = stage_u32 + kStages * kStageBytes;
+  SharedTail* st = reinterpret_cast<SharedTail*>(stage_base + static_cast<size_t>(kStages) * kStageBytes + kStoreStagingBytes);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -844,6 +893,10 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     uint32_t ring_phase = 0;
     long long w_acc = 0, busy = 0;
     Pacer pacer{ptx::smem_u32(const_cast<uint32_t*>(&st->mma_progress)), ptx::smem_u32(const_cast<int*>(&st->mma_idle)), 0, 0u, 0};
+    // Bulk stores of whole row blocks unless Linear-2 tiles of this launch wait for h (their release is a plain
+    // fence after plain stores) or the knob switches them off
+    const uint32_t my_box = (chained || !p.bulk_stores) ? 0u : store_u32 + static_cast<uint32_t>(quarter) * kStoreBoxBytes;
+    const StoreStage ss_h{my_box, &tm_h_out}, ss_y{my_box, &tm_y_out};
     bool ok = true;
     while (ok) {
       if (!ptx::mbar_wait(ptx::smem_u32(&st->ring_full[slot]), ring_phase, abort_flag)) {
@@ -873,9 +926,9 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           if (t.phase == 0) drain_swapped<true, kFp8>(t, p, t_addr, r_in_tile);
           else drain_swapped<false, kFp8>(t, p, t_addr, r_in_tile);
         } else if (t.phase == 0) {
-          drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
+          drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag, ss_h);
         } else {
-          drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
+          drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag, ss_y);
         }
         ptx::tc_fence_before_sync();
         if (chained && t.phase == 0) {
@@ -895,6 +948,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       }
       if (t.wide) acc = 0;
     }
+    if (lane == 0) ptx::bulk_wait_group_all();      // this warp's bulk stores have landed
     if (p.trace && warp == 2 && lane == 0) {
       p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
       p.trace[blockIdx.x * kMoeTraceFields + 5] = static_cast<unsigned long long>(busy);
@@ -1163,9 +1217,9 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               static_cast<uint32_t>(acc * BN_ACC);
       if (phase == 0)
-        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
+        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag, StoreStage{0u, nullptr});
       else
-        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag);
+        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag, StoreStage{0u, nullptr});
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(acc ? empty_leader1 : empty_leader0);
@@ -1379,11 +1433,14 @@ cudaError_t launch_pair(moe_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b
 struct FfnMaps {
   CUtensorMap x, wg, wu, h, wd;   // copies: the kernels take them by value
   CUtensorMap x16, h16;           // the two A matrices in boxes of 16 rows (swapped-operand tiles)
+  CUtensorMap h_out, y_out;       // the two outputs (bf16) in boxes of 32 rows (the epilogue's bulk stores)
 };
 
 static void launch_single(int grid, const FfnMaps& m, const FfnParams& p, cudaStream_t stream) {
-  if (p.fp8) expert_ffn_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, m.x16, m.h16, p);
-  else expert_ffn_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, m.x16, m.h16, p);
+  if (p.fp8)
+    expert_ffn_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, m.x16, m.h16, m.h_out, m.y_out, p);
+  else
+    expert_ffn_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(m.x, m.wg, m.wu, m.h, m.wd, m.x16, m.h16, m.h_out, m.y_out, p);
 }
 
 // Everything one expert-FFN call needs on the host side; fp8 selects E4M3 operands with epilogue scales.
@@ -1416,7 +1473,8 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     const bool ok = tensor_map_2d(ctx, c.a1, R, s.H, eb, 128, &m.x) && tensor_map_2d(ctx, c.w_gate, EF, s.H, eb, 128, &m.wg) &&
                     tensor_map_2d(ctx, c.w_up, EF, s.H, eb, 128, &m.wu) && tensor_map_2d(ctx, c.a2, R, s.F, eb, 128, &m.h) &&
                     tensor_map_2d(ctx, c.w_down, EH, s.F, eb, 128, &m.wd) &&
-                    tensor_map_2d(ctx, c.a1, R, s.H, eb, 16, &m.x16) && tensor_map_2d(ctx, c.a2, R, s.F, eb, 16, &m.h16);
+                    tensor_map_2d(ctx, c.a1, R, s.H, eb, 16, &m.x16) && tensor_map_2d(ctx, c.a2, R, s.F, eb, 16, &m.h16) &&
+                    tensor_map_2d(ctx, c.h_bf16, R, s.F, 2, 32, &m.h_out) && tensor_map_2d(ctx, c.y_perm, R, s.H, 2, 32, &m.y_out);
     if (!ok) return MOE_ERR_CUDA;
   }
 
@@ -1451,6 +1509,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   // instead of a 128-row box of mostly other experts' rows: a third less to move per K block; -1 % on the decode-like
   // layer, -0.4 % on the DeepSeek-V3-like one in steady state (larger row counts, several boxes per K block: no gain).
   p.small_a = moe_knob_value(ctx, "small_a", 16);
+  p.bulk_stores = moe_knob_value(ctx, "bulk_stores", 1);
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
   // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
   p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);
