@@ -83,8 +83,9 @@ typedef struct {
                                       status word reads MOE_ERR_TIMEOUT; outputs are then undefined; bit 3: use the
                                       CTA-pair kernel (clusters of two CTAs on 256-row tiles) for two-launch runs; by
                                       default every layer runs the single-CTA kernel, which cuts many-row experts
-                                      into 256-row tiles on its two accumulators; bit 4: accepted, no effect (it
-                                      used to switch the pair kernel off); other bits 0 */
+                                      into 256-row tiles on its two accumulators, except Linear-1 of the FP8 (per-row
+                                      scales) path on layers averaging 1024 rows per expert or more, which runs as
+                                      CTA pairs; bit 4: the single-CTA kernel there as well; other bits 0 */
 } moe_tuning;
 
 /*

@@ -1530,7 +1530,16 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   // there as well (Mixtral-like layer, steady state: -1.6 to -4 % at 8192 tokens, -6 % at 4096, -9 % at 16384; burst
   // equal): it computes an expert's remainder rows as a 128-row or swapped-operand tile instead of a whole 256-row
   // tile, draws tiles dynamically instead of in rounds, and holds a higher SM clock under the power cap.
-  const bool pairs = !one_launch && ctx->max_pairs > 0 && (tn.debug_flags & 8) != 0;
+  // One exception, per GEMM (bit 0 Linear-1, bit 1 Linear-2): with E4M3 operands on a layer averaging 1024 rows per
+  // expert or more, Linear-1 runs as CTA pairs.  Its 128-row tiles (256-row tiles do not pay there, see below) need 96
+  // operand bytes per clock and SM where an SM takes 64, which holds an E4M3 mainloop at two thirds of its rate; a pair
+  // needs 64 (Mixtral-like layer, steady state, alternating runs: Linear-1 1.94 -> 1.77 ms, the step 3.13 -> 2.92 ms;
+  // Linear-2 stays on 256-row tiles: 1.07 against 1.09 ms).  debug_flags bit 4 keeps the single-CTA kernel everywhere.
+  const bool dense = R / static_cast<uint64_t>(s.E) >= 1024;
+  const int pair_phases = !(!one_launch && ctx->max_pairs > 0) ? 0
+                          : (tn.debug_flags & 8)               ? 3
+                          : (c.fp8 && dense && !(tn.debug_flags & 16)) ? moe_knob_value(ctx, "fp8_pair_phases", 1)
+                                                                       : 0;
   unsigned long long* trace2 = trace ? ctx->d_trace + static_cast<size_t>(ctx->num_sms) * kMoeTraceFields : nullptr;
 
   if (one_launch) {
@@ -1560,8 +1569,8 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.phase_hi = 1;
     p.sched = ctx->d_sched;
     p.trace = trace ? ctx->d_trace : nullptr;
-    p.kernel_id = pairs ? 4 : 1;
-    if (pairs) {
+    p.kernel_id = (pair_phases & 1) ? 4 : 1;
+    if (pair_phases & 1) {
       if (launch_pair(ctx, m.x, m.wg, m.wu, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
       launch_single(grid, m, p, stream);
@@ -1575,8 +1584,8 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.phase_hi = 2;
     p.sched = ctx->d_sched + 2;
     p.trace = trace2;
-    p.kernel_id = pairs ? 5 : 2;
-    if (pairs) {
+    p.kernel_id = (pair_phases & 2) ? 5 : 2;
+    if (pair_phases & 2) {
       if (launch_pair(ctx, m.h, m.wd, m.wd, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
       launch_single(grid, m, p, stream);

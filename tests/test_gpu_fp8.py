@@ -116,6 +116,33 @@ def test_fused_forward_fp8_parity(cfg):
     assert rel_fro(dev_bf16_to_f64(out), full["out"]) < 0.08
 
 
+def test_fp8_kernel_choices_give_the_same_bits(monkeypatch):
+    """On a layer of many-row experts Linear-1 runs as CTA pairs by default; the single-CTA kernel everywhere
+    (debug_flags bit 4), CTA pairs for both GEMMs (bit 3) and 128-row tiles only give the same output bits."""
+    cfg = CASES[2]
+    assert cfg.R // cfg.E >= 1024
+    outs = []
+    for env, flags in ((None, 0), (None, 16), (None, 8), ("x.wide_tiles=0", 16), ("x.fp8_pair_phases=3", 0)):
+        if env is None:
+            monkeypatch.delenv("MOE_TUNING", raising=False)
+        else:
+            monkeypatch.setenv("MOE_TUNING", env)
+        L = Layer(cfg)                       # the context reads the variable when it is created
+        ctx = L.ctx
+        wq = []
+        for w in (L.w_gate, L.w_up, L.w_down):
+            E, r, c = w.shape
+            wq.extend(quantize_on_gpu(ctx, w.view(E * r, c)))
+        ws = torch.empty(ctx.workspace_layout_fp8()["total"], dtype=torch.uint8, device=DEV)
+        out = L.nan_bf16(cfg.T, cfg.H)
+        ctx.moe_fused_forward_fp8(L.x, L.d_logits, *wq, out, ws, tuning=binding.make_tuning(debug_flags=flags))
+        torch.cuda.synchronize()
+        L.check_device_status()
+        outs.append(out)
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16))
+
+
 def test_fused_forward_fp8_random_layers():
     """The same checks on random layers: ragged and empty experts, one to thousands of rows per expert."""
     rng = np.random.default_rng(8)
