@@ -16,7 +16,8 @@
 // Stores: an epilogue warp whose 32 rows all belong to the expert packs 64 output columns at a time into a
 // swizzled 4 KiB box of shared memory and one lane hands the box to the TMA unit (whole 128-byte lines, no
 // load/store-unit work per row); a warp with rows of the next expert, a paced run and a launch whose Linear-2 tiles
-// wait for h store 16 bytes per lane and row from registers instead.  Both ways write the same values.
+// wait for h store 16 bytes per lane and row from registers instead.  Both ways write the same values.  The CTA-pair
+// kernel further down stores the same way.
 //
 // Tile orders (moe_tuning.schedule):
 //   0  Expert-Wave: all Linear-1 tiles, then all Linear-2 tiles.  Inside a GEMM the order within an expert is
@@ -1006,7 +1007,8 @@ struct PairTail {
   int32_t pair_prefix[kMaxExperts + 1];   // exclusive prefix of 256-row blocks per expert
   int32_t offs[kMaxExperts + 1];          // the expert row offsets, copied once
 };
-constexpr size_t kPairSmemBytes = 1024 + static_cast<size_t>(kPairStages) * kPairStageBytes + sizeof(PairTail);
+constexpr size_t kPairSmemBytes = 1024 + static_cast<size_t>(kPairStages) * kPairStageBytes + kStoreStagingBytes +
+                                  sizeof(PairTail);   // ring, the epilogue warps' store boxes, tail
 
 __device__ __forceinline__ Tile decode_pair_tile(int tile, int phase, uint32_t rank, const PairTail* st,
                                                  const FfnParams& p) {
@@ -1032,13 +1034,15 @@ __device__ __forceinline__ Tile decode_pair_tile(int tile, int phase, uint32_t r
 template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
-                       const __grid_constant__ CUtensorMap tm_b1, const FfnParams p) {
+                       const __grid_constant__ CUtensorMap tm_b1, const __grid_constant__ CUtensorMap tm_out,
+                       const FfnParams p) {   // tm_out: this GEMM's output in boxes of 32 rows x 64 columns (stores)
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   unsigned char* stage_base = smem_raw + pad;
   const uint32_t stage_u32 = raw + pad;
-  PairTail* st = reinterpret_cast<PairTail*>(stage_base + static_cast<size_t>(kPairStages) * kPairStageBytes);
+  const uint32_t store_u32 = stage_u32 + kPairStages * kPairStageBytes;
+  PairTail* st = reinterpret_cast<PairTail*>(stage_base + static_cast<size_t>(kPairStages) * kPairStageBytes + kStoreStagingBytes);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t rank = ptx::cluster_ctarank();            // 0 = leader (issues the MMAs), 1 = peer
@@ -1206,6 +1210,7 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                 ptx::map_to_cta(ptx::smem_u32(const_cast<int*>(&st->mma_idle)), 0), 0, 0u, 0};
     const uint32_t empty_leader0 = ptx::map_to_cta(ptx::smem_u32(&st->tmem_empty[0]), 0);
     const uint32_t empty_leader1 = ptx::map_to_cta(ptx::smem_u32(&st->tmem_empty[1]), 0);
+    const StoreStage ss{p.bulk_stores ? store_u32 + static_cast<uint32_t>(quarter) * kStoreBoxBytes : 0u, &tm_out};
     for (int tile = pair; tile < total_tiles; tile += pairs) {
       const Tile t = decode_pair_tile(tile, phase, rank, st, p);
       if (!ptx::mbar_wait_timed(ptx::smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, &w_acc)) {
@@ -1217,9 +1222,9 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               static_cast<uint32_t>(acc * BN_ACC);
       if (phase == 0)
-        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag, StoreStage{0u, nullptr});
+        drain_accumulator<true, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag, ss);
       else
-        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag, StoreStage{0u, nullptr});
+        drain_accumulator<false, kFp8>(t, p, t_addr, t.row0 + r_in_tile, pacer, abort_flag, ss);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(acc ? empty_leader1 : empty_leader0);
@@ -1227,6 +1232,7 @@ expert_ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
+    if (lane == 0) ptx::bulk_wait_group_all();      // this warp's bulk stores have landed
     if (p.trace && warp == 2 && lane == 0) {
       p.trace[blockIdx.x * kMoeTraceFields + 4] = static_cast<unsigned long long>(w_acc);
       p.trace[blockIdx.x * kMoeTraceFields + 5] = static_cast<unsigned long long>(busy);
@@ -1412,7 +1418,7 @@ cudaError_t prepare_expert_ffn(moe_ctx* ctx) {
 
 namespace {
 cudaError_t launch_pair(moe_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                        const FfnParams& p, cudaStream_t stream) {
+                        const CUtensorMap& out, const FfnParams& p, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * ctx->max_pairs);
   cfg.blockDim = dim3(kThreads);
@@ -1425,8 +1431,8 @@ cudaError_t launch_pair(moe_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  return p.fp8 ? cudaLaunchKernelEx(&cfg, expert_ffn_pair_kernel<true>, a, b0, b1, p)
-               : cudaLaunchKernelEx(&cfg, expert_ffn_pair_kernel<false>, a, b0, b1, p);
+  return p.fp8 ? cudaLaunchKernelEx(&cfg, expert_ffn_pair_kernel<true>, a, b0, b1, out, p)
+               : cudaLaunchKernelEx(&cfg, expert_ffn_pair_kernel<false>, a, b0, b1, out, p);
 }
 }  // namespace
 
@@ -1571,7 +1577,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.trace = trace ? ctx->d_trace : nullptr;
     p.kernel_id = (pair_phases & 1) ? 4 : 1;
     if (pair_phases & 1) {
-      if (launch_pair(ctx, m.x, m.wg, m.wu, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+      if (launch_pair(ctx, m.x, m.wg, m.wu, m.h_out, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
       launch_single(grid, m, p, stream);
     }
@@ -1586,7 +1592,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.trace = trace2;
     p.kernel_id = (pair_phases & 2) ? 5 : 2;
     if (pair_phases & 2) {
-      if (launch_pair(ctx, m.h, m.wd, m.wd, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+      if (launch_pair(ctx, m.h, m.wd, m.wd, m.y_out, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
       launch_single(grid, m, p, stream);
     }
