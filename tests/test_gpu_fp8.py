@@ -17,6 +17,7 @@ CASES = [
     # about 1000 rows per expert in two launches: below the CTA-pair threshold, so 256-row tiles on both accumulators,
     # with a short swapped-operand or 128-row tile at the end of each expert
     gen.MoEConfig("f8_wide", T=3000, H=512, F=1024, E=6, k=2, seed=94, router="xWr"),
+    gen.MoEConfig("f8_limits", T=70, H=128, F=128, E=1024, k=32, seed=95, router="xWr"),   # the boundary's largest E and k
 ]
 
 

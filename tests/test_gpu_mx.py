@@ -102,6 +102,7 @@ def test_quantize_rows_mx_bits(rows, cols):
     (300, 512, 384, 8, 2, "xWr"),       # several row blocks per expert, ragged tails, whole column tiles
     (129, 256, 640, 16, 4, "xWr_zipf"), # skewed: empty experts, experts of one row
     (5, 384, 256, 6, 6, "xWr"),         # k = E, five rows per expert
+    (70, 128, 128, 1024, 32, "xWr"),    # the boundary's largest E and k
 ])
 @pytest.mark.parametrize("swapped", [True, False], ids=["swapped_small_experts", "128_row_tiles_only"])
 def test_expert_ffn_mx_parity(T, H, F, E, k, router, swapped, monkeypatch):

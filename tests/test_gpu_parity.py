@@ -574,6 +574,31 @@ def test_random_mid_size_layers_property():
         L.check_device_status()
 
 
+def test_largest_expert_count_and_top_k():
+    """E = 1024 experts and k = 32, the limits of the boundary: most experts hold no or a few rows, every kernel
+    variant (default, CTA pairs, one launch, interleaved) gives the default's bits and the oracle's values."""
+    cfg = gen.MoEConfig("limits", T=70, H=128, F=128, E=1024, k=32, seed=301, router="xWr")
+    L = Layer(cfg)
+    ref = oracle_for(L)
+    lay = L.ctx.workspace_layout()
+    ws = torch.empty(lay["total"], dtype=torch.uint8, device=DEV)
+    outs = []
+    for tn in (None, binding.make_tuning(1, 0, 1, debug_flags=8), binding.make_tuning(1, 0, 1, debug_flags=2),
+               binding.make_tuning(1, 0, 1, schedule=1, dep_lead_D=2)):
+        out = L.nan_bf16(cfg.T, cfg.H)
+        L.ctx.moe_fused_forward(L.x, L.d_logits, L.w_gate, L.w_up, L.w_down, out, ws, tuning=tn)
+        torch.cuda.synchronize()
+        outs.append(out)
+    for name in ("counts", "offsets", "perm", "inv_perm"):
+        n = {"counts": cfg.E, "offsets": cfg.E + 1}.get(name, cfg.R)
+        got = ws[lay[name]:lay[name] + 4 * n].view(torch.int32).cpu().numpy()
+        assert np.array_equal(got, np.asarray(ref[name]).reshape(-1)), name
+    assert_out_close(dev_bf16_to_f64(outs[0]), ref["out"], "E=1024, k=32")
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16))
+    L.check_device_status()
+
+
 def test_smaller_batches_on_one_context():
     """A context created for T tokens serves any smaller batch (moe_set_active_tokens), with a workspace sized once."""
     cfg = gen.MoEConfig("varT", T=900, H=256, F=384, E=6, k=2, seed=101, router="xWr")
