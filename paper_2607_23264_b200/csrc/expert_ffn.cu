@@ -35,7 +35,9 @@
 // side and the expert's rows, padded to a multiple of 16, its N side.  A tcgen05.mma costs 128 clocks at N = 256 but
 // 46 at N <= 32, so the two instructions per K step (one per weight box) take 92 clocks instead of 128; the
 // shared-memory stage is the same three boxes, only the MMA issue and the epilogue (lane = output column) differ.
-// A CTA-pair variant (256-row tiles over a cluster of two CTAs, cta_group::2) follows further down; it runs on request.
+// A launch whose experts all hold at most 16 rows runs on six 34 KiB stages (16-row A box + two weight boxes).
+// A CTA-pair variant (256-row tiles over a cluster of two CTAs, cta_group::2) follows further down; it runs on request
+// and for Linear-1 of the E4M3 path on layers of many-row experts.
 #include <cuda_bf16.h>
 
 #include <type_traits>
@@ -59,6 +61,13 @@ constexpr int kStageBytes = kABytes + 2 * kBHalfBytes;   // 48 KiB
 constexpr int kWideStages = 3;
 constexpr int kWideStageBytes = 2 * kABytes + 2 * kBHalfBytes;   // 64 KiB
 static_assert(kWideStages * kWideStageBytes <= kStages * kStageBytes, "the wide ring must fit in the ring's shared memory");
+// A launch whose experts all hold at most 16 rows (decode-like layers): a stage is one 16-row box of A and the two
+// weight boxes, and six of them fit in the ring plus the store boxes such a launch does not use.  These tiles live on
+// the bytes in flight.
+constexpr int kSmallStages = 6;
+constexpr int kSmallABytes = 16 * BK * 2;                          // 2 KiB
+constexpr int kSmallStageBytes = kSmallABytes + 2 * kBHalfBytes;   // 34 KiB
+constexpr int kMaxStages = kSmallStages;
 constexpr int kWideFlag = 1 << 16;   // in the per-tile word next to the tile code: a 256-row tile on both accumulators
 constexpr int kThreads = 192;
 constexpr int kMaxExperts = 1024;
@@ -70,8 +79,8 @@ constexpr int kSwapRows = 64;      // row blocks with at most this many rows (sm
 constexpr int kPhaseShift = 30;    // tile code = phase << 30 | index in the phase's tile list; -1 = no more tiles
 
 struct SharedTail {
-  uint64_t full[kStages];
-  uint64_t empty[kStages];
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint64_t ring_full[kRing];
@@ -83,6 +92,7 @@ struct SharedTail {
   volatile uint32_t mma_progress;   // K-blocks issued so far by the MMA warp (pacing clock)
   volatile int mma_idle;            // 1 while the MMA warp waits for an accumulator or has finished
   int wide;                         // this launch cuts many-row experts into 256-row blocks (wide mode)
+  int small;                        // every expert of this launch holds at most 16 rows: six 34 KiB stages
   int32_t hot_prefix[kMaxExperts + 1];    // exclusive prefix of row blocks over hot experts (cold count 0): 128-row
                                           // blocks, or 256-row blocks in wide mode
   int32_t cold_prefix[kMaxExperts + 1];   // the same over cold experts
@@ -97,6 +107,7 @@ constexpr int kStoreStagingBytes = 4 * kStoreBoxBytes;
 constexpr size_t kSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStages) * kStageBytes + kStoreStagingBytes +
                               sizeof(SharedTail);
 static_assert(kSmemBytes + 64 <= 227 * 1024, "ring + store staging + tail must fit in one CTA's shared memory");
+static_assert(kSmallStages * kSmallStageBytes <= kStages * kStageBytes + kStoreStagingBytes, "the small ring must fit too");
 
 // How one epilogue warp stores: smem == 0 = 16-byte stores from registers (each lane its own row); else the warp
 // stages 32 rows x 64 columns there and one lane hands them to the TMA unit as whole 128-byte lines.
@@ -141,6 +152,7 @@ struct FfnParams {
   int cache_hints;          // L2 eviction priorities of the TMA loads, bit mask (see run_ffn)
   int small_a;              // swapped-operand tiles of at most this many padded rows load A in 16-row boxes (0: never)
   int bulk_stores;          // single-CTA kernel: whole 32-row groups of a tile leave through shared memory and TMA stores
+  int small_ring;           // launches whose experts all hold at most 16 rows use six 34 KiB stages
   int withhold_ready;       // host-requested failure drill: Linear-1 never publishes its rows (one-launch runs)
   long long wait_budget;    // clocks a cross-CTA wait may last before it gives up
   int kernel_id;
@@ -497,7 +509,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       ptx::mbar_init(ptx::smem_u32(&st->full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&st->empty[s]), 1);
     }
@@ -527,15 +539,20 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     // it: at least three 256-row blocks for every four single-block experts.  (Measured in steady state on the
     // DeepSeek-V3-like layer at 1024 to 16384 tokens, where that ratio runs from 0.31 to 3.4: +3 %, -0.7 %, -3.1 %,
     // -5.2 %, -6.3 % with wide mode; the crossover lies near 0.5.)
-    int hot_wide_blocks = 0, cold_blocks = 0;
+    int hot_wide_blocks = 0, cold_blocks = 0, max_rows = 0;
     for (int base = 0; base < p.E; base += 32) {
       const int e = base + lane;
       const int rows = e < p.E ? p.offsets[e + 1] - p.offsets[e] : 0;
       if (rows > BM * (kHotBlocks - 1)) hot_wide_blocks += (rows + 2 * BM - 1) / (2 * BM);
       else if (rows > 0) cold_blocks += 1;
+      max_rows = max(max_rows, rows);
     }
     hot_wide_blocks = __reduce_add_sync(0xFFFFFFFFu, hot_wide_blocks);
     cold_blocks = __reduce_add_sync(0xFFFFFFFFu, cold_blocks);
+    max_rows = __reduce_max_sync(0xFFFFFFFFu, max_rows);
+    // every tile of the launch is then a swapped-operand tile that loads one 16-row box of A
+    if (lane == 0)
+      st->small = (p.small_ring != 0 && max_rows <= 16 && p.small_a >= 16 && p.swap_rows >= 16 && p.schedule == 0) ? 1 : 0;
     // (E4M3 operands: the weight-streaming tiles are a larger share of the time there, and on the same layer wide mode
     // costs 2 % at 4096 tokens; they keep the stricter rule of four 256-row blocks per single-block expert.)
     const bool enough_hot = p.fp8 ? 4 * cold_blocks <= hot_wide_blocks : 3 * cold_blocks <= 4 * hot_wide_blocks;
@@ -589,9 +606,11 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   const uint32_t tmem_base = st->tmem_base;
   // ring geometry of this launch: [A][B0][B1] x 4 stages, or in wide mode [A][A'][B0][B1] x 3 stages
   const bool wide_mode = st->wide != 0;
-  const int n_stages = wide_mode ? kWideStages : kStages;
-  const uint32_t stage_bytes = wide_mode ? kWideStageBytes : kStageBytes;
-  const uint32_t b_off = wide_mode ? 2 * kABytes : kABytes;       // offset of the first weight box inside a stage
+  const bool small_mode = st->small != 0;                          // (never together: wide mode needs many-row experts)
+  const int n_stages = wide_mode ? kWideStages : small_mode ? kSmallStages : kStages;
+  const uint32_t stage_bytes = wide_mode ? kWideStageBytes : small_mode ? kSmallStageBytes : kStageBytes;
+  // offset of the first weight box inside a stage
+  const uint32_t b_off = wide_mode ? 2 * kABytes : small_mode ? kSmallABytes : kABytes;
   const int total_blocks = st->hot_prefix[p.E] + st->cold_prefix[p.E];
   const int tiles1 = p.phase_lo == 0 ? total_blocks * p.ph[0].n_blocks : 0;   // Linear-1 tiles of this launch
   const int tiles2 = p.phase_hi == 2 ? total_blocks * p.ph[1].n_blocks : 0;   // Linear-2 tiles of this launch
@@ -784,7 +803,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           // bubble a branch opens in the issue stream costs as much as three of these instructions; with one wait per
           // two blocks the stand-alone loop goes from 723 to 588 clocks per block).
           int kb = 0;
-          for (; n_stages == kStages && kb + 2 <= k_blocks; kb += 2) {   // (the three-stage ring cannot spare two stages)
+          for (; n_stages >= kStages && kb + 2 <= k_blocks; kb += 2) {   // (the three-stage ring cannot spare two stages)
             const int s0 = stage, s1 = stage + 1 == n_stages ? 0 : stage + 1;
             const uint32_t ph1 = s1 == 0 ? phase ^ 1u : phase;
             const uint32_t bar0 = ptx::smem_u32(&st->full[s0]), bar1 = ptx::smem_u32(&st->full[s1]);
@@ -896,7 +915,9 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     Pacer pacer{ptx::smem_u32(const_cast<uint32_t*>(&st->mma_progress)), ptx::smem_u32(const_cast<int*>(&st->mma_idle)), 0, 0u, 0};
     // Bulk stores of whole row blocks unless Linear-2 tiles of this launch wait for h (their release is a plain
     // fence after plain stores) or the knob switches them off
-    const uint32_t my_box = (chained || !p.bulk_stores) ? 0u : store_u32 + static_cast<uint32_t>(quarter) * kStoreBoxBytes;
+    // (a launch on the small ring has no 128-row tiles, and its ring reaches into the boxes)
+    const uint32_t my_box = (chained || !p.bulk_stores || small_mode) ? 0u
+                                                                      : store_u32 + static_cast<uint32_t>(quarter) * kStoreBoxBytes;
     const StoreStage ss_h{my_box, &tm_h_out}, ss_y{my_box, &tm_y_out};
     bool ok = true;
     while (ok) {
@@ -1516,6 +1537,7 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   // layer, -0.4 % on the DeepSeek-V3-like one in steady state (larger row counts, several boxes per K block: no gain).
   p.small_a = moe_knob_value(ctx, "small_a", 16);
   p.bulk_stores = moe_knob_value(ctx, "bulk_stores", 1);
+  p.small_ring = moe_knob_value(ctx, "small_ring", 1);
   const int grid = ctx->num_sms;   // persistent: one CTA per SM (shared memory allows no second)
   // Algorithm 1's lead; 0 asks for the anti-starvation knee ceil(b_n K_SM / (2 h_inter)) with b_n = 128
   p.lead_D = tn.dep_lead_D > 0 ? tn.dep_lead_D : (128 * grid + 2 * s.F - 1) / (2 * s.F);
