@@ -153,6 +153,8 @@ struct FfnParams {
   int small_a;              // swapped-operand tiles of at most this many padded rows load A in 16-row boxes (0: never)
   int bulk_stores;          // single-CTA kernel: whole 32-row groups of a tile leave through shared memory and TMA stores
   int small_ring;           // launches whose experts all hold at most 16 rows use six 34 KiB stages
+  int expert_class;         // 0: all experts.  A GEMM split into two launches: 1 = the experts of at most 16 rows (all
+                            // experts, if the layer does not hold both kinds), 2 = the others (none, if it does not)
   int withhold_ready;       // host-requested failure drill: Linear-1 never publishes its rows (one-launch runs)
   long long wait_budget;    // clocks a cross-CTA wait may last before it gives up
   int kernel_id;
@@ -539,10 +541,32 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     // it: at least three 256-row blocks for every four single-block experts.  (Measured in steady state on the
     // DeepSeek-V3-like layer at 1024 to 16384 tokens, where that ratio runs from 0.31 to 3.4: +3 %, -0.7 %, -3.1 %,
     // -5.2 %, -6.3 % with wide mode; the crossover lies near 0.5.)
+    // A GEMM split by expert size (every CTA of both launches decides alike from the same counts): the split applies
+    // when the layer holds experts of at most 16 rows and larger ones; otherwise the first launch computes everything
+    // and the second nothing.  take(rows) says whether this launch computes an expert of that many rows.
+    int tiny = 0, larger = 0;
+    if (p.expert_class != 0) {
+      for (int base = 0; base < p.E; base += 32) {
+        const int e = base + lane;
+        const int rows = e < p.E ? p.offsets[e + 1] - p.offsets[e] : 0;
+        tiny += (rows > 0 && rows <= 16) ? 1 : 0;
+        larger += rows > 16 ? 1 : 0;
+      }
+      tiny = __reduce_add_sync(0xFFFFFFFFu, tiny);
+      larger = __reduce_add_sync(0xFFFFFFFFu, larger);
+    }
+    const bool both_kinds = tiny > 0 && larger > 0;
+    const int cls = p.expert_class;
+    auto take = [&](int rows) -> bool {
+      if (cls == 0) return true;
+      if (!both_kinds) return cls == 1;
+      return cls == 1 ? rows <= 16 : rows > 16;
+    };
     int hot_wide_blocks = 0, cold_blocks = 0, max_rows = 0;
     for (int base = 0; base < p.E; base += 32) {
       const int e = base + lane;
-      const int rows = e < p.E ? p.offsets[e + 1] - p.offsets[e] : 0;
+      int rows = e < p.E ? p.offsets[e + 1] - p.offsets[e] : 0;
+      if (!take(rows)) rows = 0;
       if (rows > BM * (kHotBlocks - 1)) hot_wide_blocks += (rows + 2 * BM - 1) / (2 * BM);
       else if (rows > 0) cold_blocks += 1;
       max_rows = max(max_rows, rows);
@@ -568,6 +592,7 @@ expert_ffn_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         const int32_t lo = p.offsets[e], hi = p.offsets[e + 1];
         st->offs[e + 1] = hi;
         rows = hi - lo;
+        if (!take(rows)) rows = 0;          // (an expert of another launch: no blocks here)
         v = (rows + BM - 1) / BM;
       }
       int32_t hot = v >= kHotBlocks ? (wide_mode ? (rows + 2 * BM - 1) / (2 * BM) : v) : 0;
@@ -1591,6 +1616,16 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
   // steady state: 3.07 against 3.18-3.24 ms with both, 3.22-3.23 with Linear-1 only); bf16 gains from both (4.85-4.89
   // against 5.05-5.13 ms with either one alone).
   const int wide_phases = moe_knob_value(ctx, "wide_phases", c.fp8 ? 2 : 3);
+  // Fine-grained bf16 layers (16 to 256 rows per expert on average): each GEMM as two launches, first the experts of
+  // at most 16 rows, which then run on the six-stage ring, then the others (DeepSeek-V3-like layer, steady state,
+  // alternating runs: 4.60 -> 4.53 ms through the bench, 4.52 -> 4.47 through the library alone; with E4M3 operands the
+  // same split costs 2 %, so that path keeps one launch per GEMM).  A layer without both kinds of experts runs its
+  // first launch on everything and its second on nothing.  Not while tracing (one set of counters per GEMM).
+  // (Below 16 rows per expert on average, decode-like layers, larger experts are unlikely and the empty second launch
+  // of each GEMM would cost 1 %.)
+  const uint64_t mean_rows = R / static_cast<uint64_t>(s.E);
+  const bool split_sizes = !trace && !c.fp8 && moe_knob_value(ctx, "split_sizes", 1) != 0 && mean_rows >= 16 &&
+                           mean_rows <= 256;
   if (!second_phase_only) {
     p.wide_allowed = (wide_phases & 1) ? wide_knob : 0;
     p.phase_lo = 0;
@@ -1600,6 +1635,13 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.kernel_id = (pair_phases & 1) ? 4 : 1;
     if (pair_phases & 1) {
       if (launch_pair(ctx, m.x, m.wg, m.wu, m.h_out, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+    } else if (split_sizes) {
+      p.expert_class = 1;
+      launch_single(grid, m, p, stream);
+      p.expert_class = 2;
+      launch_single(grid, m, p, stream);
+      p.expert_class = 0;
+      ctx->last_launches += 1;
     } else {
       launch_single(grid, m, p, stream);
     }
@@ -1615,6 +1657,13 @@ static moe_status run_ffn(moe_ctx* ctx, const FfnCall& c, const int32_t* offsets
     p.kernel_id = (pair_phases & 2) ? 5 : 2;
     if (pair_phases & 2) {
       if (launch_pair(ctx, m.h, m.wd, m.wd, m.y_out, p, stream) != cudaSuccess) return MOE_ERR_CUDA;
+    } else if (split_sizes) {
+      p.expert_class = 1;
+      launch_single(grid, m, p, stream);
+      p.expert_class = 2;
+      launch_single(grid, m, p, stream);
+      p.expert_class = 0;
+      ctx->last_launches += 1;
     } else {
       launch_single(grid, m, p, stream);
     }

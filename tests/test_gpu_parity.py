@@ -257,10 +257,12 @@ def test_environment_override_of_the_default_tuning(monkeypatch):
 def test_development_knobs_do_not_change_values(monkeypatch):
     """The development knobs of MOE_TUNING choose between ways of computing the same tiles (256-row tiles on or off or
     in one GEMM only, swapped operands up to 128 rows, 16-row boxes of A for larger tiles, L2 priorities off, register
-    stores, the four-stage ring for tiny experts, the CTA-pair kernel): every setting gives the bits of the default, on
-    a layer of many-row experts, on a skewed one and on a decode-like one."""
+    stores, the four-stage ring for tiny experts, one launch per GEMM on fine-grained layers, the CTA-pair kernel): every
+    setting gives the bits of the default, on a layer of many-row experts, on a skewed one (250 rows per expert on
+    average, experts of a few rows beside experts of a thousand: its GEMMs run as two launches each by default) and on a
+    decode-like one."""
     settings = ("x.wide_tiles=0", "x.wide_tiles=2", "x.wide_phases=1", "x.wide_phases=2", "x.small_a=64,x.swap_rows=128",
-                "x.small_a=0,x.swap_rows=16", "x.cache_hints=0", "x.bulk_stores=0", "x.small_ring=0", "flags=8")
+                "x.small_a=0,x.swap_rows=16", "x.cache_hints=0", "x.bulk_stores=0", "x.small_ring=0", "x.split_sizes=0", "flags=8")
     for cfg in (gen.MoEConfig("knobs_dense", T=2000, H=512, F=1024, E=6, k=2, seed=91, router="xWr"),
                 gen.MoEConfig("knobs_skew", T=1500, H=512, F=512, E=24, k=4, seed=92, router="xWr_zipf"),
                 # a few rows per expert, two launches: the six-stage ring of 16-row A boxes
